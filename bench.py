@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the RPS synchronisation step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--p 0.1]
+    python bench.py --impl reference ...        # the CPU oracle on the host cores
+
+A step is one pass of the whole hot path (drop masks, local SGD step, masked
+average, masked write-back) over all n replicas.  The metric is replica-params
+synchronised per second, n*d per step.  With N > 1 (torchrun, one rank per GPU)
+every rank runs an independent replica of the job: the path needs no exchange
+between GPUs, so there is no collective on the data path; only the timing is
+reduced (max over ranks).  Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "replica_params_synchronised_per_sec"
+UNIT = "replica-params/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of one fused-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) from
+# the ncu capture summarised under profiles/, keyed by workload; valid only for the kernel
+# sources whose digest is recorded with it.
+NCU_TRAFFIC = {
+    "kernel_digest": None,
+    "bytes_per_launch": {},
+}
+
+
+def kernel_digest() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_1810_07766_b200", "csrc")
+    for name in ("rps_device.cuh", "rps_kernels.cu"):
+        with open(os.path.join(csrc, name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while a region runs."""
+
+    REASONS = {
+        0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+        0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+        0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+    }
+
+    def __init__(self, index: int, period_s: float = 0.002):
+        self.index, self.period = index, period_s
+        self.samples, self.reason_bits = [], 0
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._nvml = None
+
+    def __enter__(self):
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self._nvml = pynvml
+            self._dev = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._dev, pynvml.NVML_CLOCK_SM))
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        except Exception:
+            self._nvml = None
+        return self
+
+    def _reasons(self):
+        nv = self._nvml
+        for fn in ("nvmlDeviceGetCurrentClocksEventReasons", "nvmlDeviceGetCurrentClocksThrottleReasons"):
+            if hasattr(nv, fn):
+                return int(getattr(nv, fn)(self._dev))
+        return 0
+
+    def _run(self):
+        nv = self._nvml
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._dev, nv.NVML_CLOCK_SM)))
+                self.reason_bits |= self._reasons() & ~0x1
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2.0)
+        return False
+
+    def summary(self):
+        reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit]
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------- multi-rank plumbing
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def max_over_ranks(value: float, device=None) -> float:
+    """Largest `value` over all ranks of the default process group (identity without one)."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier():
+    import torch.distributed as dist
+
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.barrier()
+
+
+# ----------------------------------------------------------------------------- the CUDA arm
+
+def timed_steps(torch, stream, fn, device):
+    """Device time of fn() in ms: barrier + synchronize on both sides, events on the launch stream."""
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize(device)
+    start.record(stream)
+    fn()
+    stop.record(stream)
+    torch.cuda.synchronize(device)
+    barrier()
+    return max_over_ranks(start.elapsed_time(stop), device)
+
+
+def oracle_baseline(w, b, seconds_hint="one step"):
+    """The CPU oracle, as it stands, on one full-size step of the workload (single thread)."""
+    import oracle
+    from paper_1810_07766_b200 import workloads as wl
+
+    x = wl.make_initial(w)
+    t0 = time.perf_counter()
+    oracle.step(x, b, dtype=w.dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t=0)
+    dt = time.perf_counter() - t0
+    return {"value": w.n * w.d / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"1 full-size step (n={w.n}, d={w.d}) of the fp64 C oracle, {dt:.2f} s, single thread"}
+
+
+def run_cuda(args):
+    import torch
+
+    from paper_1810_07766_b200 import binding, build
+    from paper_1810_07766_b200 import workloads as wl
+
+    rank, local_rank, world = dist_env()
+    if world != args.gpus:
+        if world == 1 and args.gpus > 1:
+            raise SystemExit("--gpus N > 1 must be launched with torchrun, one rank per GPU")
+        raise SystemExit(f"--gpus {args.gpus} does not match WORLD_SIZE {world}")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path for the product arm")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=device)
+    build.build()
+
+    w = wl.WORKLOADS[args.workload]
+    if args.p is not None:
+        from dataclasses import replace
+
+        w = replace(w, p=args.p)
+    b = wl.make_targets(w)
+    r = binding.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma)
+    r.set_targets(b)
+    stream = r.stream
+    bytes_per_step = w.bytes_per_step
+
+    # pass 1 (untimed for `value`): every launch bracketed by events -> per-kernel durations
+    r.step_n(max(args.warmup, 3))
+    r.profile(True)
+    r.step_n(args.steps)
+    fused_ms, fused_n, mask_ms, mask_n = r.profile_read()
+    r.profile(False)
+
+    # pass 2: W warm-up steps, then exactly K timed steps
+    r.step_n(args.warmup)
+    launches_before = r.launch_count()
+    with ClockSampler(local_rank) as clocks:
+        total_ms = timed_steps(torch, stream, lambda: r.step_n(args.steps), device)
+    gpu_launches = r.launch_count() - launches_before
+
+    # pass 3: end to end through the host-buffer call: H2D of x and b, the step, D2H of x, every step
+    import numpy as np
+
+    tdtype = torch.float32 if w.dtype == "f32" else torch.int16  # bf16 bit patterns travel as 16-bit words
+    x_host = torch.zeros((w.n, w.d), dtype=tdtype).pin_memory()
+    b_host = torch.from_numpy(b if w.dtype == "f32" else b.view(np.int16)).pin_memory()
+    e2e_steps = min(args.steps, args.e2e_steps)
+    for _ in range(2):
+        r.step_host(x_host, b_host)
+    e2e_ms = timed_steps(torch, stream, lambda: [r.step_host(x_host, b_host) for _ in range(e2e_steps)], device)
+    row_bytes = w.n * w.d * w.elem_bytes
+
+    peak, peak_kind = measured_peak_gbs()
+    fused_avg_ms = fused_ms / max(fused_n, 1)
+    achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
+    traffic = None
+    if NCU_TRAFFIC["kernel_digest"] == kernel_digest():
+        traffic = NCU_TRAFFIC["bytes_per_launch"].get(w.name)
+
+    line = {
+        "metric": METRIC, "value": world * w.n * w.d * args.steps / (total_ms * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {
+            "workload": f"{w.name}: n={w.n} workers, d={w.d} {w.dtype}, p={w.p}, gamma={w.gamma}, sigma={w.sigma}, "
+                        f"seed={w.seed}; quadratic objective, b_i ~ N({'mu_i' if w.hetero else '0'},1)",
+            "n": w.n, "d": w.d, "p": w.p, "replicas": "one independent job per GPU, no collective",
+            "l2": "inputs larger than L2 (x and b are %.0f MB each)" % (row_bytes / 1e6),
+            "algorithmic_bytes_per_step": bytes_per_step,
+            "hbm_gbs_whole_step": bytes_per_step / (total_ms / args.steps * 1e-3) / 1e9,
+            "frac_of_8TBs_nominal": bytes_per_step / (total_ms / args.steps * 1e-3) / 8e12,
+        },
+        "clocks": clocks.summary(),
+        "e2e": {"value": world * w.n * w.d * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
+                "h2d_bytes_per_step": 2 * row_bytes, "d2h_bytes_per_step": row_bytes,
+                "call": "rps_step_host (pinned host x and b)"},
+        "gpu_launches": gpu_launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "rps_fused_kernel",
+                     "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n,
+                     "mask_kernel_ms_per_launch": mask_ms / max(mask_n, 1), "mask_launches_timed": mask_n},
+    }
+    r.close()
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = oracle_baseline(w, b)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- the reference arm
+
+def run_reference(args):
+    """The CPU oracle timed on the host: each step is one oracle step over a prefix of the
+    workload's columns (true block and noise indices), sized to keep the run to minutes."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    import numpy as np
+
+    import oracle
+    from paper_1810_07766_b200 import workloads as wl
+
+    w = wl.WORKLOADS[args.workload]
+    if args.p is not None:
+        from dataclasses import replace
+
+        w = replace(w, p=args.p)
+    cols_n = min(w.d, args.reference_columns)
+    sample = wl.Workload(w.name, n=w.n, d=cols_n, dtype=w.dtype, p=w.p, gamma=w.gamma, sigma=w.sigma, seed=w.seed,
+                         steps=w.steps, hetero=w.hetero)
+    b = wl.make_targets(sample)
+    x = wl.make_initial(sample)
+    cols = np.arange(cols_n, dtype=np.int64)
+
+    def one(t):
+        oracle.step_columns(w.d, cols, x, b, dtype=w.dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t=t)
+
+    for t in range(args.warmup):
+        one(t)
+    t0 = time.perf_counter()
+    for t in range(args.warmup, args.warmup + args.steps):
+        one(t)
+    dt = time.perf_counter() - t0
+    value = w.n * cols_n * args.steps / dt
+    sample_txt = f"each step = the first {cols_n} of {w.d} columns, all {w.n} workers, fp64 C oracle, single thread"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name}: n={w.n} workers, d={w.d} {w.dtype}, p={w.p}, gamma={w.gamma}, "
+                               f"sigma={w.sigma}, seed={w.seed}", "sample": sample_txt},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample_txt},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=("cuda", "reference"), default="cuda")
+    ap.add_argument("--workload", choices=("cfg1", "cfg2", "cfg3", "cfg4", "cfg5"), default="cfg2")
+    ap.add_argument("--p", type=float, default=None, help="override the drop probability (p sweeps)")
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--reference-columns", type=int, default=500_000)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args(argv)
+    if args.steps < 1 or args.warmup < 0:
+        raise SystemExit("--steps must be >= 1 and --warmup >= 0")
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,204 @@
+/*
+ * rps.h: C ABI of the RPS synchronisation step on one NVIDIA B200 (sm_100a).
+ *
+ * The library simulates, on one GPU, the unreliable parameter-server step of
+ * centralized SGD from "Distributed Learning over Unreliable Networks"
+ * (Algorithm 1, "RPS"): n workers each hold a full replica x^(i) of a model of
+ * d parameters; the model is cut into n blocks, block j being averaged by one
+ * worker (its server); every worker->server and server->worker message is lost
+ * independently with probability p (Section 3).
+ *
+ * General rules
+ *   - Every function returns RPS_OK (0) or a negative rps_status; nothing throws
+ *     or aborts.  rps_last_error() gives a readable reason for the last failure
+ *     on that handle.
+ *   - "host" pointers are ordinary (preferably pinned) CPU memory, "device"
+ *     pointers are CUDA global memory of the current device.  The library never
+ *     allocates or frees device memory: the caller lends it x, b and a small
+ *     scratch buffer with rps_bind() and keeps ownership.
+ *   - Work is enqueued on the CUDA stream given to rps_bind(); calls that return
+ *     data to the host synchronise that stream first.
+ *   - A handle is not thread-safe; distinct handles are independent.
+ *   - Dense host arrays are row-major [n][d] in the replica type (float, or
+ *     bfloat16 bit patterns in uint16_t).  On the device a row occupies
+ *     rps_pitch() elements (d rounded up so that every row starts on a 128-byte
+ *     boundary); columns d..pitch-1 are padding owned by the library.
+ */
+#ifndef RPS_H
+#define RPS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rps_handle rps_handle;
+
+typedef enum rps_status {
+    RPS_OK = 0,
+    RPS_EINVAL = -1, /* bad argument (range, NULL, alignment, size)          */
+    RPS_ESTATE = -2, /* call not allowed in the handle's current state      */
+    RPS_ECUDA = -3,  /* a CUDA runtime call or kernel launch reported an error */
+    RPS_ENOMEM = -4  /* host allocation failed                               */
+} rps_status;
+
+enum { RPS_MAX_WORKERS = 64 };
+
+/* Replica storage type.  Arithmetic is always fp32 (bf16 replicas are widened
+ * on load, accumulated in fp32, and rounded to nearest-even on store).        */
+typedef enum rps_dtype { RPS_F32 = 0, RPS_BF16 = 1 } rps_dtype;
+
+/* Who averages block j at step t.
+ * RPS_ASSIGN_FIXED: worker j, every step (the simplification of Section 4.1).
+ * RPS_ASSIGN_PERM:  a uniformly random permutation drawn afresh every step, as
+ *                   Algorithm 1 states ("choose one worker b_t^(i) without
+ *                   replacement") and as the lemmas of the supplement assume. */
+typedef enum rps_assign { RPS_ASSIGN_FIXED = 0, RPS_ASSIGN_PERM = 1 } rps_assign;
+
+typedef struct rps_options {
+    int32_t dtype;         /* rps_dtype, default RPS_F32                                   */
+    int32_t assign;        /* rps_assign, default RPS_ASSIGN_FIXED                         */
+    int32_t self_delivery; /* 1 (default): a server's own copy never crosses the network,
+                              so it is always part of the average and the server always has
+                              the average (proof of Lemma 7).  0: all 2n messages of a block
+                              can be lost; a block whose server received nothing is not
+                              broadcast and every worker keeps v for it.                   */
+    int32_t mask_window;   /* drop masks are generated this many steps at a time (1..256,
+                              default 32); does not change any result                     */
+    double sigma;          /* std-dev of the Gaussian gradient noise, default 0           */
+} rps_options;
+
+/*
+ * rps_create: inputs of Algorithm 1 and of the channel model of Section 3.
+ *   n      number of workers = parameter servers = blocks, 1..RPS_MAX_WORKERS
+ *   d      model size, 1 <= d < 2^34
+ *   p      message drop probability, 0 <= p <= 1; a message is lost iff a 32-bit
+ *          Philox4x32-10 draw is below floor(p * 2^32)
+ *   gamma  learning rate (finite); rounded to float once, here
+ *   seed   key of every random stream (masks, server draw, gradient noise)
+ * The new handle starts at step t = 0 with default options; *out is owned by
+ * the library until rps_destroy().  Errors: RPS_EINVAL, RPS_ENOMEM.
+ */
+int rps_create(int n, int64_t d, double p, double gamma, uint64_t seed, rps_handle** out);
+
+/* Frees the handle (NULL is allowed).  Does not touch the caller's buffers.  */
+int rps_destroy(rps_handle* h);
+
+/* Fills *opt with the defaults listed above. */
+int rps_default_options(rps_options* opt);
+
+/* Sets the options; allowed only before rps_bind() (else RPS_ESTATE).        */
+int rps_configure(rps_handle* h, const rps_options* opt);
+
+/* Row pitch, in elements, that x and b must have on the device.              */
+int64_t rps_pitch(const rps_handle* h);
+
+/* Bytes of device scratch (drop masks of mask_window steps) rps_bind() wants. */
+size_t rps_scratch_bytes(const rps_handle* h);
+
+/*
+ * rps_bind: lends the device buffers.
+ *   x_dev, b_dev  [n][pitch] replicas and targets, 128-byte aligned, caller-owned,
+ *                 borrowed until rps_destroy() or the next rps_bind()
+ *   pitch         must equal rps_pitch(h)
+ *   scratch_dev   >= rps_scratch_bytes(h) bytes, 256-byte aligned
+ *   cuda_stream   a cudaStream_t (NULL = the default stream)
+ * Errors: RPS_EINVAL on NULL, misalignment, wrong pitch or short scratch.
+ */
+int rps_bind(rps_handle* h, void* x_dev, void* b_dev, int64_t pitch, void* scratch_dev, size_t scratch_bytes,
+             void* cuda_stream);
+
+/* Copies dense host [n][d] targets b_i of the objective f_i(x) = 0.5*||x - b_i||^2
+ * (worker i's local objective f_i of Eq. 1) to the device.  Asynchronous with
+ * respect to the host only if b_host is pinned.                               */
+int rps_set_targets(rps_handle* h, const void* b_host);
+
+/* Overwrites all replicas from a dense host [n][d] array (Algorithm 1 starts all
+ * workers from the same value; any state is accepted).                        */
+int rps_write(rps_handle* h, const void* x_host);
+
+/* Step counter t of the next rps_step (the first step is t = 0).  Because every
+ * random stream is a pure function of (seed, t, ...), rps_write + rps_set_step
+ * resume a run exactly.                                                       */
+int rps_set_step(rps_handle* h, uint64_t t);
+int rps_get_step(const rps_handle* h, uint64_t* t);
+
+/*
+ * rps_step: one iteration of Algorithm 1 for all workers, enqueued on the stream:
+ *   v^(i)      = x^(i) - gamma * ((x^(i) - b_i) + sigma * xi_t^(i))      local SGD step
+ *   vtilde^(j) = 1/|N^(j)| * sum_{k in N^(j)} v^(k,j)                    Reduce-Scatter
+ *   x^(i,j)    = vtilde^(j) if worker i received it, else v^(i,j)        All-Gather
+ * with N^(j) the workers whose block j reached its server (Section 4.1).  The
+ * drop masks of step t come from the mask kernel (generated mask_window steps at
+ * a time), the rest is one fused kernel that reads x and b once and writes x
+ * once.  Asynchronous; launch errors are returned, execution errors surface at
+ * the next synchronising call.  Needs rps_bind() (else RPS_ESTATE).
+ */
+int rps_step(rps_handle* h);
+
+/* T consecutive rps_step calls. */
+int rps_step_n(rps_handle* h, int64_t T);
+
+/*
+ * rps_step_forced: the same fused kernel with drop masks given by the caller
+ * instead of sampled: bit i of up[j] = worker i's block j reached its server,
+ * bit i of down[j] = worker i received the averaged block j (host arrays of n
+ * words, used as given; a block with up[j] == 0 is not broadcast).  Advances t.
+ * Lets a test enumerate the outcomes behind W_t^(j) of Eq. 3.
+ */
+int rps_step_forced(rps_handle* h, const uint64_t* up, const uint64_t* down);
+
+/*
+ * rps_step_host: one step with host-resident state.  Copies dense host [n][d]
+ * x_host (and b_host unless NULL, in which case the resident targets are used)
+ * to the device, runs rps_step, copies the new replicas back into x_host and
+ * synchronises.  Pinned host memory makes the copies fast; pageable works.
+ */
+int rps_step_host(rps_handle* h, void* x_host, const void* b_host);
+
+/* Synchronises and copies the replicas to a dense host [n][d] array.          */
+int rps_read(rps_handle* h, void* x_host_out);
+
+/*
+ * rps_read_masks: runs the device mask generator for step t (any t; does not
+ * disturb the run) and returns, for each block j: up[j], down[j] as above,
+ * count[j] = |N^(j)|, server[j] = the worker that averages block j.  Host arrays
+ * of n entries; server may be NULL.
+ */
+int rps_read_masks(rps_handle* h, uint64_t t, uint64_t* up, uint64_t* down, int32_t* count, int32_t* server);
+
+/*
+ * rps_diag: off the hot path.  dist2_to_opt = ||xbar - mean_i b_i||^2 (squared
+ * distance of the averaged model to the optimum of the quadratic objective) and
+ * consensus = sum_i ||x^(i) - xbar||^2 (the quantity bounded by Lemma 3).
+ * Synchronises.  Either output may be NULL.
+ */
+int rps_diag(rps_handle* h, double* dist2_to_opt, double* consensus);
+
+/*
+ * Per-kernel device timing.  rps_profile(h, 1) makes every later kernel launch of
+ * this handle be bracketed by CUDA events on the bound stream; rps_profile_read
+ * synchronises and returns the summed device time and launch count of the fused
+ * step kernel and of the mask kernel since profiling was switched on, then
+ * resets them.  rps_profile(h, 0) switches it off.
+ */
+int rps_profile(rps_handle* h, int enable);
+int rps_profile_read(rps_handle* h, double* fused_ms, int64_t* fused_launches, double* mask_ms,
+                     int64_t* mask_launches);
+
+/* Kernels launched by this handle since creation (both kinds).               */
+int64_t rps_launch_count(const rps_handle* h);
+
+/* Reason for the last failure on h ("" if none); valid until the next call.
+ * With h == NULL: reason for the last failed rps_create on this thread.       */
+const char* rps_last_error(const rps_handle* h);
+
+/* Library version, "major.minor". */
+const char* rps_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RPS_H */

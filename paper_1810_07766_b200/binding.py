@@ -1,0 +1,242 @@
+"""ctypes binding of ``librps.so`` (the C ABI declared in ``include/rps.h``).
+
+Argument marshalling only: every step of the method runs in the CUDA kernels of
+the library.  PyTorch supplies device memory and the stream, nothing else.
+There is no CPU fallback: a missing library or a failing call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+import torch
+
+_CSRC = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc")
+LIB_PATH = os.path.join(_CSRC, "librps.so")
+
+RPS_OK, RPS_EINVAL, RPS_ESTATE, RPS_ECUDA, RPS_ENOMEM = 0, -1, -2, -3, -4
+RPS_F32, RPS_BF16 = 0, 1
+RPS_ASSIGN_FIXED, RPS_ASSIGN_PERM = 0, 1
+_DTYPE = {"f32": RPS_F32, "bf16": RPS_BF16}
+
+# every symbol include/rps.h declares
+SYMBOLS = (
+    "rps_create", "rps_destroy", "rps_default_options", "rps_configure", "rps_pitch", "rps_scratch_bytes",
+    "rps_bind", "rps_set_targets", "rps_write", "rps_set_step", "rps_get_step", "rps_step", "rps_step_n",
+    "rps_step_forced", "rps_step_host", "rps_read", "rps_read_masks", "rps_diag", "rps_profile",
+    "rps_profile_read", "rps_launch_count", "rps_last_error", "rps_version",
+)
+
+
+class rps_options(ctypes.Structure):
+    _fields_ = [("dtype", ctypes.c_int32), ("assign", ctypes.c_int32), ("self_delivery", ctypes.c_int32),
+                ("mask_window", ctypes.c_int32), ("sigma", ctypes.c_double)]
+
+
+class RPSError(RuntimeError):
+    def __init__(self, code: int, where: str, why: str):
+        super().__init__(f"{where} failed with status {code}: {why}")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(path):
+        raise FileNotFoundError(
+            f"{path} is missing: build it with `python -m paper_1810_07766_b200.build` (needs nvcc)")
+    lib = ctypes.CDLL(path)
+    vp, i64, u64, dbl, cint = ctypes.c_void_p, ctypes.c_int64, ctypes.c_uint64, ctypes.c_double, ctypes.c_int
+    u64p, i32p, i64p, dblp = (ctypes.POINTER(t) for t in (u64, ctypes.c_int32, i64, dbl))
+    sig = {
+        "rps_create": (cint, [cint, i64, dbl, dbl, u64, ctypes.POINTER(vp)]),
+        "rps_destroy": (cint, [vp]),
+        "rps_default_options": (cint, [ctypes.POINTER(rps_options)]),
+        "rps_configure": (cint, [vp, ctypes.POINTER(rps_options)]),
+        "rps_pitch": (i64, [vp]),
+        "rps_scratch_bytes": (ctypes.c_size_t, [vp]),
+        "rps_bind": (cint, [vp, vp, vp, i64, vp, ctypes.c_size_t, vp]),
+        "rps_set_targets": (cint, [vp, vp]),
+        "rps_write": (cint, [vp, vp]),
+        "rps_set_step": (cint, [vp, u64]),
+        "rps_get_step": (cint, [vp, u64p]),
+        "rps_step": (cint, [vp]),
+        "rps_step_n": (cint, [vp, i64]),
+        "rps_step_forced": (cint, [vp, u64p, u64p]),
+        "rps_step_host": (cint, [vp, vp, vp]),
+        "rps_read": (cint, [vp, vp]),
+        "rps_read_masks": (cint, [vp, u64, u64p, u64p, i32p, i32p]),
+        "rps_diag": (cint, [vp, dblp, dblp]),
+        "rps_profile": (cint, [vp, cint]),
+        "rps_profile_read": (cint, [vp, dblp, i64p, dblp, i64p]),
+        "rps_launch_count": (i64, [vp]),
+        "rps_last_error": (ctypes.c_char_p, [vp]),
+        "rps_version": (ctypes.c_char_p, []),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    _lib = lib
+    return lib
+
+
+def _host_ptr(a) -> int:
+    """Address of a dense host array given as numpy array or CPU torch tensor."""
+    if isinstance(a, torch.Tensor):
+        if a.is_cuda or not a.is_contiguous():
+            raise ValueError("expected a contiguous CPU tensor")
+        return a.data_ptr()
+    if not a.flags.c_contiguous:
+        raise ValueError("expected a C-contiguous array")
+    return a.ctypes.data
+
+
+class RPS:
+    """One simulated cluster of ``n`` workers and ``n`` parameter servers on the current GPU.
+
+    Method names follow the C ABI (``rps_step`` -> ``step`` and so on).
+    """
+
+    def __init__(self, n: int, d: int, p: float, gamma: float, seed: int, *, dtype: str = "f32", sigma: float = 0.0,
+                 assign: int = RPS_ASSIGN_FIXED, self_delivery: bool = True, mask_window: int = 32,
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        if not torch.cuda.is_available():
+            raise RuntimeError("the RPS library needs a CUDA device; there is no CPU path")
+        self.n, self.d, self.dtype = int(n), int(d), dtype
+        rc = self._lib.rps_create(n, d, p, gamma, seed, ctypes.byref(self._h))
+        if rc != RPS_OK:
+            raise RPSError(rc, "rps_create", self._lib.rps_last_error(None).decode())
+        opt = rps_options()
+        self._lib.rps_default_options(ctypes.byref(opt))
+        opt.dtype, opt.assign, opt.self_delivery = _DTYPE[dtype], assign, int(self_delivery)
+        opt.mask_window, opt.sigma = mask_window, sigma
+        self._check(self._lib.rps_configure(self._h, ctypes.byref(opt)), "rps_configure")
+        self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        self.pitch = int(self._lib.rps_pitch(self._h))
+        tdtype = torch.float32 if dtype == "f32" else torch.bfloat16
+        with torch.cuda.device(self.device):
+            # device memory comes from torch; the library only borrows it
+            self.x_dev = torch.zeros((n, self.pitch), dtype=tdtype, device=self.device)
+            self.b_dev = torch.zeros((n, self.pitch), dtype=tdtype, device=self.device)
+            self.scratch = torch.zeros(int(self._lib.rps_scratch_bytes(self._h)) + 256, dtype=torch.uint8,
+                                       device=self.device)
+            self.stream = torch.cuda.current_stream(self.device) if stream is None else stream
+            scratch_ptr = (self.scratch.data_ptr() + 255) // 256 * 256
+            self._check(self._lib.rps_bind(self._h, self.x_dev.data_ptr(), self.b_dev.data_ptr(), self.pitch,
+                                           scratch_ptr, self.scratch.numel() - (scratch_ptr - self.scratch.data_ptr()),
+                                           self.stream.cuda_stream), "rps_bind")
+
+    # ------------------------------------------------------------------ plumbing
+    def _check(self, rc: int, where: str) -> None:
+        if rc != RPS_OK:
+            raise RPSError(rc, where, self._lib.rps_last_error(self._h).decode())
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            torch.cuda.synchronize(self.device)
+            self._lib.rps_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _host_array(self) -> np.ndarray:
+        return np.empty((self.n, self.d), dtype=np.float32 if self.dtype == "f32" else np.uint16)
+
+    def _expect(self, a, name: str) -> None:
+        want = (self.n, self.d)
+        if tuple(a.shape) != want:
+            raise ValueError(f"{name} must have shape {want}")
+        size = a.element_size() if isinstance(a, torch.Tensor) else a.dtype.itemsize
+        if size != (4 if self.dtype == "f32" else 2):
+            raise ValueError(f"{name} has the wrong element size for {self.dtype} replicas")
+
+    # ------------------------------------------------------------------ C ABI, one method per call
+    def set_targets(self, b_host) -> None:
+        self._expect(b_host, "b_host")
+        self._check(self._lib.rps_set_targets(self._h, _host_ptr(b_host)), "rps_set_targets")
+
+    def write(self, x_host) -> None:
+        self._expect(x_host, "x_host")
+        self._check(self._lib.rps_write(self._h, _host_ptr(x_host)), "rps_write")
+
+    def set_step(self, t: int) -> None:
+        self._check(self._lib.rps_set_step(self._h, t), "rps_set_step")
+
+    def get_step(self) -> int:
+        t = ctypes.c_uint64()
+        self._check(self._lib.rps_get_step(self._h, ctypes.byref(t)), "rps_get_step")
+        return t.value
+
+    def step(self) -> None:
+        self._check(self._lib.rps_step(self._h), "rps_step")
+
+    def step_n(self, steps: int) -> None:
+        self._check(self._lib.rps_step_n(self._h, steps), "rps_step_n")
+
+    def step_forced(self, up, down) -> None:
+        up = np.ascontiguousarray(up, dtype=np.uint64)
+        down = np.ascontiguousarray(down, dtype=np.uint64)
+        if up.shape != (self.n,) or down.shape != (self.n,):
+            raise ValueError("masks must have n entries")
+        u64p = ctypes.POINTER(ctypes.c_uint64)
+        self._check(self._lib.rps_step_forced(self._h, up.ctypes.data_as(u64p), down.ctypes.data_as(u64p)),
+                    "rps_step_forced")
+
+    def step_host(self, x_host, b_host=None) -> None:
+        self._expect(x_host, "x_host")
+        if b_host is not None:
+            self._expect(b_host, "b_host")
+        self._check(self._lib.rps_step_host(self._h, _host_ptr(x_host), None if b_host is None else _host_ptr(b_host)),
+                    "rps_step_host")
+
+    def read(self, out=None):
+        out = self._host_array() if out is None else out
+        self._expect(out, "out")
+        self._check(self._lib.rps_read(self._h, _host_ptr(out)), "rps_read")
+        return out
+
+    def read_masks(self, t: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+        up = np.zeros(self.n, dtype=np.uint64)
+        down = np.zeros(self.n, dtype=np.uint64)
+        cnt = np.zeros(self.n, dtype=np.int32)
+        server = np.zeros(self.n, dtype=np.int32)
+        u64p, i32p = ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_int32)
+        self._check(self._lib.rps_read_masks(self._h, t, up.ctypes.data_as(u64p), down.ctypes.data_as(u64p),
+                                             cnt.ctypes.data_as(i32p), server.ctypes.data_as(i32p)), "rps_read_masks")
+        return up, down, cnt, server
+
+    def diag(self) -> Tuple[float, float]:
+        a, c = ctypes.c_double(), ctypes.c_double()
+        self._check(self._lib.rps_diag(self._h, ctypes.byref(a), ctypes.byref(c)), "rps_diag")
+        return a.value, c.value
+
+    def profile(self, enable: bool) -> None:
+        self._check(self._lib.rps_profile(self._h, int(enable)), "rps_profile")
+
+    def profile_read(self):
+        """(fused_ms, fused_launches, mask_ms, mask_launches) since profiling was enabled; resets them."""
+        fm, mm = ctypes.c_double(), ctypes.c_double()
+        fl, ml = ctypes.c_int64(), ctypes.c_int64()
+        self._check(self._lib.rps_profile_read(self._h, ctypes.byref(fm), ctypes.byref(fl), ctypes.byref(mm),
+                                               ctypes.byref(ml)), "rps_profile_read")
+        return fm.value, fl.value, mm.value, ml.value
+
+    def launch_count(self) -> int:
+        return int(self._lib.rps_launch_count(self._h))
+
+
+def version() -> str:
+    return load_library().rps_version().decode()

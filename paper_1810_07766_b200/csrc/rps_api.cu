@@ -1,0 +1,479 @@
+// C ABI of the RPS library (see include/rps.h): argument checks, the step
+// counter, the window of pre-generated drop masks, copies between dense host
+// arrays and the pitched device layout, and per-kernel event timing.
+#include "rps.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "rps_device.cuh"
+#include "rps_kernels.h"
+
+static_assert(sizeof(rps::StepMasks) == rps::kStepMasksBytes, "mask record layout");
+
+namespace {
+
+constexpr size_t kDiagBytes = 256;  // two fp64 accumulators, padded
+thread_local std::string g_create_error;
+
+struct TimedLaunch {
+    cudaEvent_t start, stop;
+    int kind;  // 0 fused, 1 mask
+};
+
+}  // namespace
+
+struct rps_handle {
+    int n = 0;
+    int64_t d = 0;
+    double p = 0.0;
+    float gamma = 0.0f;
+    float sigma = 0.0f;
+    uint64_t seed = 0;
+    rps_options opt{};
+    // binding
+    bool bound = false;
+    void* x = nullptr;
+    void* b = nullptr;
+    unsigned char* scratch = nullptr;
+    cudaStream_t stream = nullptr;
+    int sm_count = 0;
+    // run state
+    uint64_t t = 0;
+    bool window_valid = false;
+    uint64_t window_t0 = 0;
+    int64_t launches = 0;
+    // timing
+    bool profiling = false;
+    std::vector<TimedLaunch> pending;
+    double ms[2] = {0.0, 0.0};
+    int64_t timed[2] = {0, 0};
+    rps::StepMasks staged{};  // host copy of caller-given masks
+    std::string error;
+
+    size_t elem() const { return opt.dtype == RPS_BF16 ? 2 : 4; }
+    int64_t pitch() const
+    {
+        const int64_t per_line = 128 / (int64_t)elem();
+        return (d + per_line - 1) / per_line * per_line;
+    }
+    double* diag_acc() const { return reinterpret_cast<double*>(scratch); }
+    rps::StepMasks* window() const { return reinterpret_cast<rps::StepMasks*>(scratch + kDiagBytes); }
+    rps::StepMasks* probe() const { return window() + opt.mask_window; }
+    rps::StepMasks* forced() const { return window() + opt.mask_window + 1; }
+    size_t scratch_bytes() const { return kDiagBytes + (size_t)(opt.mask_window + 2) * sizeof(rps::StepMasks); }
+};
+
+namespace {
+
+int fail(rps_handle* h, int code, const std::string& why)
+{
+    if (h) h->error = why;
+    return code;
+}
+
+int cuda_fail(rps_handle* h, const char* what, cudaError_t err)
+{
+    return fail(h, RPS_ECUDA, std::string(what) + ": " + cudaGetErrorString(err));
+}
+
+#define RPS_CUDA(h, call)                                         \
+    do {                                                          \
+        cudaError_t err__ = (call);                               \
+        if (err__ != cudaSuccess) return cuda_fail(h, #call, err__); \
+    } while (0)
+
+int need_bound(rps_handle* h)
+{
+    if (!h) return RPS_EINVAL;
+    if (!h->bound) return fail(h, RPS_ESTATE, "rps_bind has not been called");
+    return RPS_OK;
+}
+
+int flush_timing(rps_handle* h)
+{
+    if (h->pending.empty()) return RPS_OK;
+    RPS_CUDA(h, cudaStreamSynchronize(h->stream));
+    for (TimedLaunch& tl : h->pending) {
+        float ms = 0.0f;
+        cudaError_t err = cudaEventElapsedTime(&ms, tl.start, tl.stop);
+        cudaEventDestroy(tl.start);
+        cudaEventDestroy(tl.stop);
+        if (err != cudaSuccess) {
+            h->pending.clear();
+            return cuda_fail(h, "cudaEventElapsedTime", err);
+        }
+        h->ms[tl.kind] += ms;
+        h->timed[tl.kind] += 1;
+    }
+    h->pending.clear();
+    return RPS_OK;
+}
+
+// Runs `launch` on the stream; when profiling, brackets it with events.
+template <typename Launch>
+int timed_launch(rps_handle* h, int kind, Launch launch)
+{
+    TimedLaunch tl{nullptr, nullptr, kind};
+    if (h->profiling) {
+        if (h->pending.size() >= 2048) {
+            int rc = flush_timing(h);
+            if (rc != RPS_OK) return rc;
+        }
+        RPS_CUDA(h, cudaEventCreate(&tl.start));
+        RPS_CUDA(h, cudaEventCreate(&tl.stop));
+        RPS_CUDA(h, cudaEventRecord(tl.start, h->stream));
+    }
+    cudaError_t err = launch();
+    if (err != cudaSuccess) return cuda_fail(h, kind == 0 ? "fused step kernel launch" : "mask kernel launch", err);
+    h->launches += 1;
+    if (h->profiling) {
+        RPS_CUDA(h, cudaEventRecord(tl.stop, h->stream));
+        h->pending.push_back(tl);
+    }
+    return RPS_OK;
+}
+
+int generate_masks(rps_handle* h, rps::StepMasks* out, uint64_t t0, int steps)
+{
+    rps::MaskParams prm{};
+    prm.out = out;
+    prm.t0 = t0;
+    prm.drop_threshold = (uint64_t)std::floor(h->p * 4294967296.0);
+    prm.key0 = (uint32_t)h->seed;
+    prm.key1 = (uint32_t)(h->seed >> 32);
+    prm.n = h->n;
+    prm.self_delivery = h->opt.self_delivery;
+    prm.assign_perm = h->opt.assign == RPS_ASSIGN_PERM;
+    return timed_launch(h, 1, [&] { return rps::launch_masks(prm, steps, h->stream); });
+}
+
+int run_fused(rps_handle* h, const rps::StepMasks* masks)
+{
+    rps::FusedParams prm{};
+    prm.x = h->x;
+    prm.b = h->b;
+    prm.masks = masks;
+    prm.pitch = h->pitch();
+    prm.d = h->d;
+    prm.block_cols = (h->d + h->n - 1) / h->n;
+    prm.n = h->n;
+    prm.narrow = h->d < ((int64_t)1 << 31);
+    prm.gamma = h->gamma;
+    prm.sigma = h->sigma;
+    prm.t_lo = (uint32_t)h->t;
+    prm.t_hi = (uint32_t)(h->t >> 32);
+    prm.key0 = (uint32_t)h->seed;
+    prm.key1 = (uint32_t)(h->seed >> 32);
+    int rc = timed_launch(h, 0, [&] { return rps::launch_fused(prm, h->opt.dtype == RPS_BF16, h->sm_count, h->stream); });
+    if (rc == RPS_OK) h->t += 1;
+    return rc;
+}
+
+int copy_rows(rps_handle* h, void* dst, size_t dst_pitch_bytes, const void* src, size_t src_pitch_bytes,
+              cudaMemcpyKind kind)
+{
+    const size_t row_bytes = (size_t)h->d * h->elem();
+    if (dst_pitch_bytes < ((size_t)1 << 31) && src_pitch_bytes < ((size_t)1 << 31)) {
+        RPS_CUDA(h, cudaMemcpy2DAsync(dst, dst_pitch_bytes, src, src_pitch_bytes, row_bytes, (size_t)h->n, kind,
+                                      h->stream));
+        return RPS_OK;
+    }
+    // rows longer than the 2-D copy's pitch limit: one copy per worker
+    for (int i = 0; i < h->n; ++i)
+        RPS_CUDA(h, cudaMemcpyAsync(static_cast<char*>(dst) + (size_t)i * dst_pitch_bytes,
+                                    static_cast<const char*>(src) + (size_t)i * src_pitch_bytes, row_bytes, kind,
+                                    h->stream));
+    return RPS_OK;
+}
+
+int upload(rps_handle* h, void* dev, const void* host)
+{
+    return copy_rows(h, dev, (size_t)h->pitch() * h->elem(), host, (size_t)h->d * h->elem(), cudaMemcpyHostToDevice);
+}
+
+int download(rps_handle* h, void* host, const void* dev)
+{
+    return copy_rows(h, host, (size_t)h->d * h->elem(), dev, (size_t)h->pitch() * h->elem(), cudaMemcpyDeviceToHost);
+}
+
+}  // namespace
+
+extern "C" {
+
+int rps_default_options(rps_options* opt)
+{
+    if (!opt) return RPS_EINVAL;
+    opt->dtype = RPS_F32;
+    opt->assign = RPS_ASSIGN_FIXED;
+    opt->self_delivery = 1;
+    opt->mask_window = 32;
+    opt->sigma = 0.0;
+    return RPS_OK;
+}
+
+int rps_create(int n, int64_t d, double p, double gamma, uint64_t seed, rps_handle** out)
+{
+    if (!out) {
+        g_create_error = "out is NULL";
+        return RPS_EINVAL;
+    }
+    *out = nullptr;
+    if (n < 1 || n > RPS_MAX_WORKERS) {
+        g_create_error = "n must be in 1..64";
+        return RPS_EINVAL;
+    }
+    if (d < 1 || d >= ((int64_t)1 << 34)) {
+        g_create_error = "d must be in 1..2^34-1";
+        return RPS_EINVAL;
+    }
+    if (!(p >= 0.0 && p <= 1.0)) {
+        g_create_error = "p must be in [0, 1]";
+        return RPS_EINVAL;
+    }
+    if (!std::isfinite(gamma)) {
+        g_create_error = "gamma must be finite";
+        return RPS_EINVAL;
+    }
+    rps_handle* h = new (std::nothrow) rps_handle();
+    if (!h) {
+        g_create_error = "out of host memory";
+        return RPS_ENOMEM;
+    }
+    h->n = n;
+    h->d = d;
+    h->p = p;
+    h->gamma = (float)gamma;
+    h->seed = seed;
+    rps_default_options(&h->opt);
+    *out = h;
+    return RPS_OK;
+}
+
+int rps_destroy(rps_handle* h)
+{
+    if (!h) return RPS_OK;
+    for (TimedLaunch& tl : h->pending) {
+        cudaEventDestroy(tl.start);
+        cudaEventDestroy(tl.stop);
+    }
+    delete h;
+    return RPS_OK;
+}
+
+int rps_configure(rps_handle* h, const rps_options* opt)
+{
+    if (!h) return RPS_EINVAL;
+    if (!opt) return fail(h, RPS_EINVAL, "options are NULL");
+    if (h->bound) return fail(h, RPS_ESTATE, "options cannot change after rps_bind");
+    if (opt->dtype != RPS_F32 && opt->dtype != RPS_BF16) return fail(h, RPS_EINVAL, "unknown dtype");
+    if (opt->assign != RPS_ASSIGN_FIXED && opt->assign != RPS_ASSIGN_PERM) return fail(h, RPS_EINVAL, "unknown assign");
+    if (opt->self_delivery != 0 && opt->self_delivery != 1) return fail(h, RPS_EINVAL, "self_delivery must be 0 or 1");
+    if (opt->mask_window < 1 || opt->mask_window > 256) return fail(h, RPS_EINVAL, "mask_window must be in 1..256");
+    if (!std::isfinite(opt->sigma) || opt->sigma < 0.0) return fail(h, RPS_EINVAL, "sigma must be finite and >= 0");
+    h->opt = *opt;
+    h->sigma = (float)opt->sigma;
+    return RPS_OK;
+}
+
+int64_t rps_pitch(const rps_handle* h) { return h ? h->pitch() : (int64_t)RPS_EINVAL; }
+
+size_t rps_scratch_bytes(const rps_handle* h) { return h ? h->scratch_bytes() : 0; }
+
+int rps_bind(rps_handle* h, void* x_dev, void* b_dev, int64_t pitch, void* scratch_dev, size_t scratch_bytes,
+             void* cuda_stream)
+{
+    if (!h) return RPS_EINVAL;
+    if (!x_dev || !b_dev || !scratch_dev) return fail(h, RPS_EINVAL, "a device pointer is NULL");
+    if (((uintptr_t)x_dev | (uintptr_t)b_dev) % 128 != 0) return fail(h, RPS_EINVAL, "x and b must be 128-byte aligned");
+    if ((uintptr_t)scratch_dev % 256 != 0) return fail(h, RPS_EINVAL, "scratch must be 256-byte aligned");
+    if (pitch != h->pitch()) return fail(h, RPS_EINVAL, "pitch must equal rps_pitch()");
+    if (scratch_bytes < h->scratch_bytes()) return fail(h, RPS_EINVAL, "scratch is smaller than rps_scratch_bytes()");
+    int dev = 0;
+    RPS_CUDA(h, cudaGetDevice(&dev));
+    RPS_CUDA(h, cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, dev));
+    h->x = x_dev;
+    h->b = b_dev;
+    h->scratch = static_cast<unsigned char*>(scratch_dev);
+    h->stream = static_cast<cudaStream_t>(cuda_stream);
+    h->bound = true;
+    h->window_valid = false;
+    return RPS_OK;
+}
+
+int rps_set_targets(rps_handle* h, const void* b_host)
+{
+    int rc = need_bound(h);
+    if (rc != RPS_OK) return rc;
+    if (!b_host) return fail(h, RPS_EINVAL, "b_host is NULL");
+    return upload(h, h->b, b_host);
+}
+
+int rps_write(rps_handle* h, const void* x_host)
+{
+    int rc = need_bound(h);
+    if (rc != RPS_OK) return rc;
+    if (!x_host) return fail(h, RPS_EINVAL, "x_host is NULL");
+    return upload(h, h->x, x_host);
+}
+
+int rps_set_step(rps_handle* h, uint64_t t)
+{
+    if (!h) return RPS_EINVAL;
+    h->t = t;
+    return RPS_OK;
+}
+
+int rps_get_step(const rps_handle* h, uint64_t* t)
+{
+    if (!h || !t) return RPS_EINVAL;
+    *t = h->t;
+    return RPS_OK;
+}
+
+int rps_step(rps_handle* h)
+{
+    int rc = need_bound(h);
+    if (rc != RPS_OK) return rc;
+    const uint64_t window = (uint64_t)h->opt.mask_window;
+    if (!h->window_valid || h->t < h->window_t0 || h->t - h->window_t0 >= window) {
+        rc = generate_masks(h, h->window(), h->t, (int)window);
+        if (rc != RPS_OK) return rc;
+        h->window_valid = true;
+        h->window_t0 = h->t;
+    }
+    return run_fused(h, h->window() + (h->t - h->window_t0));
+}
+
+int rps_step_n(rps_handle* h, int64_t T)
+{
+    if (h && T < 0) return fail(h, RPS_EINVAL, "T is negative");
+    for (int64_t k = 0; k < T; ++k) {
+        int rc = rps_step(h);
+        if (rc != RPS_OK) return rc;
+    }
+    return h ? RPS_OK : RPS_EINVAL;
+}
+
+int rps_step_forced(rps_handle* h, const uint64_t* up, const uint64_t* down)
+{
+    int rc = need_bound(h);
+    if (rc != RPS_OK) return rc;
+    if (!up || !down) return fail(h, RPS_EINVAL, "a mask array is NULL");
+    const uint64_t valid = h->n == 64 ? ~(uint64_t)0 : (((uint64_t)1 << h->n) - 1);
+    std::memset(&h->staged, 0, sizeof h->staged);
+    for (int j = 0; j < h->n; ++j) {
+        if ((up[j] | down[j]) & ~valid) return fail(h, RPS_EINVAL, "a mask has a bit set for a worker >= n");
+        int cnt = 0;
+        for (int i = 0; i < h->n; ++i) cnt += (int)((up[j] >> i) & 1);
+        h->staged.up[j] = up[j];
+        h->staged.down[j] = cnt > 0 ? down[j] : 0;
+        h->staged.cnt[j] = cnt;
+        h->staged.server[j] = j;
+    }
+    // `staged` is pageable, so the copy has left it when the call returns; on the device the
+    // copy is ordered after the previous step's kernel by the stream
+    RPS_CUDA(h, cudaMemcpyAsync(h->forced(), &h->staged, sizeof h->staged, cudaMemcpyHostToDevice, h->stream));
+    return run_fused(h, h->forced());
+}
+
+int rps_step_host(rps_handle* h, void* x_host, const void* b_host)
+{
+    int rc = need_bound(h);
+    if (rc != RPS_OK) return rc;
+    if (!x_host) return fail(h, RPS_EINVAL, "x_host is NULL");
+    if ((rc = upload(h, h->x, x_host)) != RPS_OK) return rc;
+    if (b_host && (rc = upload(h, h->b, b_host)) != RPS_OK) return rc;
+    if ((rc = rps_step(h)) != RPS_OK) return rc;
+    if ((rc = download(h, x_host, h->x)) != RPS_OK) return rc;
+    RPS_CUDA(h, cudaStreamSynchronize(h->stream));
+    return RPS_OK;
+}
+
+int rps_read(rps_handle* h, void* x_host_out)
+{
+    int rc = need_bound(h);
+    if (rc != RPS_OK) return rc;
+    if (!x_host_out) return fail(h, RPS_EINVAL, "x_host_out is NULL");
+    if ((rc = download(h, x_host_out, h->x)) != RPS_OK) return rc;
+    RPS_CUDA(h, cudaStreamSynchronize(h->stream));
+    return RPS_OK;
+}
+
+int rps_read_masks(rps_handle* h, uint64_t t, uint64_t* up, uint64_t* down, int32_t* count, int32_t* server)
+{
+    int rc = need_bound(h);
+    if (rc != RPS_OK) return rc;
+    if (!up || !down || !count) return fail(h, RPS_EINVAL, "an output array is NULL");
+    if ((rc = generate_masks(h, h->probe(), t, 1)) != RPS_OK) return rc;
+    rps::StepMasks host;
+    RPS_CUDA(h, cudaMemcpyAsync(&host, h->probe(), sizeof host, cudaMemcpyDeviceToHost, h->stream));
+    RPS_CUDA(h, cudaStreamSynchronize(h->stream));
+    for (int j = 0; j < h->n; ++j) {
+        up[j] = host.up[j];
+        down[j] = host.down[j];
+        count[j] = host.cnt[j];
+        if (server) server[j] = host.server[j];
+    }
+    return RPS_OK;
+}
+
+int rps_diag(rps_handle* h, double* dist2_to_opt, double* consensus)
+{
+    int rc = need_bound(h);
+    if (rc != RPS_OK) return rc;
+    RPS_CUDA(h, cudaMemsetAsync(h->diag_acc(), 0, 2 * sizeof(double), h->stream));
+    rps::DiagParams prm{};
+    prm.x = h->x;
+    prm.b = h->b;
+    prm.out = h->diag_acc();
+    prm.pitch = h->pitch();
+    prm.d = h->d;
+    prm.n = h->n;
+    cudaError_t err = rps::launch_diag(prm, h->opt.dtype == RPS_BF16, h->sm_count, h->stream);
+    if (err != cudaSuccess) return cuda_fail(h, "diagnostic kernel launch", err);
+    double host[2] = {0.0, 0.0};
+    RPS_CUDA(h, cudaMemcpyAsync(host, h->diag_acc(), sizeof host, cudaMemcpyDeviceToHost, h->stream));
+    RPS_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (dist2_to_opt) *dist2_to_opt = host[0];
+    if (consensus) *consensus = host[1];
+    return RPS_OK;
+}
+
+int rps_profile(rps_handle* h, int enable)
+{
+    if (!h) return RPS_EINVAL;
+    if (!enable) {
+        int rc = flush_timing(h);
+        h->profiling = false;
+        return rc;
+    }
+    h->profiling = true;
+    return RPS_OK;
+}
+
+int rps_profile_read(rps_handle* h, double* fused_ms, int64_t* fused_launches, double* mask_ms, int64_t* mask_launches)
+{
+    if (!h) return RPS_EINVAL;
+    int rc = flush_timing(h);
+    if (rc != RPS_OK) return rc;
+    if (fused_ms) *fused_ms = h->ms[0];
+    if (fused_launches) *fused_launches = h->timed[0];
+    if (mask_ms) *mask_ms = h->ms[1];
+    if (mask_launches) *mask_launches = h->timed[1];
+    h->ms[0] = h->ms[1] = 0.0;
+    h->timed[0] = h->timed[1] = 0;
+    return RPS_OK;
+}
+
+int64_t rps_launch_count(const rps_handle* h) { return h ? h->launches : 0; }
+
+const char* rps_last_error(const rps_handle* h) { return h ? h->error.c_str() : g_create_error.c_str(); }
+
+const char* rps_version(void) { return "0.1"; }
+
+}  // extern "C"

@@ -1,0 +1,93 @@
+"""Host-side checks of the C ABI: the built library exports every symbol that
+include/rps.h declares, and the calls that need no GPU validate their arguments."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "rps.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_1810_07766_b200 import build, binding
+
+    build.build()
+    return binding.load_library()
+
+
+def declared_symbols():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rps_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(lib):
+    from paper_1810_07766_b200 import binding
+
+    names = declared_symbols()
+    assert len(names) >= 20
+    assert sorted(binding.SYMBOLS) == names
+    for name in names:
+        assert getattr(lib, name) is not None
+
+
+def test_create_validates_arguments(lib):
+    h = ctypes.c_void_p()
+    bad = [(0, 10, 0.1, 0.1), (65, 10, 0.1, 0.1), (4, 0, 0.1, 0.1), (4, 1 << 34, 0.1, 0.1), (4, 10, -0.1, 0.1),
+           (4, 10, 1.5, 0.1), (4, 10, float("nan"), 0.1), (4, 10, 0.1, float("inf"))]
+    for n, d, p, g in bad:
+        assert lib.rps_create(n, d, p, g, 0, ctypes.byref(h)) == -1
+        assert not h.value
+        assert lib.rps_last_error(None)
+    assert lib.rps_create(4, 10, 0.1, 0.1, 0, None) == -1
+    assert lib.rps_destroy(None) == 0
+
+
+def test_options_pitch_and_state_errors(lib):
+    from paper_1810_07766_b200.binding import rps_options
+
+    h = ctypes.c_void_p()
+    assert lib.rps_create(8, 11_173_962, 0.1, 0.05, 1, ctypes.byref(h)) == 0
+    try:
+        assert lib.rps_pitch(h) == 11_173_984                      # rounded up to 32 floats
+        opt = rps_options()
+        assert lib.rps_default_options(ctypes.byref(opt)) == 0
+        assert (opt.dtype, opt.assign, opt.self_delivery, opt.mask_window, opt.sigma) == (0, 0, 1, 32, 0.0)
+        assert lib.rps_scratch_bytes(h) == 256 + 34 * 1536
+        opt.dtype = 1
+        assert lib.rps_configure(h, ctypes.byref(opt)) == 0
+        assert lib.rps_pitch(h) == 11_174_016                      # rounded up to 64 bf16
+        for field, value in (("dtype", 7), ("assign", 2), ("self_delivery", 3), ("mask_window", 0),
+                             ("mask_window", 257), ("sigma", -1.0)):
+            bad = rps_options()
+            lib.rps_default_options(ctypes.byref(bad))
+            setattr(bad, field, value)
+            assert lib.rps_configure(h, ctypes.byref(bad)) == -1
+            assert lib.rps_last_error(h)
+        # nothing is bound yet: stepping is a state error, not a crash
+        assert lib.rps_step(h) == -2
+        assert lib.rps_step_n(h, 3) == -2
+        assert lib.rps_read(h, None) == -2
+        assert b"rps_bind" in lib.rps_last_error(h)
+        assert lib.rps_bind(h, None, None, 0, None, 0, None) == -1
+        t = ctypes.c_uint64()
+        assert lib.rps_set_step(h, 1 << 40) == 0 and lib.rps_get_step(h, ctypes.byref(t)) == 0
+        assert t.value == 1 << 40
+        assert lib.rps_launch_count(h) == 0
+    finally:
+        assert lib.rps_destroy(h) == 0
+    assert lib.rps_version() == b"0.1"
+
+
+def test_binding_refuses_to_run_without_a_gpu():
+    import torch
+
+    from paper_1810_07766_b200 import binding
+
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    with pytest.raises(RuntimeError):
+        binding.RPS(4, 16, 0.1, 0.1, 0)

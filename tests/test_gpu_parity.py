@@ -1,0 +1,341 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle.
+
+Bars: drop masks, receive counts and servers bit-exact; fp32 replicas within
+|delta| <= 1e-6 * (1 + |x|) after one step and 1e-5 (element-wise against
+1 + |x|, and relative in the 2-norm) after T steps; bf16 replicas within 1e-2.
+Every expected value comes from the oracle, which is given the same seeded
+inputs and never sees a value computed on the GPU.
+"""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+from paper_1810_07766_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+STEP_TOL = 1e-6
+RUN_TOL = 1e-5
+BF16_TOL = 1e-2
+
+
+@pytest.fixture(scope="module")
+def rps_mod():
+    if not torch.cuda.is_available():
+        pytest.fail("these tests need a CUDA device")
+    from paper_1810_07766_b200 import binding, build
+
+    build.build()
+    binding.load_library()
+    return binding
+
+
+def make(rps_mod, w, **kw):
+    args = dict(dtype=w.dtype, sigma=w.sigma)
+    args.update(kw)
+    p = args.pop("p", w.p)
+    return rps_mod.RPS(w.n, w.d, p, w.gamma, w.seed, **args)
+
+
+def assert_close(w, got, want, tol):
+    g, o = wl.as_float64(w, got), wl.as_float64(w, want)
+    err = np.abs(g - o) / (1.0 + np.abs(o))
+    assert err.max() <= tol, f"max |delta|/(1+|x|) = {err.max():.3e} at {np.unravel_index(err.argmax(), err.shape)}"
+    rel = np.linalg.norm(g - o) / max(np.linalg.norm(o), 1e-30)
+    assert rel <= tol, f"relative 2-norm error {rel:.3e}"
+    return err.max()
+
+
+# reduced-d twins of the five workloads: same n, p, gamma, sigma, seed; d ~ 1e5 with the
+# same residues d % 4 and ceil(d/n) % 4 as the full size, so the same code paths run
+TWINS = {
+    "cfg1": wl.WORKLOADS["cfg1"],
+    "cfg2": wl.WORKLOADS["cfg2"].scaled(d=100_010, steps=50),
+    "cfg3": wl.WORKLOADS["cfg3"].scaled(d=100_008, steps=40),
+    "cfg4": wl.WORKLOADS["cfg4"].scaled(d=100_005, steps=25),
+    "cfg5": wl.WORKLOADS["cfg5"].scaled(d=65_536, steps=20),
+}
+
+
+def test_twins_keep_the_residues():
+    for name, twin in TWINS.items():
+        full = wl.WORKLOADS[name]
+        assert twin.d % 4 == full.d % 4
+        assert (-(-twin.d // twin.n)) % 4 == (-(-full.d // full.n)) % 4
+
+
+# ------------------------------------------------------------------ masks: bit-exact
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 8, 16, 31, 32, 33, 64])
+def test_masks_bit_exact(rps_mod, oracle, n):
+    for p, sd, assign in itertools.product((0.0, 0.01, 0.05, 0.1, 0.2, 0.3, 0.999, 1.0), (True, False), (0, 1)):
+        r = rps_mod.RPS(n, 1000, p, 0.1, 0xDEADBEEF12345678 ^ n, self_delivery=sd, assign=assign)
+        for t in (0, 1, 2, 49, 199, (1 << 32) - 1, 1 << 32, (1 << 63) + 5):
+            got = r.read_masks(t)
+            want = oracle.masks(n, p, 0xDEADBEEF12345678 ^ n, t, self_delivery=sd, assign=assign)
+            for a, b_ in zip(got, want):
+                assert (a == b_).all(), (n, p, sd, assign, t)
+        r.close()
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+def test_masks_of_every_step_of_every_workload(rps_mod, oracle, name):
+    w = wl.WORKLOADS[name]
+    for p in (w.p_sweep or (w.p,)):
+        r = rps_mod.RPS(w.n, 4096, p, w.gamma, w.seed, dtype=w.dtype)
+        for t in range(w.steps):
+            got = r.read_masks(t)
+            want = oracle.masks(w.n, p, w.seed, t)
+            assert all((a == b_).all() for a, b_ in zip(got, want))
+        r.close()
+
+
+# ------------------------------------------------------------------ noise
+
+def test_gradient_noise_matches_the_oracle(rps_mod, oracle):
+    """x = b = 0, gamma = sigma = 1, p = 1 gives x_1 = -xi: the raw noise field."""
+    n, d = 8, 200_003
+    w = wl.Workload("noise", n=n, d=d, dtype="f32", p=1.0, gamma=1.0, sigma=1.0, seed=12345, steps=1)
+    for t in (0, 7, 1 << 33):
+        r = make(rps_mod, w)
+        r.set_step(t)
+        r.step()
+        got = r.read()
+        want = np.zeros((n, d), dtype=np.float32)
+        oracle.step(want, np.zeros((n, d), dtype=np.float32), dtype="f32", gamma=1.0, sigma=1.0, p=1.0, seed=w.seed, t=t)
+        err = np.abs(got.astype(np.float64) - want)
+        # approximate log2 / sqrt / sin / cos: absolute error of xi stays below 1e-4 even at the
+        # smallest radii (where the log loses relative accuracy), and is ~1e-6 typically
+        assert err.max() < 1e-4, err.max()
+        assert np.median(err) < 2e-6
+        assert abs(got.std() - 1.0) < 5e-3 and abs(got.mean()) < 5e-3
+        r.close()
+
+
+# ------------------------------------------------------------------ one step from a common state
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+def test_single_step_parity(rps_mod, oracle, name):
+    w = TWINS[name]
+    b = wl.make_targets(w)
+    # a state in the middle of a run, produced by the oracle alone
+    x0 = wl.make_initial(w)
+    oracle.run(x0, b, dtype=w.dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=3)
+    for p in (w.p_sweep or (w.p,)):
+        r = make(rps_mod, w, p=p)
+        r.set_targets(b)
+        for t in (3, 4):
+            r.write(x0)
+            r.set_step(t)
+            r.step()
+            got = r.read()
+            want = x0.copy()
+            oracle.step(want, b, dtype=w.dtype, gamma=w.gamma, sigma=w.sigma, p=p, seed=w.seed, t=t)
+            assert_close(w, got, want, BF16_TOL if w.dtype == "bf16" else STEP_TOL)
+            if w.dtype == "bf16":
+                # rounding to bf16 may differ by one ulp where fp32 and fp64 sums straddle a tie
+                assert (got != want).mean() < 0.02
+        assert r.launch_count() >= 2
+        r.close()
+
+
+# ------------------------------------------------------------------ T free-running steps
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+def test_free_running_parity(rps_mod, oracle, name):
+    w = TWINS[name]
+    b = wl.make_targets(w)
+    want = wl.make_initial(w)
+    oracle.run(want, b, dtype=w.dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps)
+    r = make(rps_mod, w)
+    r.set_targets(b)
+    r.write(wl.make_initial(w))
+    r.step_n(w.steps)
+    assert r.get_step() == w.steps
+    got = r.read()
+    assert_close(w, got, want, BF16_TOL if w.dtype == "bf16" else RUN_TOL)
+    # diagnostics against the oracle's, on the oracle's state
+    r.write(want)
+    dist2, cons = r.diag()
+    o_dist2, o_cons = oracle.diag(want, b, dtype=w.dtype)
+    assert dist2 == pytest.approx(o_dist2, rel=1e-9) and cons == pytest.approx(o_cons, rel=1e-9)
+    r.close()
+
+
+def test_mask_window_does_not_change_results(rps_mod):
+    w = TWINS["cfg2"].scaled(d=10_010, steps=12)
+    b = wl.make_targets(w)
+    outs = []
+    for window in (1, 5, 32):
+        r = make(rps_mod, w, mask_window=window)
+        r.set_targets(b)
+        r.step_n(w.steps)
+        outs.append(r.read())
+        r.close()
+    assert (outs[0] == outs[1]).all() and (outs[0] == outs[2]).all()
+
+
+def test_resume_from_read_write_set_step(rps_mod):
+    w = TWINS["cfg4"].scaled(d=20_005, steps=10)
+    b = wl.make_targets(w)
+    r = make(rps_mod, w)
+    r.set_targets(b)
+    r.step_n(10)
+    straight = r.read()
+    r.close()
+    r = make(rps_mod, w)
+    r.set_targets(b)
+    r.step_n(4)
+    mid = r.read()
+    r.close()
+    r = make(rps_mod, w)
+    r.set_targets(b)
+    r.write(mid)
+    r.set_step(4)
+    r.step_n(6)
+    assert (r.read() == straight).all()
+    r.close()
+
+
+# ------------------------------------------------------------------ closed forms and invariants on the GPU output
+
+def test_p0_and_p1_closed_forms(rps_mod):
+    w = wl.WORKLOADS["cfg1"].scaled(d=4099)
+    b = wl.make_targets(w)
+    g = float(np.float32(w.gamma))
+    r = make(rps_mod, w, p=0.0, sigma=0.0)
+    r.set_targets(b)
+    r.step_n(30)
+    x = r.read()
+    assert (x == x[0]).all()
+    assert np.abs(x[0] - (1 - (1 - g) ** 30) * b.astype(np.float64).mean(axis=0)).max() <= 2e-6
+    r.close()
+    r = make(rps_mod, w, p=1.0, sigma=0.0)
+    r.set_targets(b)
+    r.step_n(30)
+    assert np.abs(r.read() - (1 - (1 - g) ** 30) * b.astype(np.float64)).max() <= 2e-6
+    r.close()
+
+
+def test_receivers_hold_identical_values_and_outputs_are_convex(rps_mod, oracle):
+    w = TWINS["cfg4"].scaled(d=9_001)
+    b = wl.make_targets(w)
+    x0 = np.random.default_rng(0).standard_normal(b.shape).astype(np.float32)
+    r = make(rps_mod, w, sigma=0.0)
+    r.set_targets(b)
+    r.write(x0)
+    r.step()
+    x = r.read()
+    _, down, _, _ = oracle.masks(w.n, w.p, w.seed, 0)
+    block = -(-w.d // w.n)
+    v = x0.astype(np.float64) - float(np.float32(w.gamma)) * (x0.astype(np.float64) - b)
+    assert (x <= v.max(axis=0) + 1e-6).all() and (x >= v.min(axis=0) - 1e-6).all()
+    for j in range(w.n):
+        rows = [i for i in range(w.n) if (int(down[j]) >> i) & 1]
+        cols = slice(j * block, min((j + 1) * block, w.d))
+        assert (x[rows, cols] == x[rows[0], cols]).all()
+    r.close()
+
+
+# ------------------------------------------------------------------ forced masks: every drop pattern on tiny n
+
+@pytest.mark.parametrize("n", [2, 3])
+def test_forced_masks_every_pattern(rps_mod, oracle, n):
+    d = 2 * n + 1
+    rng = np.random.default_rng(n)
+    b = rng.standard_normal((n, d)).astype(np.float32)
+    x0 = rng.standard_normal((n, d)).astype(np.float32)
+    r = rps_mod.RPS(n, d, 0.5, 0.25, 1)
+    r.set_targets(b)
+    words = range(1 << n)
+    for up0, down0, up1 in itertools.product(words, words, words):
+        up = np.array([up0, up1] + [up0] * (n - 2), dtype=np.uint64)
+        down = np.array([down0, down0 ^ 1] + [down0] * (n - 2), dtype=np.uint64)
+        r.write(x0)
+        r.step_forced(up, down)
+        got = r.read()
+        want = x0.copy()
+        oracle.step(want, b, dtype="f32", gamma=0.25, sigma=0.0, p=0.5, seed=1, t=0, forced_up=up, forced_down=down)
+        assert np.abs(got.astype(np.float64) - want).max() <= STEP_TOL * (1 + np.abs(want).max())
+    with pytest.raises(rps_mod.RPSError):
+        r.step_forced(np.array([1 << n] * n, dtype=np.uint64), np.zeros(n, dtype=np.uint64))
+    r.close()
+
+
+# ------------------------------------------------------------------ edge shapes
+
+EDGES = [
+    # n, d, dtype
+    (1, 1, "f32"), (1, 1000, "f32"), (2, 1, "f32"), (7, 3, "f32"), (5, 5, "f32"), (3, 2, "f32"),
+    (64, 7, "f32"), (64, 64, "f32"), (64, 4099, "f32"), (33, 1025, "f32"), (17, 4097, "f32"),
+    (9, 130, "f32"), (4, 31, "f32"), (4, 33, "f32"), (12, 127, "f32"), (3, 100_001, "f32"),
+    (1, 9, "bf16"), (6, 3, "bf16"), (8, 1031, "bf16"), (16, 4097, "bf16"), (33, 2050, "bf16"), (64, 8191, "bf16"),
+]
+
+
+@pytest.mark.parametrize("n,d,dtype", EDGES)
+def test_edge_shapes(rps_mod, oracle, n, d, dtype):
+    w = wl.Workload("edge", n=n, d=d, dtype=dtype, p=0.3, gamma=0.1, sigma=0.1, seed=100 + n, steps=3)
+    b = wl.make_targets(w)
+    for sd, assign in ((True, 0), (False, 0), (True, 1)):
+        want = wl.make_initial(w)
+        oracle.run(want, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps,
+                   self_delivery=sd, assign=assign)
+        r = make(rps_mod, w, self_delivery=sd, assign=assign)
+        r.set_targets(b)
+        r.step_n(w.steps)
+        got = r.read()
+        assert_close(w, got, want, BF16_TOL if dtype == "bf16" else 3 * STEP_TOL)
+        # the padding between d and the row pitch is never disturbed
+        pad = r.x_dev[:, d:].float().cpu().numpy()
+        assert not pad.any()
+        r.close()
+
+
+def test_guard_bands_around_device_buffers(rps_mod):
+    """The kernels stay inside [n][pitch]: a sentinel pattern placed in the scratch tail and in
+    the targets' padding is intact after stepping."""
+    w = TWINS["cfg4"].scaled(d=50_001, steps=5)
+    r = make(rps_mod, w)
+    r.set_targets(wl.make_targets(w))
+    r.b_dev[:, w.d:] = 7.0
+    tail = r.scratch[-128:].clone()
+    r.step_n(w.steps)
+    torch.cuda.synchronize()
+    assert (r.b_dev[:, w.d:] == 7.0).all()
+    assert (r.scratch[-128:] == tail).all()
+    assert not r.x_dev[:, w.d:].any()
+    r.close()
+
+
+# ------------------------------------------------------------------ host-buffer step
+
+def test_step_host_equals_resident_step(rps_mod):
+    w = TWINS["cfg2"].scaled(d=30_002, steps=4)
+    b = wl.make_targets(w)
+    r = make(rps_mod, w)
+    r.set_targets(b)
+    r.step_n(w.steps)
+    want = r.read()
+    r.close()
+    r = make(rps_mod, w)
+    x_host = torch.zeros((w.n, w.d), dtype=torch.float32).pin_memory()
+    b_host = torch.from_numpy(b).pin_memory()
+    for _ in range(w.steps):
+        r.step_host(x_host, b_host)
+    assert (x_host.numpy() == want).all()
+    r.close()
+
+
+def test_profile_counts_launches(rps_mod):
+    w = TWINS["cfg1"]
+    r = make(rps_mod, w, mask_window=4)
+    r.profile(True)
+    r.step_n(8)
+    fused_ms, fused_n, mask_ms, mask_n = r.profile_read()
+    assert (fused_n, mask_n) == (8, 2) and fused_ms > 0 and mask_ms > 0
+    r.profile(False)
+    assert r.launch_count() == 10
+    r.close()
