@@ -224,7 +224,7 @@ def run_cuda(args):
     tdtype = torch.float32 if w.dtype == "f32" else torch.int16  # bf16 bit patterns travel as 16-bit words
     x_host = torch.zeros((w.n, w.d), dtype=tdtype).pin_memory()
     b_host = torch.from_numpy(b if w.dtype == "f32" else b.view(np.int16)).pin_memory()
-    e2e_steps = min(args.steps, args.e2e_steps)
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
     for _ in range(2):
         r.step_host(x_host, b_host)
     e2e_ms = timed_steps(torch, stream, lambda: [r.step_host(x_host, b_host) for _ in range(e2e_steps)], device)
