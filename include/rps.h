@@ -41,7 +41,8 @@ typedef enum rps_status {
     RPS_EINVAL = -1, /* bad argument (range, NULL, alignment, size)          */
     RPS_ESTATE = -2, /* call not allowed in the handle's current state      */
     RPS_ECUDA = -3,  /* a CUDA runtime call or kernel launch reported an error */
-    RPS_ENOMEM = -4  /* host allocation failed                               */
+    RPS_ENOMEM = -4, /* host allocation failed                               */
+    RPS_ELIMIT = -5  /* a size exceeds a fixed capacity built into the library */
 } rps_status;
 
 enum { RPS_MAX_WORKERS = 64 };
@@ -187,6 +188,45 @@ int rps_diag(rps_handle* h, double* dist2_to_opt, double* consensus);
 int rps_profile(rps_handle* h, int enable);
 int rps_profile_read(rps_handle* h, double* fused_ms, int64_t* fused_launches, double* mask_ms,
                      int64_t* mask_launches);
+
+/*
+ * rps_step_static: one step of the same method with no handle, no rps_bind() and
+ * no scratch buffer from the caller.  (The paper has no counterpart: this entry
+ * point exists for the sake of callers, not of the algorithm.)
+ *
+ * Who needs it: code that cannot call cudaMalloc or any allocating routine where
+ * it runs.  Examples are a plug-in living inside another framework's fixed
+ * memory pool, a control loop that may not block on the driver's allocator, or a
+ * host that hands out device buffers and forbids further allocation.  Such a
+ * caller already owns x and b; the only other device memory a step needs is the
+ * record of that step's drop masks, which here lives in a fixed 1536-byte array
+ * compiled into the library (room for RPS_MAX_WORKERS workers).  Every GPU that
+ * loads the library carries that array until the process exits.
+ *
+ *   n, d, p, gamma, seed   as for rps_create; n > RPS_MAX_WORKERS returns RPS_ELIMIT
+ *                          because the built-in mask record cannot hold more workers
+ *   dtype                  rps_dtype of x_dev and b_dev
+ *   x_dev                  device [n][pitch] replicas, 128-byte aligned; input and output
+ *   b_dev                  device [n][pitch] targets, 128-byte aligned; input
+ *   pitch                  d rounded up to 32 (fp32) or 64 (bf16) elements
+ *   sigma                  std-dev of the gradient noise, >= 0
+ *   t                      step counter; the caller advances it (0, 1, 2, ...)
+ *   cuda_stream            cudaStream_t the two kernels are enqueued on (NULL = default)
+ *
+ * Fixed assignment and self-delivery, as in the default options.  Calls with the
+ * same arguments give the same replicas as rps_step() on a handle at step t.
+ * The call allocates nothing on the device and frees nothing.  Its first call on
+ * a device looks up the array's device address and the SM count (once per
+ * device, with that device current); make that first call outside any stream
+ * capture.  All calls on a device share the one array, which keeps whatever the
+ * previous call left in it; each call rewrites the part it reads, so nothing
+ * needs clearing, but two calls that overlap on the GPU (different streams, or
+ * different host threads on different streams) race on it: keep them on one
+ * stream or order them with events.  Returns RPS_OK, RPS_EINVAL, RPS_ELIMIT or
+ * RPS_ECUDA; asynchronous like rps_step().
+ */
+int rps_step_static(int n, int64_t d, int dtype, void* x_dev, const void* b_dev, int64_t pitch, double p,
+                    double gamma, double sigma, uint64_t seed, uint64_t t, void* cuda_stream);
 
 /* Kernels launched by this handle since creation (both kinds).               */
 int64_t rps_launch_count(const rps_handle* h);

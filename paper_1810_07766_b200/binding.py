@@ -17,6 +17,7 @@ _CSRC = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc")
 LIB_PATH = os.path.join(_CSRC, "librps.so")
 
 RPS_OK, RPS_EINVAL, RPS_ESTATE, RPS_ECUDA, RPS_ENOMEM = 0, -1, -2, -3, -4
+RPS_ELIMIT = -5
 RPS_F32, RPS_BF16 = 0, 1
 RPS_ASSIGN_FIXED, RPS_ASSIGN_PERM = 0, 1
 _DTYPE = {"f32": RPS_F32, "bf16": RPS_BF16}
@@ -26,7 +27,7 @@ SYMBOLS = (
     "rps_create", "rps_destroy", "rps_default_options", "rps_configure", "rps_pitch", "rps_scratch_bytes",
     "rps_bind", "rps_set_targets", "rps_write", "rps_set_step", "rps_get_step", "rps_step", "rps_step_n",
     "rps_step_forced", "rps_step_host", "rps_read", "rps_read_masks", "rps_diag", "rps_profile",
-    "rps_profile_read", "rps_launch_count", "rps_last_error", "rps_version",
+    "rps_profile_read", "rps_launch_count", "rps_last_error", "rps_version", "rps_step_static",
 )
 
 
@@ -79,6 +80,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         "rps_launch_count": (i64, [vp]),
         "rps_last_error": (ctypes.c_char_p, [vp]),
         "rps_version": (ctypes.c_char_p, []),
+        "rps_step_static": (cint, [cint, i64, cint, vp, vp, i64, dbl, dbl, dbl, u64, u64, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -236,6 +238,25 @@ class RPS:
 
     def launch_count(self) -> int:
         return int(self._lib.rps_launch_count(self._h))
+
+
+def step_static(x_dev: torch.Tensor, b_dev: torch.Tensor, *, n: int, d: int, dtype: str, p: float, gamma: float,
+                sigma: float, seed: int, t: int, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """``rps_step_static``: one step on caller-owned ``[n][pitch]`` device tensors, for callers
+    that may not allocate device memory; the library uses its built-in mask record instead of
+    a scratch buffer.  Advances nothing: pass ``t`` yourself."""
+    if not (x_dev.is_cuda and b_dev.is_cuda and x_dev.is_contiguous() and b_dev.is_contiguous()):
+        raise ValueError("x_dev and b_dev must be contiguous CUDA tensors")
+    if x_dev.dim() != 2 or x_dev.shape != b_dev.shape or x_dev.shape[0] != n:
+        raise ValueError("x_dev and b_dev must both be [n][pitch]")
+    stream = torch.cuda.current_stream(x_dev.device) if stream is None else stream
+    with torch.cuda.device(x_dev.device):
+        rc = load_library().rps_step_static(n, d, _DTYPE[dtype], x_dev.data_ptr(), b_dev.data_ptr(), x_dev.shape[1],
+                                            p, gamma, sigma, seed, t, stream.cuda_stream)
+    if rc != RPS_OK:
+        reason = {RPS_EINVAL: "bad argument", RPS_ELIMIT: "n exceeds the built-in mask record (64 workers)",
+                  RPS_ECUDA: "CUDA error"}.get(rc, "error")
+        raise RPSError(rc, "rps_step_static", reason)
 
 
 def version() -> str:

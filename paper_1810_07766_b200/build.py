@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(CSRC, "librps.so")
-SOURCES = ["rps_api.cu", "rps_kernels.cu"]
+SOURCES = ["rps_api.cu", "rps_kernels.cu", "rps_static.cu"]
 HEADERS = ["rps_device.cuh", "rps_kernels.h"]
 
 
