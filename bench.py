@@ -42,7 +42,7 @@ NCU_TRAFFIC = {
 def kernel_digest() -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_1810_07766_b200", "csrc")
-    for name in ("rps_device.cuh", "rps_kernels.cu"):
+    for name in ("rps_device.cuh", "rps_kernels.cu", "rps_staged.cu"):
         with open(os.path.join(csrc, name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -198,8 +198,11 @@ def run_cuda(args):
         from dataclasses import replace
 
         w = replace(w, p=args.p)
+    if args.d is not None:
+        w = w.scaled(d=args.d)
     b = wl.make_targets(w)
-    r = binding.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma)
+    r = binding.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma, kernel=args.kernel,
+                    workers_per_lane=args.workers_per_lane, stages=args.stages, consumer_warps=args.consumer_warps, copy_mode=args.copy_mode)
     r.set_targets(b)
     stream = r.stream
     bytes_per_step = w.bytes_per_step
@@ -219,15 +222,20 @@ def run_cuda(args):
     gpu_launches = r.launch_count() - launches_before
 
     # pass 3: end to end through the host-buffer call: H2D of x and b, the step, D2H of x, every step
-    import numpy as np
+    e2e = None
+    if not args.skip_e2e:
+        import numpy as np
 
-    tdtype = torch.float32 if w.dtype == "f32" else torch.int16  # bf16 bit patterns travel as 16-bit words
-    x_host = torch.zeros((w.n, w.d), dtype=tdtype).pin_memory()
-    b_host = torch.from_numpy(b if w.dtype == "f32" else b.view(np.int16)).pin_memory()
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    for _ in range(2):
-        r.step_host(x_host, b_host)
-    e2e_ms = timed_steps(torch, stream, lambda: [r.step_host(x_host, b_host) for _ in range(e2e_steps)], device)
+        tdtype = torch.float32 if w.dtype == "f32" else torch.int16  # bf16 bit patterns travel as 16-bit words
+        x_host = torch.zeros((w.n, w.d), dtype=tdtype).pin_memory()
+        b_host = torch.from_numpy(b if w.dtype == "f32" else b.view(np.int16)).pin_memory()
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        for _ in range(2):
+            r.step_host(x_host, b_host)
+        e2e_ms = timed_steps(torch, stream, lambda: [r.step_host(x_host, b_host) for _ in range(e2e_steps)], device)
+        e2e = {"value": world * w.n * w.d * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
+               "h2d_bytes_per_step": 2 * w.n * w.d * w.elem_bytes, "d2h_bytes_per_step": w.n * w.d * w.elem_bytes,
+               "call": "rps_step_host (pinned host x and b)"}
     row_bytes = w.n * w.d * w.elem_bytes
 
     peak, peak_kind = measured_peak_gbs()
@@ -245,15 +253,15 @@ def run_cuda(args):
             "workload": f"{w.name}: n={w.n} workers, d={w.d} {w.dtype}, p={w.p}, gamma={w.gamma}, sigma={w.sigma}, "
                         f"seed={w.seed}; quadratic objective, b_i ~ N({'mu_i' if w.hetero else '0'},1)",
             "n": w.n, "d": w.d, "p": w.p, "replicas": "one independent job per GPU, no collective",
+            "kernel_shape": {"kernel": args.kernel, "workers_per_lane": args.workers_per_lane, "stages": args.stages,
+                             "consumer_warps": args.consumer_warps, "copy_mode": args.copy_mode},
             "l2": "inputs larger than L2 (x and b are %.0f MB each)" % (row_bytes / 1e6),
             "algorithmic_bytes_per_step": bytes_per_step,
             "hbm_gbs_whole_step": bytes_per_step / (total_ms / args.steps * 1e-3) / 1e9,
             "frac_of_8TBs_nominal": bytes_per_step / (total_ms / args.steps * 1e-3) / 8e12,
         },
         "clocks": clocks.summary(),
-        "e2e": {"value": world * w.n * w.d * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
-                "h2d_bytes_per_step": 2 * row_bytes, "d2h_bytes_per_step": row_bytes,
-                "call": "rps_step_host (pinned host x and b)"},
+        "e2e": e2e,
         "gpu_launches": gpu_launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "rps_fused_kernel",
@@ -328,9 +336,16 @@ def main(argv=None):
     ap.add_argument("--impl", choices=("cuda", "reference"), default="cuda")
     ap.add_argument("--workload", choices=("cfg1", "cfg2", "cfg3", "cfg4", "cfg5"), default="cfg2")
     ap.add_argument("--p", type=float, default=None, help="override the drop probability (p sweeps)")
+    ap.add_argument("--d", type=int, default=None, help="override the model size (small profiler captures)")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--reference-columns", type=int, default=500_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-e2e", action="store_true", help="tuning sweeps only: leave the host-buffer pass out")
+    ap.add_argument("--kernel", type=int, default=0, help="0 library's choice, 1 direct loads, 2 staged")
+    ap.add_argument("--workers-per-lane", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--consumer-warps", type=int, default=0)
+    ap.add_argument("--copy-mode", type=int, default=0, help="staged kernel: 1 bulk copy per row, 2 TMA boxes")
     args = ap.parse_args(argv)
     if args.steps < 1 or args.warmup < 0:
         raise SystemExit("--steps must be >= 1 and --warmup >= 0")

@@ -22,7 +22,8 @@
  *   - Dense host arrays are row-major [n][d] in the replica type (float, or
  *     bfloat16 bit patterns in uint16_t).  On the device a row occupies
  *     rps_pitch() elements (d rounded up so that every row starts on a 128-byte
- *     boundary); columns d..pitch-1 are padding owned by the library.
+ *     boundary, plus row_skew_lines lines); columns d..pitch-1 are padding that
+ *     the library reads but never writes.
  */
 #ifndef RPS_H
 #define RPS_H
@@ -69,6 +70,19 @@ typedef struct rps_options {
     int32_t mask_window;   /* drop masks are generated this many steps at a time (1..256,
                               default 32); does not change any result                     */
     double sigma;          /* std-dev of the Gaussian gradient noise, default 0           */
+    /* Shape of the fused kernel; 0 = the library's choice.  None of these changes what is
+     * computed beyond the order of the fp32 additions inside the masked average.           */
+    int32_t row_skew_lines;   /* extra 128-byte lines of padding per device row, -1 = automatic
+                                 (keeps the n rows from all mapping to one DRAM channel when
+                                 the row size is a multiple of a large power of two)         */
+    int32_t kernel;           /* 1: lanes load their slices directly from global memory;
+                                 2: slices are staged through shared memory by bulk
+                                 asynchronous copies (default)                               */
+    int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */
+    int32_t stages;           /* depth of the shared-memory ring of kernel 2 (2..8)          */
+    int32_t consumer_warps;   /* compute warps per CTA of kernel 2 (1..16)                   */
+    int32_t copy_mode;        /* kernel 2 fills a stage with 1: one bulk copy per row,
+                                 2: two-dimensional TMA boxes covering all n rows            */
 } rps_options;
 
 /*
@@ -199,7 +213,7 @@ int rps_profile_read(rps_handle* h, double* fused_ms, int64_t* fused_launches, d
  * memory pool, a control loop that may not block on the driver's allocator, or a
  * host that hands out device buffers and forbids further allocation.  Such a
  * caller already owns x and b; the only other device memory a step needs is the
- * record of that step's drop masks, which here lives in a fixed 1536-byte array
+ * record of that step's drop masks, which here lives in a fixed 1792-byte array
  * compiled into the library (room for RPS_MAX_WORKERS workers).  Every GPU that
  * loads the library carries that array until the process exits.
  *
@@ -208,7 +222,7 @@ int rps_profile_read(rps_handle* h, double* fused_ms, int64_t* fused_launches, d
  *   dtype                  rps_dtype of x_dev and b_dev
  *   x_dev                  device [n][pitch] replicas, 128-byte aligned; input and output
  *   b_dev                  device [n][pitch] targets, 128-byte aligned; input
- *   pitch                  d rounded up to 32 (fp32) or 64 (bf16) elements
+ *   pitch                  row pitch in elements: >= d and a multiple of 32 (fp32) or 64 (bf16)
  *   sigma                  std-dev of the gradient noise, >= 0
  *   t                      step counter; the caller advances it (0, 1, 2, ...)
  *   cuda_stream            cudaStream_t the two kernels are enqueued on (NULL = default)

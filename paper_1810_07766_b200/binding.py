@@ -33,7 +33,10 @@ SYMBOLS = (
 
 class rps_options(ctypes.Structure):
     _fields_ = [("dtype", ctypes.c_int32), ("assign", ctypes.c_int32), ("self_delivery", ctypes.c_int32),
-                ("mask_window", ctypes.c_int32), ("sigma", ctypes.c_double)]
+                ("mask_window", ctypes.c_int32), ("sigma", ctypes.c_double), ("row_skew_lines", ctypes.c_int32),
+                ("kernel", ctypes.c_int32),
+                ("workers_per_lane", ctypes.c_int32), ("stages", ctypes.c_int32), ("consumer_warps", ctypes.c_int32),
+                ("copy_mode", ctypes.c_int32)]
 
 
 class RPSError(RuntimeError):
@@ -108,7 +111,8 @@ class RPS:
 
     def __init__(self, n: int, d: int, p: float, gamma: float, seed: int, *, dtype: str = "f32", sigma: float = 0.0,
                  assign: int = RPS_ASSIGN_FIXED, self_delivery: bool = True, mask_window: int = 32,
-                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+                 kernel: int = 0, workers_per_lane: int = 0, stages: int = 0, consumer_warps: int = 0,
+                 row_skew_lines: int = -1, copy_mode: int = 0, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         if not torch.cuda.is_available():
@@ -121,6 +125,8 @@ class RPS:
         self._lib.rps_default_options(ctypes.byref(opt))
         opt.dtype, opt.assign, opt.self_delivery = _DTYPE[dtype], assign, int(self_delivery)
         opt.mask_window, opt.sigma = mask_window, sigma
+        opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps = kernel, workers_per_lane, stages, consumer_warps
+        opt.row_skew_lines, opt.copy_mode = row_skew_lines, copy_mode
         self._check(self._lib.rps_configure(self._h, ctypes.byref(opt)), "rps_configure")
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
         self.pitch = int(self._lib.rps_pitch(self._h))

@@ -15,9 +15,19 @@
 
 static_assert(sizeof(rps::StepMasks) == rps::kStepMasksBytes, "mask record layout");
 
+// Extra 128-byte lines appended to every row so that the rows of x and b do not all start at
+// the same offset modulo a large power of two (which would send the n row streams of a tile
+// to the same DRAM channel and bank).  `asked` < 0 = automatic.
+static int64_t rps_row_skew_lines(int64_t lines, int32_t asked)
+{
+    if (asked >= 0) return asked;
+    return (lines % 2 == 0) ? 1 : 0;
+}
+
 namespace {
 
-constexpr size_t kDiagBytes = 256;  // two fp64 accumulators, padded
+constexpr size_t kDiagBytes = 256;   // two fp64 accumulators, then the kernels' error word, padded
+constexpr size_t kErrorOffset = 64;
 thread_local std::string g_create_error;
 
 struct TimedLaunch {
@@ -59,9 +69,15 @@ struct rps_handle {
     int64_t pitch() const
     {
         const int64_t per_line = 128 / (int64_t)elem();
-        return (d + per_line - 1) / per_line * per_line;
+        const int64_t lines = (d + per_line - 1) / per_line;
+        return (lines + rps_row_skew_lines(lines, opt.row_skew_lines)) * per_line;
     }
     double* diag_acc() const { return reinterpret_cast<double*>(scratch); }
+    int32_t* error_word() const { return reinterpret_cast<int32_t*>(scratch + kErrorOffset); }
+    rps::FusedTuning tuning() const
+    {
+        return rps::FusedTuning{opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps, opt.copy_mode};
+    }
     rps::StepMasks* window() const { return reinterpret_cast<rps::StepMasks*>(scratch + kDiagBytes); }
     rps::StepMasks* probe() const { return window() + opt.mask_window; }
     rps::StepMasks* forced() const { return window() + opt.mask_window + 1; }
@@ -163,13 +179,12 @@ int run_fused(rps_handle* h, const rps::StepMasks* masks)
     prm.block_cols = (h->d + h->n - 1) / h->n;
     prm.n = h->n;
     prm.narrow = h->d < ((int64_t)1 << 31);
-    prm.gamma = h->gamma;
-    prm.sigma = h->sigma;
+    prm.error = h->error_word();
+    rps::set_sgd_scalars(prm, h->gamma, h->sigma);
     prm.t_lo = (uint32_t)h->t;
     prm.t_hi = (uint32_t)(h->t >> 32);
-    prm.key0 = (uint32_t)h->seed;
-    prm.key1 = (uint32_t)(h->seed >> 32);
-    int rc = timed_launch(h, 0, [&] { return rps::launch_fused(prm, h->opt.dtype == RPS_BF16, h->sm_count, h->stream); });
+    rps::set_philox_key(prm, h->seed);
+    int rc = timed_launch(h, 0, [&] { return rps::launch_fused(prm, h->tuning(), h->opt.dtype == RPS_BF16, h->sm_count, h->stream); });
     if (rc == RPS_OK) h->t += 1;
     return rc;
 }
@@ -201,6 +216,18 @@ int download(rps_handle* h, void* host, const void* dev)
     return copy_rows(h, host, (size_t)h->d * h->elem(), dev, (size_t)h->pitch() * h->elem(), cudaMemcpyDeviceToHost);
 }
 
+// Drains the stream and reports a kernel that gave up on a bounded wait.
+int finish(rps_handle* h)
+{
+    int32_t word = 0;
+    RPS_CUDA(h, cudaMemcpyAsync(&word, h->error_word(), sizeof word, cudaMemcpyDeviceToHost, h->stream));
+    RPS_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (word != 0)
+        return fail(h, RPS_ECUDA, word == 1 ? "the fused kernel's producer gave up waiting for a free stage"
+                                            : "the fused kernel's consumers gave up waiting for data");
+    return RPS_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -213,6 +240,12 @@ int rps_default_options(rps_options* opt)
     opt->self_delivery = 1;
     opt->mask_window = 32;
     opt->sigma = 0.0;
+    opt->row_skew_lines = -1;
+    opt->kernel = 0;
+    opt->workers_per_lane = 0;
+    opt->stages = 0;
+    opt->consumer_warps = 0;
+    opt->copy_mode = 0;
     return RPS_OK;
 }
 
@@ -275,6 +308,16 @@ int rps_configure(rps_handle* h, const rps_options* opt)
     if (opt->self_delivery != 0 && opt->self_delivery != 1) return fail(h, RPS_EINVAL, "self_delivery must be 0 or 1");
     if (opt->mask_window < 1 || opt->mask_window > 256) return fail(h, RPS_EINVAL, "mask_window must be in 1..256");
     if (!std::isfinite(opt->sigma) || opt->sigma < 0.0) return fail(h, RPS_EINVAL, "sigma must be finite and >= 0");
+    if (opt->row_skew_lines < -1 || opt->row_skew_lines > 4096)
+        return fail(h, RPS_EINVAL, "row_skew_lines must be -1 (auto) or 0..4096");
+    if (opt->kernel < 0 || opt->kernel > 2) return fail(h, RPS_EINVAL, "kernel must be 0 (auto), 1 or 2");
+    if (opt->workers_per_lane != 0 && opt->workers_per_lane != 2 && opt->workers_per_lane != 4 &&
+        opt->workers_per_lane != 8)
+        return fail(h, RPS_EINVAL, "workers_per_lane must be 0 (auto), 2, 4 or 8");
+    if (opt->stages != 0 && (opt->stages < 2 || opt->stages > 8)) return fail(h, RPS_EINVAL, "stages must be 0 or 2..8");
+    if (opt->consumer_warps < 0 || opt->consumer_warps > 16)
+        return fail(h, RPS_EINVAL, "consumer_warps must be 0 (auto) or 1..16");
+    if (opt->copy_mode < 0 || opt->copy_mode > 2) return fail(h, RPS_EINVAL, "copy_mode must be 0 (auto), 1 or 2");
     h->opt = *opt;
     h->sigma = (float)opt->sigma;
     return RPS_OK;
@@ -302,6 +345,7 @@ int rps_bind(rps_handle* h, void* x_dev, void* b_dev, int64_t pitch, void* scrat
     h->stream = static_cast<cudaStream_t>(cuda_stream);
     h->bound = true;
     h->window_valid = false;
+    RPS_CUDA(h, cudaMemsetAsync(h->error_word(), 0, sizeof(int32_t), h->stream));
     return RPS_OK;
 }
 
@@ -374,6 +418,7 @@ int rps_step_forced(rps_handle* h, const uint64_t* up, const uint64_t* down)
         h->staged.down[j] = cnt > 0 ? down[j] : 0;
         h->staged.cnt[j] = cnt;
         h->staged.server[j] = j;
+        h->staged.inv_cnt[j] = cnt > 0 ? 1.0f / (float)cnt : 0.0f;
     }
     // `staged` is pageable, so the copy has left it when the call returns; on the device the
     // copy is ordered after the previous step's kernel by the stream
@@ -390,8 +435,7 @@ int rps_step_host(rps_handle* h, void* x_host, const void* b_host)
     if (b_host && (rc = upload(h, h->b, b_host)) != RPS_OK) return rc;
     if ((rc = rps_step(h)) != RPS_OK) return rc;
     if ((rc = download(h, x_host, h->x)) != RPS_OK) return rc;
-    RPS_CUDA(h, cudaStreamSynchronize(h->stream));
-    return RPS_OK;
+    return finish(h);
 }
 
 int rps_read(rps_handle* h, void* x_host_out)
@@ -400,8 +444,7 @@ int rps_read(rps_handle* h, void* x_host_out)
     if (rc != RPS_OK) return rc;
     if (!x_host_out) return fail(h, RPS_EINVAL, "x_host_out is NULL");
     if ((rc = download(h, x_host_out, h->x)) != RPS_OK) return rc;
-    RPS_CUDA(h, cudaStreamSynchronize(h->stream));
-    return RPS_OK;
+    return finish(h);
 }
 
 int rps_read_masks(rps_handle* h, uint64_t t, uint64_t* up, uint64_t* down, int32_t* count, int32_t* server)

@@ -1,11 +1,14 @@
 // Device-side building blocks of the RPS step: Philox4x32-10, the counter
-// layout of the three random streams, the Gaussian transform, and the layout of
-// one step's drop masks in global memory.
+// layout of the random streams, the Gaussian transform, the layout of one
+// step's drop masks, and the per-lane arithmetic shared by the fused kernels
+// (local SGD step, masked average, masked write-back).
 #pragma once
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include "rps_kernels.h"
 
 namespace rps {
 
@@ -26,6 +29,7 @@ struct StepMasks {
     uint64_t down[kMaxWorkers];
     int32_t cnt[kMaxWorkers];
     int32_t server[kMaxWorkers];
+    float inv_cnt[kMaxWorkers];  // 1 / cnt[j] rounded to nearest, 0 where cnt[j] == 0
 };
 
 struct Philox4 {
@@ -42,32 +46,251 @@ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint3
     constexpr uint32_t kWeylA = 0x9E3779B9u, kWeylB = 0xBB67AE85u;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        const uint32_t hi_a = __umulhi(kMulA, c0), lo_a = kMulA * c0;
-        const uint32_t hi_b = __umulhi(kMulB, c2), lo_b = kMulB * c2;
-        c0 = hi_b ^ c1 ^ k0;
-        c1 = lo_b;
-        c2 = hi_a ^ c3 ^ k1;
-        c3 = lo_a;
+        const uint64_t prod_a = (uint64_t)kMulA * c0;
+        const uint64_t prod_b = (uint64_t)kMulB * c2;
+        c0 = (uint32_t)(prod_b >> 32) ^ c1 ^ k0;
+        c1 = (uint32_t)prod_b;
+        c2 = (uint32_t)(prod_a >> 32) ^ c3 ^ k1;
+        c3 = (uint32_t)prod_a;
         k0 += kWeylA;
         k1 += kWeylB;
     }
     return Philox4{c0, c1, c2, c3};
 }
 
-// One Box-Muller pair from one 32-bit word: the low 16 bits pick the radius
-// uniform and the high 16 bits the angle uniform, both at bin centres
-// (k + 1/2) / 2^16, which fp32 represents exactly.  Returns (r cos a, r sin a).
-__device__ __forceinline__ float2 gaussian_pair(uint32_t word)
+// The same generator with the ten round keys k + r * (Weyl constants) prepared by the host
+// (FusedParams::round_key): inside the fused kernels the key never changes, so the key
+// schedule costs nothing per draw.
+__device__ __forceinline__ Philox4 philox4x32_10_keyed(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                       const uint32_t (&round_key)[10][2])
 {
-    // 1.0f + k * 2^-16 built in the mantissa, minus (1 - 2^-17): exact.
-    const float u_radius = __uint_as_float(0x3F800000u | ((word & 0xFFFFu) << 7)) - 0.99999237060546875f;
-    const float u_angle = __uint_as_float(0x3F800000u | ((word >> 16) << 7)) - 0.99999237060546875f;
-    // r = sqrt(-2 ln u) with ln u = ln 2 * log2 u
-    float radius;
-    asm("sqrt.approx.f32 %0, %1;" : "=f"(radius) : "f"(-1.3862943611198906f * __log2f(u_radius)));
-    float s, c;
-    __sincosf(6.283185307179586f * u_angle, &s, &c);
-    return make_float2(radius * c, radius * s);
+    constexpr uint32_t kMulA = 0xD2511F53u, kMulB = 0xCD9E8D57u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t prod_a = (uint64_t)kMulA * c0;
+        const uint64_t prod_b = (uint64_t)kMulB * c2;
+        c0 = (uint32_t)(prod_b >> 32) ^ c1 ^ round_key[r][0];
+        c1 = (uint32_t)prod_b;
+        c2 = (uint32_t)(prod_a >> 32) ^ c3 ^ round_key[r][1];
+        c3 = (uint32_t)prod_a;
+    }
+    return Philox4{c0, c1, c2, c3};
+}
+
+// One Box-Muller pair from one 32-bit word, already scaled by gamma*sigma.  The low
+// 16 bits pick the radius uniform and the high 16 bits the angle uniform, both at
+// bin centres (k + 1/2) / 2^16.  2^23 + k is built in the mantissa, so one fma
+// gives the uniform exactly.  Returns radius, and (cos, sin) of the angle.
+struct ScaledPair {
+    float radius, c, s;
+};
+
+__device__ __forceinline__ ScaledPair gaussian_pair(uint32_t word, float noise_scale)
+{
+    const float k_radius = __uint_as_float(__byte_perm(word, 0x4B000000u, 0x7410));  // 2^23 + low half
+    const float k_angle = __uint_as_float(__byte_perm(word, 0x4B000000u, 0x7432));   // 2^23 + high half
+    // u = (k + 1/2) / 2^16 = (2^23 + k) * 2^-16 - (128 - 2^-17), exact in fp32
+    const float u = fmaf(k_radius, 1.52587890625e-05f, -127.99999237060546875f);
+    // the angle in turns, exact for the same reason; it is scaled by 2 pi only after that, so that
+    // the rounding of the constant is not multiplied by 2^23
+    const float angle_turns = fmaf(k_angle, 1.52587890625e-05f, -127.99999237060546875f);
+    ScaledPair out;
+    // radius = gamma*sigma * sqrt(-2 ln u), with ln u = ln 2 * log2 u folded into noise_scale.
+    // The special-function unit's approximations are used in their flush-to-zero forms: no
+    // operand here is subnormal (u >= 2^-17), so the slower subnormal handling buys nothing.
+    float log2_u, turns_to_rad = 6.283185307179586f * angle_turns;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(log2_u) : "f"(u));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(out.radius) : "f"(noise_scale * log2_u));
+    asm("sin.approx.ftz.f32 %0, %1;" : "=f"(out.s) : "f"(turns_to_rad));
+    asm("cos.approx.ftz.f32 %0, %1;" : "=f"(out.c) : "f"(turns_to_rad));
+    return out;
+}
+
+// 16-byte row slices: VEC replica-typed elements <-> fp32 registers.
+template <typename T, int VEC>
+struct RowVec;
+
+template <>
+struct RowVec<float, 4> {
+    static __device__ __forceinline__ void unpack(const uint4 raw, float (&out)[4])
+    {
+        out[0] = __uint_as_float(raw.x), out[1] = __uint_as_float(raw.y);
+        out[2] = __uint_as_float(raw.z), out[3] = __uint_as_float(raw.w);
+    }
+    static __device__ __forceinline__ float narrow(float v) { return v; }
+    static __device__ __forceinline__ uint4 pack(const float (&in)[4])
+    {
+        return make_uint4(__float_as_uint(in[0]), __float_as_uint(in[1]), __float_as_uint(in[2]),
+                          __float_as_uint(in[3]));
+    }
+};
+
+template <>
+struct RowVec<__nv_bfloat16, 8> {
+    static __device__ __forceinline__ void unpack(const uint4 raw, float (&out)[8])
+    {
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            out[2 * k] = __uint_as_float(w[k] << 16);  // bf16 -> fp32 is exact
+            out[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
+        }
+    }
+    static __device__ __forceinline__ __nv_bfloat16 narrow(float v) { return __float2bfloat16_rn(v); }
+    static __device__ __forceinline__ uint4 pack(const float (&in)[8])
+    {
+        uint32_t w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const __nv_bfloat162 pair = __floats2bfloat162_rn(in[2 * k], in[2 * k + 1]);  // nearest-even
+            w[k] = *reinterpret_cast<const uint32_t*>(&pair);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+// Local SGD step of one lane: WPT workers (starting at the even worker w_first) x
+// VEC consecutive columns starting at column c, evaluated as
+//   v = x - gamma * ((x - b) + sigma * xi) = keep * x + gamma * b - (gamma * sigma) * xi,  keep = 1 - gamma.
+// One Philox draw serves a worker pair on four columns.
+template <int VEC, int WPT>
+__device__ __forceinline__ void local_sgd(const float (&xv)[WPT][VEC], const float (&bv)[WPT][VEC],
+                                          float (&v)[WPT][VEC], int64_t c, int w_first, const FusedParams& prm)
+{
+    static_assert(WPT % 2 == 0 && VEC % 4 == 0, "noise draws cover worker pairs and 4 columns");
+#pragma unroll
+    for (int w = 0; w < WPT; ++w)
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) v[w][e] = fmaf(prm.gamma, bv[w][e], prm.keep * xv[w][e]);
+    if (!prm.noisy) return;
+#pragma unroll
+    for (int w = 0; w < WPT; w += 2) {
+#pragma unroll
+        for (int q = 0; q < VEC / 4; ++q) {
+            const Philox4 r = philox4x32_10_keyed(prm.t_lo, prm.t_hi, (uint32_t)(c >> 2) + q,
+                                                  kStreamNoise | ((uint32_t)((w_first + w) >> 1) << 8), prm.round_key);
+            const uint32_t words[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+                const ScaledPair z = gaussian_pair(words[m], prm.noise_scale);
+                float(&row)[VEC] = v[w + (m >> 1)];  // words 0,1 -> worker w, words 2,3 -> worker w+1
+                const int k = 4 * q + 2 * (m & 1);
+                row[k] = fmaf(-z.radius, z.c, row[k]);
+                row[k + 1] = fmaf(-z.radius, z.s, row[k + 1]);
+            }
+        }
+    }
+}
+
+// s += v where `take` is set, as one predicated add (no branch, no select); a value that is
+// not taken never enters the sum, whatever it is.
+__device__ __forceinline__ void add_if(float& s, float v, uint32_t take)
+{
+    asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p add.f32 %0, %0, %1;\n\t}" : "+f"(s) : "f"(v), "r"(take));
+}
+
+template <int G>
+__device__ __forceinline__ float sum_over_groups(float s)
+{
+#pragma unroll
+    for (int off = 32 / G; off < 32; off <<= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
+    return s;
+}
+
+// Block (parameter server) of column c: columns are cut into n blocks of
+// block_cols = ceil(d / n) columns (Step 0, model partitioning).
+__device__ __forceinline__ int block_of(int64_t c, const FusedParams& prm)
+{
+    return prm.narrow ? (int)((uint32_t)c / (uint32_t)prm.block_cols) : (int)(c / prm.block_cols);
+}
+
+// What a lane needs to know about the masks: the words of block j, shifted so
+// that bit w is worker w_first + w, and 1 / |N^(j)|.
+struct MaskView {
+    const uint64_t* up;
+    const uint64_t* down;
+    const float* inv_cnt;  // 1 / cnt[j], 0 where cnt[j] == 0
+};
+
+// Remembers the block a lane was last in: lanes walk the columns upwards, so the block
+// index is recomputed (one division) only when a lane crosses into a new block.
+struct BlockCursor {
+    int64_t begin = 0, end = 0;  // columns [begin, end) belong to block j; empty at first
+    int j = 0;
+    __device__ __forceinline__ int locate(int64_t c, const FusedParams& prm)
+    {
+        if (c < begin || c >= end) {
+            j = block_of(c, prm);
+            begin = (int64_t)j * prm.block_cols;
+            end = begin + prm.block_cols;
+        }
+        return j;
+    }
+};
+
+// RS + AG for one lane after local_sgd: masked sum over the lane's workers, xor
+// butterfly over the G lane groups, multiply by 1/|N|, then every worker takes
+// the average where its down-bit is set and keeps v otherwise.  On return v
+// holds x_{t+1}; the result has bit e set iff column c + e exists (< d).  Lanes
+// whose VEC columns straddle two blocks or the end of the row send the whole
+// warp through the per-column path.  All lanes of the warp must call this
+// together.
+template <int VEC, int WPT, int G>
+__device__ __forceinline__ uint32_t average_and_select(float (&v)[WPT][VEC], int64_t c, bool col_live, int w_first,
+                                                       const MaskView& masks, BlockCursor& cursor,
+                                                       const FusedParams& prm)
+{
+    const int j_first = col_live ? cursor.locate(c, prm) : 0;
+    const bool uniform = !col_live || (c + VEC <= cursor.end && c + VEC <= prm.d);
+    if (__all_sync(0xFFFFFFFFu, uniform)) {
+        const uint32_t up = (uint32_t)(masks.up[j_first] >> w_first);
+        const uint32_t down = (uint32_t)(masks.down[j_first] >> w_first);
+        const float inv = masks.inv_cnt[j_first];
+        float s[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) s[e] = 0.0f;
+#pragma unroll
+        for (int w = 0; w < WPT; ++w) {
+            const uint32_t arrived = (up >> w) & 1u;  // worker's copy reached the server: it is in N
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) add_if(s[e], v[w][e], arrived);
+        }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) s[e] = sum_over_groups<G>(s[e]) * inv;  // 1/|N| * sum over N (RS step)
+#pragma unroll
+        for (int w = 0; w < WPT; ++w) {
+            const bool received = (down >> w) & 1u;  // AG step: receivers take the average
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) v[w][e] = received ? s[e] : v[w][e];
+        }
+        return col_live ? (1u << VEC) - 1u : 0u;
+    }
+    uint32_t live_bits = 0;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+        const bool live = c + e < prm.d;
+        const int j = live ? block_of(c + e, prm) : 0;
+        const uint32_t up = (uint32_t)(masks.up[j] >> w_first);
+        const uint32_t down = (uint32_t)(masks.down[j] >> w_first);
+        float s = 0.0f;
+#pragma unroll
+        for (int w = 0; w < WPT; ++w) add_if(s, v[w][e], (up >> w) & 1u);
+        const float avg = sum_over_groups<G>(s) * masks.inv_cnt[j];
+#pragma unroll
+        for (int w = 0; w < WPT; ++w) v[w][e] = ((down >> w) & 1u) ? avg : v[w][e];
+        live_bits |= (live ? 1u : 0u) << e;
+    }
+    return live_bits;
+}
+
+// Writes one worker's results at the ragged end of a row, element by element: only the columns
+// that exist (the padding between d and the row pitch is never written).
+template <typename T, int VEC>
+__device__ __forceinline__ void store_ragged(T* dst, const float (&vals)[VEC], uint32_t live_bits)
+{
+#pragma unroll
+    for (int e = 0; e < VEC; ++e)
+        if ((live_bits >> e) & 1u) dst[e] = RowVec<T, VEC>::narrow(vals[e]);
 }
 
 }  // namespace rps

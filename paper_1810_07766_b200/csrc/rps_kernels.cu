@@ -1,6 +1,6 @@
 // CUDA kernels of the RPS step for sm_100a: the Philox drop-mask generator, the
-// fused local-SGD + masked-average + masked-write-back pass, and an off-path
-// diagnostic reduction.  Host launch wrappers are at the bottom.
+// direct form of the fused local-SGD + masked-average + masked-write-back pass,
+// and an off-path diagnostic reduction.  Host launch wrappers are at the bottom.
 #include "rps_kernels.h"
 
 #include "rps_device.cuh"
@@ -64,199 +64,69 @@ __global__ void __launch_bounds__(256) rps_mask_kernel(const MaskParams prm)
             out->down[j] = down;
             out->cnt[j] = cnt;
             out->server[j] = server[j];
+            out->inv_cnt[j] = cnt > 0 ? 1.0f / (float)cnt : 0.0f;
         }
     }
 }
 
 // --------------------------------------------------------------------------
-// Fused step.  A warp owns LPG * VEC consecutive columns per iteration; its 32
-// lanes are G groups of LPG = 32 / G lanes.  Group g handles workers
-// g*WPT .. g*WPT + WPT - 1, lane `sub` of a group handles VEC consecutive columns
-// of each of those workers with one vector load per row, so a group reads whole
-// contiguous row segments.  Each lane keeps its WPT x VEC values of v in
-// registers, sums the ones whose up-bit is set, the G partial sums are combined
-// with xor-shuffles (every lane ends with the same total, bit for bit), and
-// each lane writes back either the average or its own v according to the
-// down-bit.  x is read once and written once, b is read once.
+// Fused step, direct form: every lane loads its row slices straight from global
+// memory into registers.  A warp owns LPG * VEC consecutive columns per
+// iteration; its 32 lanes are G groups of LPG = 32 / G lanes.  Group g handles
+// workers g*WPT .. g*WPT + WPT - 1, lane `sub` of a group handles VEC consecutive
+// columns of each of those workers with one 16-byte load per row, so a group
+// reads whole contiguous row segments.  x is read once and written once, b is
+// read once.  (The staged form in rps_staged.cu does the same arithmetic with
+// the loads decoupled from the warps through shared memory.)
 // --------------------------------------------------------------------------
-template <typename T, int VEC>
-struct RowVec;
-
-template <>
-struct RowVec<float, 4> {
-    static __device__ __forceinline__ void load(const float* p, float (&out)[4])
-    {
-        const float4 v = __ldcs(reinterpret_cast<const float4*>(p));
-        out[0] = v.x, out[1] = v.y, out[2] = v.z, out[3] = v.w;
-    }
-    static __device__ __forceinline__ void store(float* p, const float (&in)[4])
-    {
-        __stcs(reinterpret_cast<float4*>(p), make_float4(in[0], in[1], in[2], in[3]));
-    }
-};
-
-template <>
-struct RowVec<__nv_bfloat16, 8> {
-    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&out)[8])
-    {
-        const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p));
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            out[2 * k] = __uint_as_float(w[k] << 16);            // bf16 -> fp32 is exact
-            out[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
-        }
-    }
-    static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&in)[8])
-    {
-        uint32_t w[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const __nv_bfloat162 pair = __floats2bfloat162_rn(in[2 * k], in[2 * k + 1]);  // nearest-even
-            w[k] = *reinterpret_cast<const uint32_t*>(&pair);
-        }
-        __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
-    }
-};
-
-template <int G>
-__device__ __forceinline__ float sum_over_groups(float s)
-{
-#pragma unroll
-    for (int off = 32 / G; off < 32; off <<= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
-    return s;
-}
-
-__device__ __forceinline__ int block_of(int64_t c, const FusedParams& prm)
-{
-    // columns are cut into n blocks of block_cols = ceil(d / n) columns (Step 0)
-    return prm.narrow ? (int)((uint32_t)c / (uint32_t)prm.block_cols) : (int)(c / prm.block_cols);
-}
-
 template <typename T, int VEC, int WPT, int G, int THREADS>
-__global__ void __launch_bounds__(THREADS) rps_fused_kernel(const FusedParams prm)
+__global__ void __launch_bounds__(THREADS) rps_fused_direct_kernel(const FusedParams prm)
 {
-    static_assert(WPT % 2 == 0 && VEC % 4 == 0, "noise draws cover worker pairs and 4 columns");
     constexpr int LPG = 32 / G;
     constexpr int WARP_COLS = LPG * VEC;
     const int lane = threadIdx.x & 31;
     const int sub = lane % LPG;
     const int w_first = (lane / LPG) * WPT;  // first worker of this lane's group
     const int n = prm.n;
-    const int64_t d = prm.d;
     T* __restrict__ x = static_cast<T*>(prm.x);
     const T* __restrict__ b = static_cast<const T*>(prm.b);
-    const StepMasks* __restrict__ masks = prm.masks;
-    const float gamma = prm.gamma, sigma = prm.sigma;
+    const MaskView masks{prm.masks->up, prm.masks->down, prm.masks->inv_cnt};
 
     const int64_t warps_total = (int64_t)gridDim.x * (THREADS / 32);
-    const int64_t tiles = (d + WARP_COLS - 1) / WARP_COLS;
+    const int64_t tiles = (prm.d + WARP_COLS - 1) / WARP_COLS;
+    BlockCursor cursor;
     for (int64_t tile = (int64_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5); tile < tiles;
          tile += warps_total) {
         const int64_t c = tile * WARP_COLS + (int64_t)sub * VEC;
-        const bool col_live = c < d;  // the row pitch covers the whole vector even when c + VEC > d
+        const bool col_live = c < prm.d;  // the row pitch covers the whole slice even when c + VEC > d
 
-        float xv[WPT][VEC], v[WPT][VEC];
+        float v[WPT][VEC];
         {
-            float bv[WPT][VEC];
+            float xv[WPT][VEC], bv[WPT][VEC];
+            // lanes past the end of the row and workers past n read a real slice all the same (column
+            // 0 / the last row): their values are masked out and never stored
+            const int64_t c_read = col_live ? c : 0;
 #pragma unroll
             for (int w = 0; w < WPT; ++w) {
-                if (col_live && w_first + w < n) {
-                    const int64_t at = (int64_t)(w_first + w) * prm.pitch + c;
-                    RowVec<T, VEC>::load(x + at, xv[w]);
-                    RowVec<T, VEC>::load(b + at, bv[w]);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < VEC; ++e) xv[w][e] = bv[w][e] = 0.0f;
-                }
+                const int row = w_first + w < n ? w_first + w : n - 1;
+                const int64_t at = (int64_t)row * prm.pitch + c_read;
+                const uint4 raw_x = __ldcs(reinterpret_cast<const uint4*>(x + at));
+                const uint4 raw_b = __ldcs(reinterpret_cast<const uint4*>(b + at));
+                RowVec<T, VEC>::unpack(raw_x, xv[w]);
+                RowVec<T, VEC>::unpack(raw_b, bv[w]);
             }
-            // local SGD step: v = x - gamma * grad F_i(x; xi), grad = (x - b_i) + sigma * xi
-            if (sigma != 0.0f) {
-#pragma unroll
-                for (int w = 0; w < WPT; w += 2) {
-#pragma unroll
-                    for (int q = 0; q < VEC / 4; ++q) {
-                        const Philox4 r = philox4x32_10(prm.t_lo, prm.t_hi, (uint32_t)(c >> 2) + q,
-                                                        kStreamNoise | ((uint32_t)((w_first + w) >> 1) << 8),
-                                                        prm.key0, prm.key1);
-                        const float2 z0 = gaussian_pair(r.x), z1 = gaussian_pair(r.y);
-                        const float2 z2 = gaussian_pair(r.z), z3 = gaussian_pair(r.w);
-                        const float za[4] = {z0.x, z0.y, z1.x, z1.y};
-                        const float zb[4] = {z2.x, z2.y, z3.x, z3.y};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int k = 4 * q + e;
-                            v[w][k] = fmaf(-gamma, fmaf(sigma, za[e], xv[w][k] - bv[w][k]), xv[w][k]);
-                            v[w + 1][k] = fmaf(-gamma, fmaf(sigma, zb[e], xv[w + 1][k] - bv[w + 1][k]), xv[w + 1][k]);
-                        }
-                    }
-                }
-            } else {
-#pragma unroll
-                for (int w = 0; w < WPT; ++w)
-#pragma unroll
-                    for (int e = 0; e < VEC; ++e) v[w][e] = fmaf(-gamma, xv[w][e] - bv[w][e], xv[w][e]);
-            }
+            local_sgd<VEC, WPT>(xv, bv, v, c, w_first, prm);
         }
-
-        const int j_first = col_live ? block_of(c, prm) : 0;
-        const bool uniform = !col_live || (c + VEC <= d && block_of(c + VEC - 1, prm) == j_first);
-        if (__all_sync(0xFFFFFFFFu, uniform)) {
-            // all VEC columns of this lane lie in one block: one mask word serves them
-            const uint32_t up = (uint32_t)(masks->up[j_first] >> w_first);
-            const uint32_t down = (uint32_t)(masks->down[j_first] >> w_first);
-            const int cnt = masks->cnt[j_first];
-            float avg[VEC];
+        const uint32_t live_bits = average_and_select<VEC, WPT, G>(v, c, col_live, w_first, masks, cursor, prm);
+        T* dst = x + (int64_t)w_first * prm.pitch + c;  // this lane's slice of its first worker's row
+        if (live_bits == (1u << VEC) - 1u) {
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) {
-                float s = 0.0f;
+            for (int w = 0; w < WPT; ++w, dst += prm.pitch)
+                if (w_first + w < n) __stcs(reinterpret_cast<uint4*>(dst), RowVec<T, VEC>::pack(v[w]));
+        } else if (live_bits != 0) {
 #pragma unroll
-                for (int w = 0; w < WPT; ++w) s += ((up >> w) & 1u) ? v[w][e] : 0.0f;
-                s = sum_over_groups<G>(s);
-                avg[e] = cnt > 0 ? s / (float)cnt : 0.0f;  // 1/|N| * sum over N (RS step)
-            }
-            if (col_live) {
-#pragma unroll
-                for (int w = 0; w < WPT; ++w) {
-                    if (w_first + w < n) {
-                        float out[VEC];
-#pragma unroll
-                        for (int e = 0; e < VEC; ++e) out[e] = ((down >> w) & 1u) ? avg[e] : v[w][e];  // AG step
-                        RowVec<T, VEC>::store(x + (int64_t)(w_first + w) * prm.pitch + c, out);
-                    }
-                }
-            }
-        } else {
-            // a lane of this warp straddles a block boundary or the end of the row:
-            // every column looks up its own block
-            float avg[VEC];
-            uint32_t down[VEC];
-            bool live[VEC];
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) {
-                live[e] = c + e < d;
-                const int j = live[e] ? block_of(c + e, prm) : 0;
-                const uint32_t up = (uint32_t)(masks->up[j] >> w_first);
-                down[e] = (uint32_t)(masks->down[j] >> w_first);
-                const int cnt = masks->cnt[j];
-                float s = 0.0f;
-#pragma unroll
-                for (int w = 0; w < WPT; ++w) s += ((up >> w) & 1u) ? v[w][e] : 0.0f;
-                s = sum_over_groups<G>(s);
-                avg[e] = cnt > 0 ? s / (float)cnt : 0.0f;
-            }
-            if (col_live) {
-#pragma unroll
-                for (int w = 0; w < WPT; ++w) {
-                    if (w_first + w < n) {
-                        float out[VEC];
-#pragma unroll
-                        for (int e = 0; e < VEC; ++e)
-                            out[e] = !live[e] ? xv[w][e] : (((down[e] >> w) & 1u) ? avg[e] : v[w][e]);
-                        RowVec<T, VEC>::store(x + (int64_t)(w_first + w) * prm.pitch + c, out);
-                    }
-                }
-            }
+            for (int w = 0; w < WPT; ++w, dst += prm.pitch)
+                if (w_first + w < n) store_ragged<T, VEC>(dst, v[w], live_bits);
         }
     }
 }
@@ -332,7 +202,7 @@ namespace {
 constexpr int kThreads = 256;
 
 template <typename T, int VEC, int WPT, int G>
-cudaError_t launch_fused_as(const FusedParams& prm, int sm_count, cudaStream_t stream)
+cudaError_t launch_direct_as(const FusedParams& prm, int sm_count, cudaStream_t stream)
 {
     constexpr int warp_cols = (32 / G) * VEC;
     const int64_t tiles = (prm.d + warp_cols - 1) / warp_cols;
@@ -341,7 +211,7 @@ cudaError_t launch_fused_as(const FusedParams& prm, int sm_count, cudaStream_t s
     if (per_sm == 0) {
         int occ = 0;
         cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-            &occ, rps_fused_kernel<T, VEC, WPT, G, kThreads>, kThreads, 0);
+            &occ, rps_fused_direct_kernel<T, VEC, WPT, G, kThreads>, kThreads, 0);
         if (err != cudaSuccess) return err;
         per_sm = occ < 1 ? 1 : occ;
     }
@@ -349,28 +219,62 @@ cudaError_t launch_fused_as(const FusedParams& prm, int sm_count, cudaStream_t s
     int64_t grid = (int64_t)sm_count * per_sm;
     if (grid > ctas_needed) grid = ctas_needed;
     if (grid < 1) grid = 1;
-    rps_fused_kernel<T, VEC, WPT, G, kThreads><<<(unsigned)grid, kThreads, 0, stream>>>(prm);
+    rps_fused_direct_kernel<T, VEC, WPT, G, kThreads><<<(unsigned)grid, kThreads, 0, stream>>>(prm);
     return cudaGetLastError();
 }
 
 template <typename T, int VEC>
-cudaError_t launch_fused_for_n(const FusedParams& prm, int sm_count, cudaStream_t stream)
+cudaError_t launch_direct_for_n(const FusedParams& prm, int wpt, int sm_count, cudaStream_t stream)
 {
     const int n = prm.n;
-    if (n <= 2) return launch_fused_as<T, VEC, 2, 1>(prm, sm_count, stream);
-    if (n <= 4) return launch_fused_as<T, VEC, 4, 1>(prm, sm_count, stream);
-    if (n <= 8) return launch_fused_as<T, VEC, 8, 1>(prm, sm_count, stream);
-    if (n <= 16) return launch_fused_as<T, VEC, 8, 2>(prm, sm_count, stream);
-    if (n <= 32) return launch_fused_as<T, VEC, 8, 4>(prm, sm_count, stream);
-    return launch_fused_as<T, VEC, 8, 8>(prm, sm_count, stream);
+    if (wpt == 4) {
+        if (n <= 4) return launch_direct_as<T, VEC, 4, 1>(prm, sm_count, stream);
+        if (n <= 8) return launch_direct_as<T, VEC, 4, 2>(prm, sm_count, stream);
+        if (n <= 16) return launch_direct_as<T, VEC, 4, 4>(prm, sm_count, stream);
+        if (n <= 32) return launch_direct_as<T, VEC, 4, 8>(prm, sm_count, stream);
+        return launch_direct_as<T, VEC, 4, 16>(prm, sm_count, stream);
+    }
+    if (n <= 2) return launch_direct_as<T, VEC, 2, 1>(prm, sm_count, stream);
+    if (n <= 4) return launch_direct_as<T, VEC, 4, 1>(prm, sm_count, stream);
+    if (n <= 8) return launch_direct_as<T, VEC, 8, 1>(prm, sm_count, stream);
+    if (n <= 16) return launch_direct_as<T, VEC, 8, 2>(prm, sm_count, stream);
+    if (n <= 32) return launch_direct_as<T, VEC, 8, 4>(prm, sm_count, stream);
+    return launch_direct_as<T, VEC, 8, 8>(prm, sm_count, stream);
 }
 
 }  // namespace
 
-cudaError_t launch_fused(const FusedParams& prm, bool bf16, int sm_count, cudaStream_t stream)
+cudaError_t launch_fused_direct(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
+                                cudaStream_t stream)
 {
-    if (bf16) return launch_fused_for_n<__nv_bfloat16, 8>(prm, sm_count, stream);
-    return launch_fused_for_n<float, 4>(prm, sm_count, stream);
+    if (bf16) return launch_direct_for_n<__nv_bfloat16, 8>(prm, tune.workers_per_lane, sm_count, stream);
+    return launch_direct_for_n<float, 4>(prm, tune.workers_per_lane, sm_count, stream);
+}
+
+cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
+                         cudaStream_t stream)
+{
+    if (tune.kernel == 1) return launch_fused_direct(prm, tune, bf16, sm_count, stream);
+    return launch_fused_staged(prm, tune, bf16, sm_count, stream);
+}
+
+void set_philox_key(FusedParams& prm, uint64_t seed)
+{
+    prm.key0 = (uint32_t)seed;
+    prm.key1 = (uint32_t)(seed >> 32);
+    for (uint32_t r = 0; r < 10; ++r) {
+        prm.round_key[r][0] = prm.key0 + r * 0x9E3779B9u;
+        prm.round_key[r][1] = prm.key1 + r * 0xBB67AE85u;
+    }
+}
+
+void set_sgd_scalars(FusedParams& prm, float gamma, float sigma)
+{
+    prm.gamma = gamma;
+    prm.keep = 1.0f - gamma;
+    const double gs = (double)gamma * (double)sigma;
+    prm.noise_scale = (float)(-2.0 * 0.6931471805599453 * gs * gs);
+    prm.noisy = sigma != 0.0f;
 }
 
 cudaError_t launch_diag(const DiagParams& prm, bool bf16, int sm_count, cudaStream_t stream)

@@ -6,9 +6,9 @@
 
 namespace rps {
 
-struct StepMasks;  // defined in rps_device.cuh; 1536 bytes per step
+struct StepMasks;  // defined in rps_device.cuh
 
-constexpr size_t kStepMasksBytes = 64 * 8 * 2 + 64 * 4 * 2;
+constexpr size_t kStepMasksBytes = 64 * 8 * 2 + 64 * 4 * 3;  // 1792 bytes per step
 
 struct MaskParams {
     StepMasks* out;           // [steps] mask records, device
@@ -20,19 +20,40 @@ struct MaskParams {
     int32_t assign_perm;
 };
 
+// Which fused kernel runs and how it is shaped; 0 everywhere = the library's choice.
+struct FusedTuning {
+    int32_t kernel;            // 1 direct (register loads), 2 staged (bulk-async copies into shared memory)
+    int32_t workers_per_lane;  // 2, 4 or 8
+    int32_t stages;            // shared-memory ring depth of the staged kernel
+    int32_t consumer_warps;    // compute warps per CTA of the staged kernel
+    int32_t copy_mode;         // staged kernel: 1 one bulk copy per row, 2 two-dimensional TMA boxes
+};
+
 struct FusedParams {
     void* x;        // [n][pitch] replicas, updated in place
     const void* b;  // [n][pitch] targets of the quadratic objective
     const StepMasks* masks;
+    int32_t* error;      // device word set non-zero when a bounded wait gave up (may be NULL)
     int64_t pitch;       // row pitch in elements
     int64_t d;           // model size
     int64_t block_cols;  // ceil(d / n): columns per parameter-server block
     int32_t n;
     int32_t narrow;  // d < 2^31: block index by 32-bit division
-    float gamma, sigma;
+    // v = keep * x + gamma * b - (gamma * sigma) * xi
+    float keep;         // 1 - gamma
+    float gamma;
+    float noise_scale;  // -2 ln 2 * (gamma * sigma)^2
+    int32_t noisy;      // sigma != 0
     uint32_t t_lo, t_hi;
     uint32_t key0, key1;
+    uint32_t round_key[10][2];  // Philox round keys: key + r * (0x9E3779B9, 0xBB67AE85)
 };
+
+// Fills key0, key1 and round_key from the 64-bit seed.
+void set_philox_key(FusedParams& prm, uint64_t seed);
+
+// Fills keep, gamma, noise_scale and noisy from the float learning rate and noise level.
+void set_sgd_scalars(FusedParams& prm, float gamma, float sigma);
 
 struct DiagParams {
     const void* x;
@@ -44,7 +65,12 @@ struct DiagParams {
 };
 
 cudaError_t launch_masks(const MaskParams& prm, int steps, cudaStream_t stream);
-cudaError_t launch_fused(const FusedParams& prm, bool bf16, int sm_count, cudaStream_t stream);
+cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
+                         cudaStream_t stream);
+cudaError_t launch_fused_direct(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
+                                cudaStream_t stream);
+cudaError_t launch_fused_staged(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
+                                cudaStream_t stream);
 cudaError_t launch_diag(const DiagParams& prm, bool bf16, int sm_count, cudaStream_t stream);
 
 }  // namespace rps

@@ -17,7 +17,7 @@
 
 namespace {
 
-// Drop masks of ONE step for up to RPS_MAX_WORKERS workers (1536 bytes).  Every GPU
+// Drop masks of ONE step for up to RPS_MAX_WORKERS workers (1792 bytes).  Every GPU
 // that loads the library holds this array until the process exits.  In host code
 // the name below is only a stand-in for the symbol, not a device address: its
 // address on a device comes from cudaGetSymbolAddress (see device_state()).
@@ -66,7 +66,7 @@ extern "C" int rps_step_static(int n, int64_t d, int dtype, void* x_dev, const v
     if (!(p >= 0.0 && p <= 1.0) || !std::isfinite(gamma) || !std::isfinite(sigma) || sigma < 0.0) return RPS_EINVAL;
     if (!x_dev || !b_dev || ((uintptr_t)x_dev | (uintptr_t)b_dev) % 128 != 0) return RPS_EINVAL;
     const int64_t per_line = dtype == RPS_BF16 ? 64 : 32;
-    if (pitch != (d + per_line - 1) / per_line * per_line) return RPS_EINVAL;
+    if (pitch < d || pitch % per_line != 0) return RPS_EINVAL;
 
     DeviceState* st = nullptr;
     int rc = device_state(&st);
@@ -94,12 +94,12 @@ extern "C" int rps_step_static(int n, int64_t d, int dtype, void* x_dev, const v
     fp.block_cols = (d + n - 1) / n;
     fp.n = n;
     fp.narrow = d < ((int64_t)1 << 31);
-    fp.gamma = (float)gamma;
-    fp.sigma = (float)sigma;
+    fp.error = nullptr;  // nobody reads back here; a wait that gives up just ends the kernel early
+    rps::set_sgd_scalars(fp, (float)gamma, (float)sigma);
     fp.t_lo = (uint32_t)t;
     fp.t_hi = (uint32_t)(t >> 32);
-    fp.key0 = (uint32_t)seed;
-    fp.key1 = (uint32_t)(seed >> 32);
-    if (rps::launch_fused(fp, dtype == RPS_BF16, st->sm_count, stream) != cudaSuccess) return RPS_ECUDA;
+    rps::set_philox_key(fp, seed);
+    if (rps::launch_fused(fp, rps::FusedTuning{}, dtype == RPS_BF16, st->sm_count, stream) != cudaSuccess)
+        return RPS_ECUDA;
     return RPS_OK;
 }

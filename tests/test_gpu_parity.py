@@ -283,14 +283,36 @@ def test_edge_shapes(rps_mod, oracle, n, d, dtype):
         want = wl.make_initial(w)
         oracle.run(want, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps,
                    self_delivery=sd, assign=assign)
-        r = make(rps_mod, w, self_delivery=sd, assign=assign)
+        for kernel, copy_mode in ((1, 0), (2, 1), (2, 2)):
+            r = make(rps_mod, w, self_delivery=sd, assign=assign, kernel=kernel, copy_mode=copy_mode)
+            r.set_targets(b)
+            r.x_dev[:, d:] = 3.0         # sentinel in the padding between d and the row pitch
+            r.step_n(w.steps)
+            got = r.read()
+            assert_close(w, got, want, BF16_TOL if dtype == "bf16" else 3 * STEP_TOL)
+            assert (r.x_dev[:, d:].float() == 3.0).all()      # never written
+            r.close()
+
+
+# every shape of the fused kernel computes the same step:
+# (kernel, workers_per_lane, stages, consumer_warps, copy_mode)
+VARIANTS = [(1, 0, 0, 0, 0), (1, 4, 0, 0, 0), (2, 0, 0, 0, 0), (2, 2, 0, 0, 1), (2, 4, 2, 4, 2), (2, 8, 4, 3, 1),
+            (2, 4, 5, 16, 2), (2, 2, 8, 1, 2), (2, 8, 2, 8, 2), (2, 4, 3, 5, 1), (2, 8, 2, 12, 1)]
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
+def test_kernel_variants(rps_mod, oracle, name):
+    w = TWINS[name].scaled(d=TWINS[name].d // 2 + (3 if name != "cfg5" else 0), steps=3)
+    b = wl.make_targets(w)
+    want = wl.make_initial(w)
+    oracle.run(want, b, dtype=w.dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps)
+    for kernel, wpt, stages, warps, copy_mode in VARIANTS:
+        r = make(rps_mod, w, kernel=kernel, workers_per_lane=wpt, stages=stages, consumer_warps=warps,
+                 copy_mode=copy_mode)
         r.set_targets(b)
         r.step_n(w.steps)
         got = r.read()
-        assert_close(w, got, want, BF16_TOL if dtype == "bf16" else 3 * STEP_TOL)
-        # the padding between d and the row pitch is never disturbed
-        pad = r.x_dev[:, d:].float().cpu().numpy()
-        assert not pad.any()
+        assert_close(w, got, want, BF16_TOL if w.dtype == "bf16" else 3 * STEP_TOL)
         r.close()
 
 
@@ -307,6 +329,7 @@ def test_guard_bands_around_device_buffers(rps_mod):
     assert (r.b_dev[:, w.d:] == 7.0).all()
     assert (r.scratch[-128:] == tail).all()
     assert not r.x_dev[:, w.d:].any()
+    r.read()                              # also checks the kernels' error word
     r.close()
 
 
