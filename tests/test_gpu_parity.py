@@ -362,3 +362,41 @@ def test_profile_counts_launches(rps_mod):
     r.profile(False)
     assert r.launch_count() == 10
     r.close()
+
+
+# ------------------------------------------------------------------ full sizes, sampled columns
+
+def sampled_columns(w, rng, count=4096):
+    """Random columns plus the first and last few columns of every block and of the row."""
+    block = -(-w.d // w.n)
+    edges = [0, 1, 2, 3, w.d - 4, w.d - 3, w.d - 2, w.d - 1]
+    for j in range(1, w.n):
+        for off in (-5, -4, -3, -2, -1, 0, 1, 2, 3, 4):
+            edges.append(j * block + off)
+    cols = np.concatenate([rng.integers(0, w.d, size=count), np.array(edges)])
+    return np.unique(cols[(cols >= 0) & (cols < w.d)]).astype(np.int64)
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
+def test_full_size_sampled_columns(rps_mod, oracle, name):
+    """The workload at its full size, in the launch configuration the benchmark times (library
+    defaults): T = 3 free-running steps, checked on sampled columns that the oracle recomputes
+    from the same inputs (columns evolve independently of one another)."""
+    w = wl.WORKLOADS[name]
+    steps = 3
+    b = wl.make_targets(w)
+    cols = sampled_columns(w, np.random.default_rng(w.seed))
+    want = np.ascontiguousarray(wl.make_initial(w)[:, cols])
+    b_cols = np.ascontiguousarray(b[:, cols])
+    for t in range(steps):
+        oracle.step_columns(w.d, cols, want, b_cols, dtype=w.dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t=t)
+    r = make(rps_mod, w)
+    r.set_targets(b)
+    del b
+    r.step_n(steps)
+    got = r.read()[:, cols]
+    assert_close(w, got, want, BF16_TOL if w.dtype == "bf16" else 3 * STEP_TOL)
+    for t in range(steps):
+        assert all((a == o).all() for a, o in zip(r.read_masks(t), oracle.masks(w.n, w.p, w.seed, t)))
+    r.close()
+    torch.cuda.empty_cache()
