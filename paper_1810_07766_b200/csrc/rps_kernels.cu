@@ -256,10 +256,11 @@ cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool b
 {
     if (tune.kernel == 1) return launch_fused_direct(prm, tune, bf16, sm_count, stream);
     if (tune.kernel == 0) {
-        // A model this short gives the staged kernel's ring fewer than a couple of tiles per SM: there
+        // A model this short gives the staged kernel's ring less than a tile per SM: there
         // is nothing to pipeline and its set-up dominates; the step is launch bound and L2 resident.
         const int64_t bytes_per_column = (int64_t)prm.n * (bf16 ? 2 : 4);
-        if (prm.d * bytes_per_column < (int64_t)sm_count * 2 * 32768) return launch_fused_direct(prm, tune, bf16, sm_count, stream);
+        if (prm.d * bytes_per_column < (int64_t)sm_count * 8192)
+            return launch_fused_direct(prm, tune, bf16, sm_count, stream);
     }
     return launch_fused_staged(prm, tune, bf16, sm_count, stream);
 }
