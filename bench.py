@@ -34,8 +34,9 @@ FALLBACK_HBM_GBS = 6650.0
 # the ncu capture summarised under profiles/, keyed by workload; valid only for the kernel
 # sources whose digest is recorded with it.
 NCU_TRAFFIC = {
-    "kernel_digest": None,
-    "bytes_per_launch": {},
+    "kernel_digest": "d9cb96b9944b0c40",
+    "bytes_per_launch": {"cfg2": 1022099456, "cfg4": 1492908032,
+                         "cfg5": 6073307136},  # cfg5: the d = 2,097,152 capture x 8 (traffic is proportional to d)
 }
 
 
@@ -46,6 +47,14 @@ def kernel_digest() -> str:
         with open(os.path.join(csrc, name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
+
+
+def fused_kernel_name(args, w) -> str:
+    """Which fused kernel the library picks for this workload (see launch_fused in csrc/rps_kernels.cu)."""
+    small = w.n * w.d * w.elem_bytes < 148 * 8192
+    if args.kernel == 1 or (args.kernel == 0 and small):
+        return "rps_fused_direct_kernel"
+    return "rps_fused_staged_kernel"
 
 
 def measured_peak_gbs():
@@ -242,7 +251,8 @@ def run_cuda(args):
     fused_avg_ms = fused_ms / max(fused_n, 1)
     achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
     traffic = None
-    if NCU_TRAFFIC["kernel_digest"] == kernel_digest():
+    default_shape = not (args.kernel or args.workers_per_lane or args.stages or args.consumer_warps or args.copy_mode)
+    if default_shape and NCU_TRAFFIC["kernel_digest"] == kernel_digest():
         traffic = NCU_TRAFFIC["bytes_per_launch"].get(w.name)
 
     line = {
@@ -264,7 +274,7 @@ def run_cuda(args):
         "e2e": e2e,
         "gpu_launches": gpu_launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "rps_fused_kernel",
+                     "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": fused_kernel_name(args, w),
                      "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n,
                      "mask_kernel_ms_per_launch": mask_ms / max(mask_n, 1), "mask_launches_timed": mask_n},
     }
