@@ -23,7 +23,8 @@
  *     bfloat16 bit patterns in uint16_t).  On the device a row occupies
  *     rps_pitch() elements (d rounded up so that every row starts on a 128-byte
  *     boundary, plus row_skew_lines lines); columns d..pitch-1 are padding that
- *     the library reads but never writes.
+ *     belongs to the library: it reads it, may zero the few padding columns that
+ *     share a 16-byte unit with column d-1, and leaves the rest as it found it.
  */
 #ifndef RPS_H
 #define RPS_H
@@ -80,9 +81,14 @@ typedef struct rps_options {
                                  asynchronous copies (default)                               */
     int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */
     int32_t stages;           /* depth of the shared-memory ring of kernel 2 (2..8)          */
-    int32_t consumer_warps;   /* compute warps per CTA of kernel 2 (1..16)                   */
+    int32_t consumer_warps;   /* compute warps per CTA of kernel 2 (1..24; shapes that need
+                                 many registers are clamped lower)                           */
     int32_t copy_mode;        /* kernel 2 fills a stage with 1: one bulk copy per row,
                                  2: two-dimensional TMA boxes covering all n rows            */
+    int32_t slice_bytes;      /* kernel 2, bf16 replicas: bytes of a row handled by one lane,
+                                 16 or 8 (8 = more, lighter warps per tile)                  */
+    int32_t store_mode;       /* kernel 2 writes results 1: from registers, 16 bytes per lane,
+                                 2: through shared memory with TMA tensor stores             */
 } rps_options;
 
 /*

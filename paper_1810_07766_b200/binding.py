@@ -36,7 +36,8 @@ class rps_options(ctypes.Structure):
                 ("mask_window", ctypes.c_int32), ("sigma", ctypes.c_double), ("row_skew_lines", ctypes.c_int32),
                 ("kernel", ctypes.c_int32),
                 ("workers_per_lane", ctypes.c_int32), ("stages", ctypes.c_int32), ("consumer_warps", ctypes.c_int32),
-                ("copy_mode", ctypes.c_int32)]
+                ("copy_mode", ctypes.c_int32), ("slice_bytes", ctypes.c_int32),
+                ("store_mode", ctypes.c_int32)]
 
 
 class RPSError(RuntimeError):
@@ -112,7 +113,7 @@ class RPS:
     def __init__(self, n: int, d: int, p: float, gamma: float, seed: int, *, dtype: str = "f32", sigma: float = 0.0,
                  assign: int = RPS_ASSIGN_FIXED, self_delivery: bool = True, mask_window: int = 32,
                  kernel: int = 0, workers_per_lane: int = 0, stages: int = 0, consumer_warps: int = 0,
-                 row_skew_lines: int = -1, copy_mode: int = 0, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+                 row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         if not torch.cuda.is_available():
@@ -126,7 +127,8 @@ class RPS:
         opt.dtype, opt.assign, opt.self_delivery = _DTYPE[dtype], assign, int(self_delivery)
         opt.mask_window, opt.sigma = mask_window, sigma
         opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps = kernel, workers_per_lane, stages, consumer_warps
-        opt.row_skew_lines, opt.copy_mode = row_skew_lines, copy_mode
+        opt.row_skew_lines, opt.copy_mode, opt.slice_bytes = row_skew_lines, copy_mode, slice_bytes
+        opt.store_mode = store_mode
         self._check(self._lib.rps_configure(self._h, ctypes.byref(opt)), "rps_configure")
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
         self.pitch = int(self._lib.rps_pitch(self._h))

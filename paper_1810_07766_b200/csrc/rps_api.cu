@@ -76,7 +76,7 @@ struct rps_handle {
     int32_t* error_word() const { return reinterpret_cast<int32_t*>(scratch + kErrorOffset); }
     rps::FusedTuning tuning() const
     {
-        return rps::FusedTuning{opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps, opt.copy_mode};
+        return rps::FusedTuning{opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps, opt.copy_mode, opt.slice_bytes, opt.store_mode};
     }
     rps::StepMasks* window() const { return reinterpret_cast<rps::StepMasks*>(scratch + kDiagBytes); }
     rps::StepMasks* probe() const { return window() + opt.mask_window; }
@@ -246,6 +246,8 @@ int rps_default_options(rps_options* opt)
     opt->stages = 0;
     opt->consumer_warps = 0;
     opt->copy_mode = 0;
+    opt->slice_bytes = 0;
+    opt->store_mode = 0;
     return RPS_OK;
 }
 
@@ -315,8 +317,11 @@ int rps_configure(rps_handle* h, const rps_options* opt)
         opt->workers_per_lane != 8)
         return fail(h, RPS_EINVAL, "workers_per_lane must be 0 (auto), 2, 4 or 8");
     if (opt->stages != 0 && (opt->stages < 2 || opt->stages > 8)) return fail(h, RPS_EINVAL, "stages must be 0 or 2..8");
-    if (opt->consumer_warps < 0 || opt->consumer_warps > 16)
-        return fail(h, RPS_EINVAL, "consumer_warps must be 0 (auto) or 1..16");
+    if (opt->consumer_warps < 0 || opt->consumer_warps > 24)
+        return fail(h, RPS_EINVAL, "consumer_warps must be 0 (auto) or 1..24");
+    if (opt->slice_bytes != 0 && opt->slice_bytes != 8 && opt->slice_bytes != 16)
+        return fail(h, RPS_EINVAL, "slice_bytes must be 0 (auto), 8 or 16");
+    if (opt->store_mode < 0 || opt->store_mode > 2) return fail(h, RPS_EINVAL, "store_mode must be 0 (auto), 1 or 2");
     if (opt->copy_mode < 0 || opt->copy_mode > 2) return fail(h, RPS_EINVAL, "copy_mode must be 0 (auto), 1 or 2");
     h->opt = *opt;
     h->sigma = (float)opt->sigma;

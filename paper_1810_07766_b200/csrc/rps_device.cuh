@@ -106,12 +106,13 @@ __device__ __forceinline__ ScaledPair gaussian_pair(uint32_t word, float noise_s
     return out;
 }
 
-// 16-byte row slices: VEC replica-typed elements <-> fp32 registers.
+// Row slices of one lane: VEC replica-typed elements (16 bytes, or 8 for the narrow bf16 form) <-> fp32 registers.
 template <typename T, int VEC>
 struct RowVec;
 
 template <>
 struct RowVec<float, 4> {
+    using Raw = uint4;
     static __device__ __forceinline__ void unpack(const uint4 raw, float (&out)[4])
     {
         out[0] = __uint_as_float(raw.x), out[1] = __uint_as_float(raw.y);
@@ -127,6 +128,7 @@ struct RowVec<float, 4> {
 
 template <>
 struct RowVec<__nv_bfloat16, 8> {
+    using Raw = uint4;
     static __device__ __forceinline__ void unpack(const uint4 raw, float (&out)[8])
     {
         const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
@@ -146,6 +148,23 @@ struct RowVec<__nv_bfloat16, 8> {
             w[k] = *reinterpret_cast<const uint32_t*>(&pair);
         }
         return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+// 8-byte slices of bf16 rows: half the columns per lane, so twice the lanes (and warps) per tile.
+template <>
+struct RowVec<__nv_bfloat16, 4> {
+    using Raw = uint2;
+    static __device__ __forceinline__ void unpack(const uint2 raw, float (&out)[4])
+    {
+        out[0] = __uint_as_float(raw.x << 16), out[1] = __uint_as_float(raw.x & 0xFFFF0000u);
+        out[2] = __uint_as_float(raw.y << 16), out[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+    }
+    static __device__ __forceinline__ __nv_bfloat16 narrow(float v) { return __float2bfloat16_rn(v); }
+    static __device__ __forceinline__ uint2 pack(const float (&in)[4])
+    {
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(in[0], in[1]), hi = __floats2bfloat162_rn(in[2], in[3]);
+        return make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
     }
 };
 
@@ -231,7 +250,7 @@ struct BlockCursor {
 // RS + AG for one lane after local_sgd: masked sum over the lane's workers, xor
 // butterfly over the G lane groups, multiply by 1/|N|, then every worker takes
 // the average where its down-bit is set and keeps v otherwise.  On return v
-// holds x_{t+1}; the result has bit e set iff column c + e exists (< d).  Lanes
+// holds x_{t+1} (0 for columns that do not exist); the result has bit e set iff column c + e exists (< d).  Lanes
 // whose VEC columns straddle two blocks or the end of the row send the whole
 // warp through the per-column path.  All lanes of the warp must call this
 // together.
@@ -277,7 +296,7 @@ __device__ __forceinline__ uint32_t average_and_select(float (&v)[WPT][VEC], int
         for (int w = 0; w < WPT; ++w) add_if(s, v[w][e], (up >> w) & 1u);
         const float avg = sum_over_groups<G>(s) * masks.inv_cnt[j];
 #pragma unroll
-        for (int w = 0; w < WPT; ++w) v[w][e] = ((down >> w) & 1u) ? avg : v[w][e];
+        for (int w = 0; w < WPT; ++w) v[w][e] = !live ? 0.0f : (((down >> w) & 1u) ? avg : v[w][e]);
         live_bits |= (live ? 1u : 0u) << e;
     }
     return live_bits;

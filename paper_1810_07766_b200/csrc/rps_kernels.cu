@@ -110,8 +110,9 @@ __global__ void __launch_bounds__(THREADS) rps_fused_direct_kernel(const FusedPa
             for (int w = 0; w < WPT; ++w) {
                 const int row = w_first + w < n ? w_first + w : n - 1;
                 const int64_t at = (int64_t)row * prm.pitch + c_read;
-                const uint4 raw_x = __ldcs(reinterpret_cast<const uint4*>(x + at));
-                const uint4 raw_b = __ldcs(reinterpret_cast<const uint4*>(b + at));
+                using Raw = typename RowVec<T, VEC>::Raw;
+                const Raw raw_x = __ldcs(reinterpret_cast<const Raw*>(x + at));
+                const Raw raw_b = __ldcs(reinterpret_cast<const Raw*>(b + at));
                 RowVec<T, VEC>::unpack(raw_x, xv[w]);
                 RowVec<T, VEC>::unpack(raw_b, bv[w]);
             }
@@ -122,7 +123,8 @@ __global__ void __launch_bounds__(THREADS) rps_fused_direct_kernel(const FusedPa
         if (live_bits == (1u << VEC) - 1u) {
 #pragma unroll
             for (int w = 0; w < WPT; ++w, dst += prm.pitch)
-                if (w_first + w < n) __stcs(reinterpret_cast<uint4*>(dst), RowVec<T, VEC>::pack(v[w]));
+                if (w_first + w < n)
+                    __stcs(reinterpret_cast<typename RowVec<T, VEC>::Raw*>(dst), RowVec<T, VEC>::pack(v[w]));
         } else if (live_bits != 0) {
 #pragma unroll
             for (int w = 0; w < WPT; ++w, dst += prm.pitch)

@@ -16,8 +16,10 @@
 // Consumer warp w of a CTA owns columns [w * WARP_COLS, (w+1) * WARP_COLS) of
 // the tile and maps its lanes to (worker group, 16-byte column slice) exactly as
 // the direct kernel does; the arithmetic is the same code (rps_device.cuh).
-// Results go from registers straight to global memory with 16-byte streaming
-// stores.
+// Results leave either straight from registers with 16-byte streaming stores,
+// or, where a lane group would write less than a full line per row (many
+// workers), through a double-buffered tile in shared memory and TMA tensor
+// stores of whole boxes (clipped at column d by the tensor map).
 //
 // Every wait on an mbarrier is bounded (2 s of %globaltimer); a wait that gives
 // up records a code in *prm.error and the warp leaves the kernel.
@@ -34,7 +36,9 @@ namespace {
 constexpr int kMaxStages = 8;
 constexpr int kMaxConsumerWarps = 16;
 constexpr int kMaxBoxCols = 256;  // a TMA box is at most 256 elements wide
-constexpr uint32_t kSmemHeaderBytes = 128 + 2 * kMaxWorkers * 8 + kMaxWorkers * 4;  // barriers + mask copy
+constexpr uint32_t kSmemHeaderBytes = 128 + 2 * kMaxWorkers * 8 + kMaxWorkers * 4 + 128;  // barriers, mask copy, flags
+constexpr uint32_t kAbortFlagOffset = kSmemHeaderBytes - 128;
+constexpr int kOutBuffers = 2;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 static_assert(kSmemHeaderBytes % 128 == 0, "tile data must start on a 128-byte boundary");
 
@@ -51,6 +55,14 @@ struct StagedShape {
     uint32_t box_bytes;    // the same rounded up to 128: boxes start on 128-byte boundaries
     uint32_t array_bytes;  // all boxes of one array
     uint32_t stage_bytes;  // both arrays, rounded up to 128
+    // results leave through shared memory and TMA tensor stores (store_boxes = 1) or straight from registers
+    int32_t store_boxes;
+    int32_t out_box_cols;
+    int32_t out_boxes_per_tile;
+    uint32_t out_row_bytes;   // out_box_cols elements
+    uint32_t out_box_bytes;   // n rows, rounded up to 128
+    uint32_t out_bytes;       // one output buffer: all boxes of a tile
+    uint32_t out_offset;      // of the first output buffer, from the start of the ring
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -127,18 +139,30 @@ __device__ __forceinline__ void bulk_load_row(uint32_t dst_smem, const void* src
                  : "memory");
 }
 
+// TMA tensor store shared -> global of one box; the unit clips what lies outside the tensor (columns >= d).
+__device__ __forceinline__ void tma_store_box(const CUtensorMap* map, int32_t column, int32_t row, uint32_t src_smem)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(column),
+                 "r"(row), "r"(src_smem)
+                 : "memory");
+}
+
 __device__ __forceinline__ void report_timeout(const FusedParams& prm, int code)
 {
     if (prm.error != nullptr) atomicExch(prm.error, code);
 }
 
-// Eight workers per lane need more registers than 17 warps leave: that shape runs with at most 12 consumer warps.
-constexpr int max_consumer_warps(int wpt) { return wpt >= 8 ? 12 : kMaxConsumerWarps; }
+// Eight workers per lane need more registers than 17 warps leave: that shape runs with at most 12 consumer
+// warps, or 20 in the narrow bf16 form (8-byte slices: half the raw registers, half the shared memory per warp).
+constexpr int max_consumer_warps(int wpt, int vec, int elem)
+{
+    return wpt >= 8 ? ((elem == 2 && vec == 4) ? 20 : 12) : kMaxConsumerWarps;
+}
 
 template <typename T, int VEC, int WPT, int G>
-__global__ void __launch_bounds__((max_consumer_warps(WPT) + 1) * 32)
+__global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) + 1) * 32)
     rps_fused_staged_kernel(const FusedParams prm, const StagedShape shape, const __grid_constant__ CUtensorMap map_x,
-                            const __grid_constant__ CUtensorMap map_b)
+                            const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out)
 {
     constexpr int LPG = 32 / G;
     constexpr int WARP_COLS = LPG * VEC;
@@ -162,6 +186,8 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT) + 1) * 32)
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kAbortFlagOffset);
+    if (threadIdx.x == 0) *abort_flag = 0;
     for (int j = threadIdx.x; j < kMaxWorkers; j += blockDim.x) {
         const bool used = j < n;
         s_up[j] = used ? prm.masks->up[j] : 0;
@@ -247,53 +273,100 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT) + 1) * 32)
     const int col_in_tile = warp * WARP_COLS + sub * VEC;
     const uint32_t lane_off =
         (uint32_t)(col_in_tile / shape.box_cols) * shape.box_bytes + (uint32_t)(col_in_tile % shape.box_cols) * elem;
-    int stage = 0;
+    const uint32_t lane_out_off = shape.store_boxes ? (uint32_t)(col_in_tile / shape.out_box_cols) * shape.out_box_bytes +
+                                                          (uint32_t)(col_in_tile % shape.out_box_cols) * elem
+                                                    : 0u;
+    const bool store_leader = threadIdx.x == 0;  // issues the tensor stores of the whole CTA
+    const uint32_t consumer_threads = (uint32_t)consumer_warps * 32u;
+    if (shape.store_boxes && store_leader) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
+    int stage = 0, out_slot = 0;
     uint32_t phase = 0;
+    // A warp whose wait gave up stops working but keeps meeting the other compute warps at the
+    // per-tile barrier below, so that nobody is left waiting for it.
+    bool dead = false;
     BlockCursor cursor;
     for (int64_t tile = blockIdx.x; tile < shape.tiles; tile += gridDim.x) {
-        if (!mbar_wait(smem_addr(&full[stage]), phase)) {
+        if (!dead && !__all_sync(0xFFFFFFFFu, mbar_wait(smem_addr(&full[stage]), phase))) {
             report_timeout(prm, 2);
-            return;
+            *abort_flag = 1;
+            dead = true;
+            if (!shape.store_boxes) return;  // no barrier to keep: leave
         }
-        const int64_t c = tile * shape.tile_cols + warp * WARP_COLS + sub * VEC;
-        const bool col_live = c < prm.d;
-        const unsigned char* base = ring + (size_t)stage * shape.stage_bytes + lane_off;
+        if (!dead) {
+            const int64_t c = tile * shape.tile_cols + warp * WARP_COLS + sub * VEC;
+            const bool col_live = c < prm.d;
+            const unsigned char* base = ring + (size_t)stage * shape.stage_bytes + lane_off;
 
-        float v[WPT][VEC];
-        {
-            float xv[WPT][VEC], bv[WPT][VEC];
+            float v[WPT][VEC];
+            {
+                float xv[WPT][VEC], bv[WPT][VEC];
 #pragma unroll
-            for (int w = 0; w < WPT; ++w) {
-                // workers past n read the last real row: their values are masked out (their mask bits
-                // are 0) and never stored, so no lane needs a zero-filled stand-in
-                const int row = w_first + w < n ? w_first + w : n - 1;
-                const uint4 raw_x = *reinterpret_cast<const uint4*>(base + (size_t)row * shape.row_bytes);
-                const uint4 raw_b =
-                    *reinterpret_cast<const uint4*>(base + shape.array_bytes + (size_t)row * shape.row_bytes);
-                RowVec<T, VEC>::unpack(raw_x, xv[w]);
-                RowVec<T, VEC>::unpack(raw_b, bv[w]);
+                for (int w = 0; w < WPT; ++w) {
+                    // workers past n read the last real row: their values are masked out (their mask bits
+                    // are 0) and never stored, so no lane needs a zero-filled stand-in
+                    const int row = w_first + w < n ? w_first + w : n - 1;
+                    using Raw = typename RowVec<T, VEC>::Raw;
+                    const Raw raw_x = *reinterpret_cast<const Raw*>(base + (size_t)row * shape.row_bytes);
+                    const Raw raw_b =
+                        *reinterpret_cast<const Raw*>(base + shape.array_bytes + (size_t)row * shape.row_bytes);
+                    RowVec<T, VEC>::unpack(raw_x, xv[w]);
+                    RowVec<T, VEC>::unpack(raw_b, bv[w]);
+                }
+                // this warp has read everything it needs from the stage: hand it back to the producer
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_addr(&empty[stage]));
+                local_sgd<VEC, WPT>(xv, bv, v, c, w_first, prm);
             }
-            // this warp has read everything it needs from the stage: hand it back to the producer
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_addr(&empty[stage]));
-            local_sgd<VEC, WPT>(xv, bv, v, c, w_first, prm);
+            const uint32_t live_bits = average_and_select<VEC, WPT, G>(v, c, col_live, w_first, masks, cursor, prm);
+            if (shape.store_boxes) {
+                // results go to this tile's output buffer in box layout; columns past d are written
+                // here too and clipped by the tensor store
+                unsigned char* out = ring + shape.out_offset + (size_t)out_slot * shape.out_bytes + lane_out_off;
+#pragma unroll
+                for (int w = 0; w < WPT; ++w)
+                    if (w_first + w < n)
+                        *reinterpret_cast<typename RowVec<T, VEC>::Raw*>(out + (size_t)(w_first + w) * shape.out_row_bytes) =
+                            RowVec<T, VEC>::pack(v[w]);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // visible to the TMA unit
+            } else {
+                T* dst = xg + (int64_t)w_first * prm.pitch + c;  // this lane's slice of its first worker's row
+                if (live_bits == (1u << VEC) - 1u) {
+#pragma unroll
+                    for (int w = 0; w < WPT; ++w, dst += prm.pitch)
+                        if (w_first + w < n)
+                            __stcs(reinterpret_cast<typename RowVec<T, VEC>::Raw*>(dst), RowVec<T, VEC>::pack(v[w]));
+                } else if (live_bits != 0) {
+#pragma unroll
+                    for (int w = 0; w < WPT; ++w, dst += prm.pitch)
+                        if (w_first + w < n) store_ragged<T, VEC>(dst, v[w], live_bits);
+                }
+            }
         }
-        const uint32_t live_bits = average_and_select<VEC, WPT, G>(v, c, col_live, w_first, masks, cursor, prm);
-        T* dst = xg + (int64_t)w_first * prm.pitch + c;  // this lane's slice of its first worker's row
-        if (live_bits == (1u << VEC) - 1u) {
-#pragma unroll
-            for (int w = 0; w < WPT; ++w, dst += prm.pitch)
-                if (w_first + w < n) __stcs(reinterpret_cast<uint4*>(dst), RowVec<T, VEC>::pack(v[w]));
-        } else if (live_bits != 0) {
-#pragma unroll
-            for (int w = 0; w < WPT; ++w, dst += prm.pitch)
-                if (w_first + w < n) store_ragged<T, VEC>(dst, v[w], live_bits);
+        if (shape.store_boxes) {
+            // One meeting of the compute warps per tile.  Before it the leader sees the previous tile's
+            // stores finish reading their buffer, so after it (a) the other buffer is free for the next
+            // tile and (b) every warp's results for this tile are in place.
+            if (store_leader && !dead) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            asm volatile("bar.sync 1, %0;" ::"r"(consumer_threads) : "memory");
+            if (*abort_flag) dead = true;
+            if (store_leader && !dead) {
+                const int32_t c0 = (int32_t)(tile * shape.tile_cols);
+                const uint32_t src = smem_addr(ring) + shape.out_offset + (uint32_t)out_slot * shape.out_bytes;
+                for (int k = 0; k < shape.out_boxes_per_tile; ++k) {
+                    const int32_t col = c0 + k * shape.out_box_cols;
+                    if (col < prm.d) tma_store_box(&map_out, col, 0, src + (uint32_t)k * shape.out_box_bytes);
+                }
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+            out_slot ^= 1;
         }
         if (++stage == shape.stages) {
             stage = 0;
             phase ^= 1u;
         }
     }
+    // the stores still read this CTA's shared memory: see them through before the CTA retires
+    if (shape.store_boxes && store_leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 struct Plan {
@@ -302,26 +375,24 @@ struct Plan {
     StagedShape shape;
 };
 
-// Shapes the tile and the ring for one instantiation; false if no ring of >= 2 stages fits.
-bool make_plan(const FusedParams& prm, const FusedTuning& tune, int vec, int wpt, int g, size_t elem,
-               size_t smem_limit, Plan* out)
+// Shapes the tile and the ring for one instantiation with the given number of compute warps; false if
+// a ring of 2 stages (plus the output buffers) does not fit in shared memory.
+bool shape_for(const FusedParams& prm, const FusedTuning& tune, int vec, int g, size_t elem, size_t smem_limit,
+               int warps, Plan* out)
 {
-    // defaults from sweeps on B200: many light warps when a lane holds 2 or 4 workers, fewer heavy
-    // ones when it holds 8 (fp32: 8 warps; bf16, twice the columns per lane: 12)
-    int warps = tune.consumer_warps > 0 ? tune.consumer_warps : (wpt >= 8 ? (elem == 2 ? 12 : 8) : 16);
-    if (warps > max_consumer_warps(wpt)) warps = max_consumer_warps(wpt);
     const int warp_cols = (32 / g) * vec;
     StagedShape& sh = out->shape;
     sh.consumer_warps = warps;
     sh.tile_cols = warps * warp_cols;
+    // the widest box (<= 256 elements) that tiles the tile exactly; warp_cols always does
+    int box_cols = warp_cols;
+    for (int k = 1; k <= warps; ++k)
+        if (warps % k == 0 && k * warp_cols <= kMaxBoxCols) box_cols = k * warp_cols;
     // 2-D boxes when many rows would otherwise mean many small copies, or when asked for
     const int mode = tune.copy_mode != 0 ? tune.copy_mode : (prm.n > 16 ? 2 : 1);
     sh.use_boxes = mode == 2;
     if (sh.use_boxes) {
-        // the widest box (<= 256 elements) that tiles the tile exactly; warp_cols always does
-        sh.box_cols = warp_cols;
-        for (int k = 1; k <= warps; ++k)
-            if (warps % k == 0 && k * warp_cols <= kMaxBoxCols) sh.box_cols = k * warp_cols;
+        sh.box_cols = box_cols;
         sh.boxes_per_tile = sh.tile_cols / sh.box_cols;
         sh.row_bytes = (uint32_t)(sh.box_cols * elem);
     } else {
@@ -335,14 +406,38 @@ bool make_plan(const FusedParams& prm, const FusedTuning& tune, int vec, int wpt
     sh.array_bytes = (uint32_t)sh.boxes_per_tile * sh.box_bytes;
     sh.stage_bytes = (2u * sh.array_bytes + 127u) / 128u * 128u;
     sh.tiles = (prm.d + sh.tile_cols - 1) / sh.tile_cols;
+    // Results: tensor stores from shared memory when a lane group writes less than a 128-byte line per
+    // row and instruction (many workers), else 16-byte stores from registers; or as asked.
+    const int store_mode = tune.store_mode != 0 ? tune.store_mode : ((32 / g) * vec * (int)elem < 128 ? 2 : 1);
+    sh.store_boxes = store_mode == 2;
+    sh.out_box_cols = box_cols;
+    sh.out_boxes_per_tile = sh.tile_cols / sh.out_box_cols;
+    sh.out_row_bytes = (uint32_t)(sh.out_box_cols * elem);
+    sh.out_box_bytes = ((uint32_t)prm.n * sh.out_row_bytes + 127u) / 128u * 128u;
+    sh.out_bytes = (uint32_t)sh.out_boxes_per_tile * sh.out_box_bytes;
+    const size_t out_total = sh.store_boxes ? (size_t)kOutBuffers * sh.out_bytes : 0;
     int stages = tune.stages > 0 ? tune.stages : 2;
     if (stages > kMaxStages) stages = kMaxStages;
-    while (stages > 2 && kSmemHeaderBytes + (size_t)stages * sh.stage_bytes > smem_limit) --stages;
-    if (stages < 2 || kSmemHeaderBytes + (size_t)stages * sh.stage_bytes > smem_limit) return false;
+    while (stages > 2 && kSmemHeaderBytes + (size_t)stages * sh.stage_bytes + out_total > smem_limit) --stages;
+    if (stages < 2 || kSmemHeaderBytes + (size_t)stages * sh.stage_bytes + out_total > smem_limit) return false;
     sh.stages = stages;
+    sh.out_offset = (uint32_t)stages * sh.stage_bytes;
     out->threads = (warps + 1) * 32;
-    out->smem_bytes = kSmemHeaderBytes + (uint32_t)stages * sh.stage_bytes;
+    out->smem_bytes = kSmemHeaderBytes + (uint32_t)stages * sh.stage_bytes + (uint32_t)out_total;
     return true;
+}
+
+// The plan with as many compute warps as asked for (or the default) that still fits in shared memory.
+bool make_plan(const FusedParams& prm, const FusedTuning& tune, int vec, int wpt, int g, size_t elem,
+               size_t smem_limit, Plan* out)
+{
+    // defaults from sweeps on B200: many light warps when a lane holds 2 or 4 workers, fewer heavy
+    // ones when it holds 8 (fp32: 8 warps; bf16, twice the columns per lane: 12)
+    int warps = tune.consumer_warps > 0 ? tune.consumer_warps : (wpt >= 8 ? (elem == 2 ? 12 : 8) : 16);
+    if (warps > max_consumer_warps(wpt, vec, (int)elem)) warps = max_consumer_warps(wpt, vec, (int)elem);
+    for (; warps >= 1; --warps)
+        if (shape_for(prm, tune, vec, g, elem, smem_limit, warps, out)) return true;
+    return false;
 }
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -363,13 +458,14 @@ EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-// Describes one [n][pitch] array to the TMA unit, with boxes of n rows x box_cols columns.
-bool encode_rows(CUtensorMap* map, const void* base, bool bf16, const FusedParams& prm, int box_cols)
+// Describes one [n][pitch] array to the TMA unit, with boxes of n rows x box_cols columns; `cols` columns
+// of every row belong to the tensor (the pitch for loads, d for stores: what lies beyond is not written).
+bool encode_rows(CUtensorMap* map, const void* base, bool bf16, const FusedParams& prm, int box_cols, int64_t cols)
 {
     EncodeTiledFn encode = encode_tiled_fn();
     if (encode == nullptr) return false;
     const size_t elem = bf16 ? 2 : 4;
-    const cuuint64_t dims[2] = {(cuuint64_t)prm.pitch, (cuuint64_t)prm.n};
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)prm.n};
     const cuuint64_t strides[1] = {(cuuint64_t)prm.pitch * elem};  // bytes between rows
     const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)prm.n};
     const cuuint32_t elem_strides[2] = {1, 1};
@@ -398,9 +494,11 @@ cudaError_t launch_staged_as(const FusedParams& prm, const FusedTuning& tune, in
     Plan plan;
     if (!make_plan(prm, tune, VEC, WPT, G, sizeof(T), smem_limit, &plan)) return cudaErrorInvalidConfiguration;
     constexpr bool bf16 = sizeof(T) == 2;
-    alignas(64) CUtensorMap map_x, map_b;
+    alignas(64) CUtensorMap map_x, map_b, map_out;
     const int map_box_cols = plan.shape.use_boxes ? plan.shape.box_cols : 16;  // unused by 1-D copies, but valid
-    if (!encode_rows(&map_x, prm.x, bf16, prm, map_box_cols) || !encode_rows(&map_b, prm.b, bf16, prm, map_box_cols))
+    if (!encode_rows(&map_x, prm.x, bf16, prm, map_box_cols, prm.pitch) ||
+        !encode_rows(&map_b, prm.b, bf16, prm, map_box_cols, prm.pitch) ||
+        !encode_rows(&map_out, prm.x, bf16, prm, plan.shape.out_box_cols, prm.d))
         return cudaErrorInvalidValue;
     if (plan.smem_bytes > smem_granted) {
         if ((err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes)) !=
@@ -421,7 +519,7 @@ cudaError_t launch_staged_as(const FusedParams& prm, const FusedTuning& tune, in
     int64_t grid = (int64_t)sm_count * occ_per_sm;
     if (grid > plan.shape.tiles) grid = plan.shape.tiles;
     if (grid < 1) grid = 1;
-    kernel<<<(unsigned)grid, plan.threads, plan.smem_bytes, stream>>>(prm, plan.shape, map_x, map_b);
+    kernel<<<(unsigned)grid, plan.threads, plan.smem_bytes, stream>>>(prm, plan.shape, map_x, map_b, map_out);
     return cudaGetLastError();
 }
 
@@ -462,6 +560,14 @@ cudaError_t launch_fused_staged(const FusedParams& prm, const FusedTuning& tune,
 {
     // TMA coordinates are 32-bit: rows of 2^31 elements or more go through the direct kernel
     if (prm.pitch >= ((int64_t)1 << 31)) return launch_fused_direct(prm, tune, bf16, sm_count, stream);
+    if (bf16 && tune.slice_bytes == 8) {
+        // narrow bf16 slices exist for 8 workers per lane only
+        const int n = prm.n;
+        if (n <= 8) return launch_staged_as<__nv_bfloat16, 4, 8, 1>(prm, tune, sm_count, stream);
+        if (n <= 16) return launch_staged_as<__nv_bfloat16, 4, 8, 2>(prm, tune, sm_count, stream);
+        if (n <= 32) return launch_staged_as<__nv_bfloat16, 4, 8, 4>(prm, tune, sm_count, stream);
+        return launch_staged_as<__nv_bfloat16, 4, 8, 8>(prm, tune, sm_count, stream);
+    }
     if (bf16) return launch_staged_for_n<__nv_bfloat16, 8>(prm, tune, sm_count, stream);
     return launch_staged_for_n<float, 4>(prm, tune, sm_count, stream);
 }

@@ -283,21 +283,33 @@ def test_edge_shapes(rps_mod, oracle, n, d, dtype):
         want = wl.make_initial(w)
         oracle.run(want, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps,
                    self_delivery=sd, assign=assign)
-        for kernel, copy_mode in ((1, 0), (2, 1), (2, 2)):
-            r = make(rps_mod, w, self_delivery=sd, assign=assign, kernel=kernel, copy_mode=copy_mode)
+        for kernel, copy_mode, slice_bytes, store_mode in ((1, 0, 0, 0), (2, 1, 0, 1), (2, 2, 0, 2), (2, 0, 8, 2),
+                                                            (2, 1, 0, 2)):
+            if slice_bytes == 8 and dtype != "bf16":
+                continue
+            r = make(rps_mod, w, self_delivery=sd, assign=assign, kernel=kernel, copy_mode=copy_mode,
+                     slice_bytes=slice_bytes, store_mode=store_mode)
             r.set_targets(b)
             r.x_dev[:, d:] = 3.0         # sentinel in the padding between d and the row pitch
             r.step_n(w.steps)
             got = r.read()
             assert_close(w, got, want, BF16_TOL if dtype == "bf16" else 3 * STEP_TOL)
-            assert (r.x_dev[:, d:].float() == 3.0).all()      # never written
+            # padding is left alone, except that the columns sharing a 16-byte unit with the last
+            # real column may be zeroed
+            unit = 4 if dtype == "f32" else 8
+            edge = -(-d // unit) * unit
+            assert (r.x_dev[:, edge:].float() == 3.0).all()
+            shared_unit = r.x_dev[:, d:edge].float()
+            assert ((shared_unit == 3.0) | (shared_unit == 0.0)).all()
             r.close()
 
 
 # every shape of the fused kernel computes the same step:
-# (kernel, workers_per_lane, stages, consumer_warps, copy_mode)
-VARIANTS = [(1, 0, 0, 0, 0), (1, 4, 0, 0, 0), (2, 0, 0, 0, 0), (2, 2, 0, 0, 1), (2, 4, 2, 4, 2), (2, 8, 4, 3, 1),
-            (2, 4, 5, 16, 2), (2, 2, 8, 1, 2), (2, 8, 2, 8, 2), (2, 4, 3, 5, 1), (2, 8, 2, 12, 1)]
+# (kernel, workers_per_lane, stages, consumer_warps, copy_mode, slice_bytes, store_mode)
+VARIANTS = [(1, 0, 0, 0, 0, 0, 0), (1, 4, 0, 0, 0, 0, 0), (2, 0, 0, 0, 0, 0, 0), (2, 2, 0, 0, 1, 0, 1),
+            (2, 4, 2, 4, 2, 0, 2), (2, 8, 4, 3, 1, 0, 2), (2, 4, 5, 16, 2, 0, 1), (2, 2, 8, 1, 2, 0, 2),
+            (2, 8, 2, 8, 2, 0, 1), (2, 4, 3, 5, 1, 0, 2), (2, 8, 2, 12, 1, 0, 1), (2, 8, 2, 20, 2, 8, 2),
+            (2, 8, 3, 7, 1, 8, 1), (2, 4, 2, 16, 0, 0, 2), (2, 8, 2, 8, 0, 0, 2)]
 
 
 @pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
@@ -306,9 +318,9 @@ def test_kernel_variants(rps_mod, oracle, name):
     b = wl.make_targets(w)
     want = wl.make_initial(w)
     oracle.run(want, b, dtype=w.dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps)
-    for kernel, wpt, stages, warps, copy_mode in VARIANTS:
+    for kernel, wpt, stages, warps, copy_mode, slice_bytes, store_mode in VARIANTS:
         r = make(rps_mod, w, kernel=kernel, workers_per_lane=wpt, stages=stages, consumer_warps=warps,
-                 copy_mode=copy_mode)
+                 copy_mode=copy_mode, slice_bytes=slice_bytes, store_mode=store_mode)
         r.set_targets(b)
         r.step_n(w.steps)
         got = r.read()
