@@ -88,7 +88,8 @@ typedef struct rps_options {
     int32_t slice_bytes;      /* kernel 2, bf16 replicas: bytes of a row handled by one lane,
                                  16 or 8 (8 = more, lighter warps per tile)                  */
     int32_t store_mode;       /* kernel 2 writes results 1: from registers, 16 bytes per lane,
-                                 2: through shared memory with TMA tensor stores             */
+                                 2: through an output tile in shared memory with TMA tensor
+                                 stores, 3: in place in the stage, stored by a store warp    */
 } rps_options;
 
 /*

@@ -321,7 +321,7 @@ int rps_configure(rps_handle* h, const rps_options* opt)
         return fail(h, RPS_EINVAL, "consumer_warps must be 0 (auto) or 1..24");
     if (opt->slice_bytes != 0 && opt->slice_bytes != 8 && opt->slice_bytes != 16)
         return fail(h, RPS_EINVAL, "slice_bytes must be 0 (auto), 8 or 16");
-    if (opt->store_mode < 0 || opt->store_mode > 2) return fail(h, RPS_EINVAL, "store_mode must be 0 (auto), 1 or 2");
+    if (opt->store_mode < 0 || opt->store_mode > 3) return fail(h, RPS_EINVAL, "store_mode must be 0 (auto) or 1..3");
     if (opt->copy_mode < 0 || opt->copy_mode > 2) return fail(h, RPS_EINVAL, "copy_mode must be 0 (auto), 1 or 2");
     h->opt = *opt;
     h->sigma = (float)opt->sigma;

@@ -28,7 +28,7 @@ struct FusedTuning {
     int32_t consumer_warps;    // compute warps per CTA of the staged kernel
     int32_t copy_mode;         // staged kernel: 1 one bulk copy per row, 2 two-dimensional TMA boxes
     int32_t slice_bytes;       // staged kernel, bf16: bytes of a row one lane handles, 16 or 8
-    int32_t store_mode;        // staged kernel: 1 stores from registers, 2 TMA tensor stores from shared memory
+    int32_t store_mode;        // staged kernel: 1 stores from registers, 2 TMA stores from an output tile, 3 TMA stores in place
 };
 
 struct FusedParams {

@@ -55,8 +55,10 @@ struct StagedShape {
     uint32_t box_bytes;    // the same rounded up to 128: boxes start on 128-byte boundaries
     uint32_t array_bytes;  // all boxes of one array
     uint32_t stage_bytes;  // both arrays, rounded up to 128
-    // results leave through shared memory and TMA tensor stores (store_boxes = 1) or straight from registers
-    int32_t store_boxes;
+    // how results leave: 1 straight from registers; 2 through a double-buffered output tile in shared
+    // memory and TMA tensor stores issued by a compute thread; 3 written back in place over the x half of
+    // the stage and stored from there by a dedicated store warp, which then frees the stage
+    int32_t store_mode;
     int32_t out_box_cols;
     int32_t out_boxes_per_tile;
     uint32_t out_row_bytes;   // out_box_cols elements
@@ -160,7 +162,7 @@ constexpr int max_consumer_warps(int wpt, int vec, int elem)
 }
 
 template <typename T, int VEC, int WPT, int G>
-__global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) + 1) * 32)
+__global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) + 2) * 32)
     rps_fused_staged_kernel(const FusedParams prm, const StagedShape shape, const __grid_constant__ CUtensorMap map_x,
                             const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out)
 {
@@ -182,7 +184,8 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
     if (threadIdx.x == 0) {
         for (int s = 0; s < shape.stages; ++s) {
             mbar_init(smem_addr(&full[s]), 1);
-            mbar_init(smem_addr(&empty[s]), (uint32_t)consumer_warps);
+            // a stage is handed back by every compute warp, or (in-place results) by the store warp alone
+            mbar_init(smem_addr(&empty[s]), shape.store_mode == 3 ? 1u : (uint32_t)consumer_warps);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -264,6 +267,33 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
         return;
     }
 
+    const uint32_t consumer_threads = (uint32_t)consumer_warps * 32u;
+    if (warp == consumer_warps + 1) {
+        // ---------------- store warp (in-place results only): when every compute warp has put its results
+        // of a tile back into the stage, send the x half of the stage to global memory and free the stage
+        if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
+        int stage = 0;
+        bool dead = false;
+        for (int64_t tile = blockIdx.x; tile < shape.tiles; tile += gridDim.x) {
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + stage), "r"(consumer_threads + 32u) : "memory");
+            if (*abort_flag) dead = true;
+            if (lane == 0 && !dead) {
+                const int32_t c0 = (int32_t)(tile * shape.tile_cols);
+                const uint32_t src = smem_addr(ring) + (uint32_t)stage * shape.stage_bytes;
+                for (int k = 0; k < shape.boxes_per_tile; ++k) {
+                    const int32_t col = c0 + k * shape.box_cols;
+                    if (col < prm.d) tma_store_box(&map_out, col, 0, src + (uint32_t)k * shape.box_bytes);
+                }
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // the unit has read the stage
+                mbar_arrive(smem_addr(&empty[stage]));
+            }
+            if (++stage == shape.stages) stage = 0;
+        }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        return;
+    }
+
     // ---------------- consumers
     T* __restrict__ xg = static_cast<T*>(prm.x);
     const MaskView masks{s_up, s_down, s_inv};
@@ -273,12 +303,12 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
     const int col_in_tile = warp * WARP_COLS + sub * VEC;
     const uint32_t lane_off =
         (uint32_t)(col_in_tile / shape.box_cols) * shape.box_bytes + (uint32_t)(col_in_tile % shape.box_cols) * elem;
-    const uint32_t lane_out_off = shape.store_boxes ? (uint32_t)(col_in_tile / shape.out_box_cols) * shape.out_box_bytes +
-                                                          (uint32_t)(col_in_tile % shape.out_box_cols) * elem
-                                                    : 0u;
-    const bool store_leader = threadIdx.x == 0;  // issues the tensor stores of the whole CTA
-    const uint32_t consumer_threads = (uint32_t)consumer_warps * 32u;
-    if (shape.store_boxes && store_leader) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
+    const bool out_tiles = shape.store_mode == 2, in_place = shape.store_mode == 3;
+    const uint32_t lane_out_off = out_tiles ? (uint32_t)(col_in_tile / shape.out_box_cols) * shape.out_box_bytes +
+                                                  (uint32_t)(col_in_tile % shape.out_box_cols) * elem
+                                            : 0u;
+    const bool store_leader = threadIdx.x == 0;  // issues the tensor stores of mode 2
+    if (out_tiles && store_leader) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
     int stage = 0, out_slot = 0;
     uint32_t phase = 0;
     // A warp whose wait gave up stops working but keeps meeting the other compute warps at the
@@ -290,12 +320,12 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
             report_timeout(prm, 2);
             *abort_flag = 1;
             dead = true;
-            if (!shape.store_boxes) return;  // no barrier to keep: leave
+            if (shape.store_mode == 1) return;  // no barrier to keep: leave
         }
         if (!dead) {
             const int64_t c = tile * shape.tile_cols + warp * WARP_COLS + sub * VEC;
             const bool col_live = c < prm.d;
-            const unsigned char* base = ring + (size_t)stage * shape.stage_bytes + lane_off;
+            unsigned char* base = ring + (size_t)stage * shape.stage_bytes + lane_off;
 
             float v[WPT][VEC];
             {
@@ -312,13 +342,24 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
                     RowVec<T, VEC>::unpack(raw_x, xv[w]);
                     RowVec<T, VEC>::unpack(raw_b, bv[w]);
                 }
-                // this warp has read everything it needs from the stage: hand it back to the producer
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_addr(&empty[stage]));
+                if (!in_place) {
+                    // this warp has read everything it needs from the stage: hand it back to the producer
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_addr(&empty[stage]));
+                }
                 local_sgd<VEC, WPT>(xv, bv, v, c, w_first, prm);
             }
             const uint32_t live_bits = average_and_select<VEC, WPT, G>(v, c, col_live, w_first, masks, cursor, prm);
-            if (shape.store_boxes) {
+            if (in_place) {
+                // every lane overwrites exactly the slices of x it read; columns past d are clipped by
+                // the tensor store
+#pragma unroll
+                for (int w = 0; w < WPT; ++w)
+                    if (w_first + w < n)
+                        *reinterpret_cast<typename RowVec<T, VEC>::Raw*>(base + (size_t)(w_first + w) * shape.row_bytes) =
+                            RowVec<T, VEC>::pack(v[w]);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // visible to the TMA unit
+            } else if (out_tiles) {
                 // results go to this tile's output buffer in box layout; columns past d are written
                 // here too and clipped by the tensor store
                 unsigned char* out = ring + shape.out_offset + (size_t)out_slot * shape.out_bytes + lane_out_off;
@@ -342,7 +383,10 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
                 }
             }
         }
-        if (shape.store_boxes) {
+        if (in_place) {
+            // tell the store warp (dead warps too, so that it never waits for nothing)
+            asm volatile("bar.arrive %0, %1;" ::"r"(1 + stage), "r"(consumer_threads + 32u) : "memory");
+        } else if (out_tiles) {
             // One meeting of the compute warps per tile.  Before it the leader sees the previous tile's
             // stores finish reading their buffer, so after it (a) the other buffer is free for the next
             // tile and (b) every warp's results for this tile are in place.
@@ -366,7 +410,7 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
         }
     }
     // the stores still read this CTA's shared memory: see them through before the CTA retires
-    if (shape.store_boxes && store_leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (out_tiles && store_leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 struct Plan {
@@ -378,7 +422,7 @@ struct Plan {
 // Shapes the tile and the ring for one instantiation with the given number of compute warps; false if
 // a ring of 2 stages (plus the output buffers) does not fit in shared memory.
 bool shape_for(const FusedParams& prm, const FusedTuning& tune, int vec, int g, size_t elem, size_t smem_limit,
-               int warps, Plan* out)
+               int warps, int default_store_mode, Plan* out)
 {
     const int warp_cols = (32 / g) * vec;
     StagedShape& sh = out->shape;
@@ -389,7 +433,11 @@ bool shape_for(const FusedParams& prm, const FusedTuning& tune, int vec, int g, 
     for (int k = 1; k <= warps; ++k)
         if (warps % k == 0 && k * warp_cols <= kMaxBoxCols) box_cols = k * warp_cols;
     // 2-D boxes when many rows would otherwise mean many small copies, or when asked for
-    const int mode = tune.copy_mode != 0 ? tune.copy_mode : (prm.n > 16 ? 2 : 1);
+    // Results: 16-byte stores from registers, or TMA tensor stores from shared memory: from a separate
+    // double-buffered output tile (2), or in place from the stage by a store warp (3) where shared memory
+    // is too scarce for output tiles (8 workers per lane).  In place needs the box layout.
+    const int store_mode = tune.store_mode != 0 ? tune.store_mode : default_store_mode;
+    const int mode = store_mode == 3 ? 2 : (tune.copy_mode != 0 ? tune.copy_mode : (prm.n > 16 ? 2 : 1));
     sh.use_boxes = mode == 2;
     if (sh.use_boxes) {
         sh.box_cols = box_cols;
@@ -406,23 +454,20 @@ bool shape_for(const FusedParams& prm, const FusedTuning& tune, int vec, int g, 
     sh.array_bytes = (uint32_t)sh.boxes_per_tile * sh.box_bytes;
     sh.stage_bytes = (2u * sh.array_bytes + 127u) / 128u * 128u;
     sh.tiles = (prm.d + sh.tile_cols - 1) / sh.tile_cols;
-    // Results: tensor stores from shared memory when a lane group writes less than a 128-byte line per
-    // row and instruction (many workers), else 16-byte stores from registers; or as asked.
-    const int store_mode = tune.store_mode != 0 ? tune.store_mode : ((32 / g) * vec * (int)elem < 128 ? 2 : 1);
-    sh.store_boxes = store_mode == 2;
+    sh.store_mode = store_mode;
     sh.out_box_cols = box_cols;
     sh.out_boxes_per_tile = sh.tile_cols / sh.out_box_cols;
     sh.out_row_bytes = (uint32_t)(sh.out_box_cols * elem);
     sh.out_box_bytes = ((uint32_t)prm.n * sh.out_row_bytes + 127u) / 128u * 128u;
     sh.out_bytes = (uint32_t)sh.out_boxes_per_tile * sh.out_box_bytes;
-    const size_t out_total = sh.store_boxes ? (size_t)kOutBuffers * sh.out_bytes : 0;
+    const size_t out_total = store_mode == 2 ? (size_t)kOutBuffers * sh.out_bytes : 0;
     int stages = tune.stages > 0 ? tune.stages : 2;
     if (stages > kMaxStages) stages = kMaxStages;
     while (stages > 2 && kSmemHeaderBytes + (size_t)stages * sh.stage_bytes + out_total > smem_limit) --stages;
     if (stages < 2 || kSmemHeaderBytes + (size_t)stages * sh.stage_bytes + out_total > smem_limit) return false;
     sh.stages = stages;
     sh.out_offset = (uint32_t)stages * sh.stage_bytes;
-    out->threads = (warps + 1) * 32;
+    out->threads = (warps + (store_mode == 3 ? 2 : 1)) * 32;
     out->smem_bytes = kSmemHeaderBytes + (uint32_t)stages * sh.stage_bytes + (uint32_t)out_total;
     return true;
 }
@@ -431,12 +476,15 @@ bool shape_for(const FusedParams& prm, const FusedTuning& tune, int vec, int g, 
 bool make_plan(const FusedParams& prm, const FusedTuning& tune, int vec, int wpt, int g, size_t elem,
                size_t smem_limit, Plan* out)
 {
-    // defaults from sweeps on B200: many light warps when a lane holds 2 or 4 workers, fewer heavy
-    // ones when it holds 8 (fp32: 8 warps; bf16, twice the columns per lane: 12)
-    int warps = tune.consumer_warps > 0 ? tune.consumer_warps : (wpt >= 8 ? (elem == 2 ? 12 : 8) : 16);
+    // Defaults from sweeps on B200.  A lane holding 2 or 4 workers: 16 light compute warps and a separate
+    // output tile (the ring is small).  A lane holding 8 workers: 12 heavier warps, and no room for output
+    // tiles: fp32 results go back in place through the store warp, bf16 results (half the bytes per
+    // replica-param, bound by instruction issue rather than by HBM) leave straight from registers.
+    int warps = tune.consumer_warps > 0 ? tune.consumer_warps : (wpt >= 8 ? 12 : 16);
     if (warps > max_consumer_warps(wpt, vec, (int)elem)) warps = max_consumer_warps(wpt, vec, (int)elem);
+    const int default_store_mode = wpt >= 8 ? (elem == 2 ? 1 : 3) : 2;
     for (; warps >= 1; --warps)
-        if (shape_for(prm, tune, vec, g, elem, smem_limit, warps, out)) return true;
+        if (shape_for(prm, tune, vec, g, elem, smem_limit, warps, default_store_mode, out)) return true;
     return false;
 }
 

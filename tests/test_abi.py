@@ -64,7 +64,7 @@ def test_options_pitch_and_state_errors(lib):
         assert lib.rps_pitch(h) == 11_174_080                      # rounded up to 64 bf16, plus one skew line
         for field, value in (("dtype", 7), ("assign", 2), ("self_delivery", 3), ("mask_window", 0),
                              ("mask_window", 257), ("sigma", -1.0), ("kernel", 3), ("workers_per_lane", 3), ("stages", 1),
-                             ("stages", 9), ("consumer_warps", 25), ("slice_bytes", 4), ("store_mode", 3), ("row_skew_lines", -2), ("copy_mode", 3)):
+                             ("stages", 9), ("consumer_warps", 25), ("slice_bytes", 4), ("store_mode", 4), ("row_skew_lines", -2), ("copy_mode", 3)):
             bad = rps_options()
             lib.rps_default_options(ctypes.byref(bad))
             setattr(bad, field, value)

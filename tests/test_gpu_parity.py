@@ -284,7 +284,7 @@ def test_edge_shapes(rps_mod, oracle, n, d, dtype):
         oracle.run(want, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps,
                    self_delivery=sd, assign=assign)
         for kernel, copy_mode, slice_bytes, store_mode in ((1, 0, 0, 0), (2, 1, 0, 1), (2, 2, 0, 2), (2, 0, 8, 2),
-                                                            (2, 1, 0, 2)):
+                                                            (2, 1, 0, 2), (2, 0, 0, 3), (2, 0, 8, 3)):
             if slice_bytes == 8 and dtype != "bf16":
                 continue
             r = make(rps_mod, w, self_delivery=sd, assign=assign, kernel=kernel, copy_mode=copy_mode,
@@ -309,7 +309,8 @@ def test_edge_shapes(rps_mod, oracle, n, d, dtype):
 VARIANTS = [(1, 0, 0, 0, 0, 0, 0), (1, 4, 0, 0, 0, 0, 0), (2, 0, 0, 0, 0, 0, 0), (2, 2, 0, 0, 1, 0, 1),
             (2, 4, 2, 4, 2, 0, 2), (2, 8, 4, 3, 1, 0, 2), (2, 4, 5, 16, 2, 0, 1), (2, 2, 8, 1, 2, 0, 2),
             (2, 8, 2, 8, 2, 0, 1), (2, 4, 3, 5, 1, 0, 2), (2, 8, 2, 12, 1, 0, 1), (2, 8, 2, 20, 2, 8, 2),
-            (2, 8, 3, 7, 1, 8, 1), (2, 4, 2, 16, 0, 0, 2), (2, 8, 2, 8, 0, 0, 2)]
+            (2, 8, 3, 7, 1, 8, 1), (2, 4, 2, 16, 0, 0, 2), (2, 8, 2, 8, 0, 0, 2), (2, 8, 2, 12, 0, 0, 3),
+            (2, 4, 2, 16, 0, 0, 3), (2, 8, 3, 5, 0, 8, 3), (2, 2, 2, 3, 1, 0, 3)]
 
 
 @pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
