@@ -34,9 +34,9 @@ FALLBACK_HBM_GBS = 6650.0
 # the ncu capture summarised under profiles/, keyed by workload; valid only for the kernel
 # sources whose digest is recorded with it.
 NCU_TRAFFIC = {
-    "kernel_digest": "d9cb96b9944b0c40",
-    "bytes_per_launch": {"cfg2": 1022099456, "cfg4": 1492908032,
-                         "cfg5": 6073307136},  # cfg5: the d = 2,097,152 capture x 8 (traffic is proportional to d)
+    "kernel_digest": "ab25329539aedc19",
+    # cfg3 and cfg5 come from captures at d/4 and d/8, scaled (traffic is proportional to d)
+    "bytes_per_launch": {"cfg2": 1023694080, "cfg3": 4727221248, "cfg4": 1488895128, "cfg5": 6058887168},
 }
 
 
