@@ -90,6 +90,12 @@ typedef struct rps_options {
     int32_t store_mode;       /* kernel 2 writes results 1: from registers, 16 bytes per lane,
                                  2: through an output tile in shared memory with TMA tensor
                                  stores, 3: in place in the stage, stored by a store warp    */
+    int32_t wait_limit_ms;    /* kernel 2: every wait of a warp on data or on a free stage gives
+                                 up after this many milliseconds (0 = 2000); the next
+                                 synchronising call then returns RPS_ECUDA                   */
+    int32_t withhold_copies;  /* kernel 2, test aid for that time-out path: 1 = the producer warp
+                                 issues no copies, so the compute warps' waits run out, x is
+                                 left unchanged and the error is reported; 0 otherwise       */
 } rps_options;
 
 /*

@@ -76,7 +76,8 @@ struct rps_handle {
     int32_t* error_word() const { return reinterpret_cast<int32_t*>(scratch + kErrorOffset); }
     rps::FusedTuning tuning() const
     {
-        return rps::FusedTuning{opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps, opt.copy_mode, opt.slice_bytes, opt.store_mode};
+        return rps::FusedTuning{opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps, opt.copy_mode, opt.slice_bytes, opt.store_mode,
+                                 opt.wait_limit_ms, opt.withhold_copies};
     }
     rps::StepMasks* window() const { return reinterpret_cast<rps::StepMasks*>(scratch + kDiagBytes); }
     rps::StepMasks* probe() const { return window() + opt.mask_window; }
@@ -248,6 +249,8 @@ int rps_default_options(rps_options* opt)
     opt->copy_mode = 0;
     opt->slice_bytes = 0;
     opt->store_mode = 0;
+    opt->wait_limit_ms = 0;
+    opt->withhold_copies = 0;
     return RPS_OK;
 }
 
@@ -321,6 +324,10 @@ int rps_configure(rps_handle* h, const rps_options* opt)
         return fail(h, RPS_EINVAL, "consumer_warps must be 0 (auto) or 1..24");
     if (opt->slice_bytes != 0 && opt->slice_bytes != 8 && opt->slice_bytes != 16)
         return fail(h, RPS_EINVAL, "slice_bytes must be 0 (auto), 8 or 16");
+    if (opt->wait_limit_ms < 0 || opt->wait_limit_ms > 10000)
+        return fail(h, RPS_EINVAL, "wait_limit_ms must be 0 (default) or 1..10000");
+    if (opt->withhold_copies != 0 && opt->withhold_copies != 1)
+        return fail(h, RPS_EINVAL, "withhold_copies must be 0 or 1");
     if (opt->store_mode < 0 || opt->store_mode > 3) return fail(h, RPS_EINVAL, "store_mode must be 0 (auto) or 1..3");
     if (opt->copy_mode < 0 || opt->copy_mode > 2) return fail(h, RPS_EINVAL, "copy_mode must be 0 (auto), 1 or 2");
     h->opt = *opt;

@@ -29,6 +29,8 @@ struct FusedTuning {
     int32_t copy_mode;         // staged kernel: 1 one bulk copy per row, 2 two-dimensional TMA boxes
     int32_t slice_bytes;       // staged kernel, bf16: bytes of a row one lane handles, 16 or 8
     int32_t store_mode;        // staged kernel: 1 stores from registers, 2 TMA stores from an output tile, 3 TMA stores in place
+    int32_t wait_limit_ms;     // staged kernel: bound of every mbarrier wait (0 = 2000 ms)
+    int32_t withhold_copies;   // staged kernel, test aid: issue no copies so that the bounded waits run out
 };
 
 struct FusedParams {

@@ -21,8 +21,8 @@
 // workers), through a double-buffered tile in shared memory and TMA tensor
 // stores of whole boxes (clipped at column d by the tensor map).
 //
-// Every wait on an mbarrier is bounded (2 s of %globaltimer); a wait that gives
-// up records a code in *prm.error and the warp leaves the kernel.
+// Every wait on an mbarrier is bounded (2 s of %globaltimer by default); a wait
+// that gives up records a code in *prm.error and the warp stops working.
 #include <cuda.h>
 
 #include "rps_kernels.h"
@@ -39,7 +39,7 @@ constexpr int kMaxBoxCols = 256;  // a TMA box is at most 256 elements wide
 constexpr uint32_t kSmemHeaderBytes = 128 + 2 * kMaxWorkers * 8 + kMaxWorkers * 4 + 128;  // barriers, mask copy, flags
 constexpr uint32_t kAbortFlagOffset = kSmemHeaderBytes - 128;
 constexpr int kOutBuffers = 2;
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
+constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;
 static_assert(kSmemHeaderBytes % 128 == 0, "tile data must start on a 128-byte boundary");
 
 struct StagedShape {
@@ -65,6 +65,8 @@ struct StagedShape {
     uint32_t out_box_bytes;   // n rows, rounded up to 128
     uint32_t out_bytes;       // one output buffer: all boxes of a tile
     uint32_t out_offset;      // of the first output buffer, from the start of the ring
+    uint64_t wait_limit_ns;   // how long a wait on an mbarrier may last before the warp gives up
+    int32_t withhold_copies;  // test aid: the producer issues nothing, so that the waits run out
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -107,15 +109,15 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     return t;
 }
 
-// Waits for the phase with the given parity to complete; gives up after kWaitLimitNs.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// Waits for the phase with the given parity to complete; gives up after limit_ns.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t start = global_timer_ns();
 #pragma unroll 1
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - start > kWaitLimitNs) return false;
+        if (global_timer_ns() - start > limit_ns) return false;
     }
 }
 
@@ -203,6 +205,7 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
     constexpr uint32_t elem = (uint32_t)sizeof(T);
     if (warp == consumer_warps) {
         // ---------------- producer warp: keeps the ring full
+        if (shape.withhold_copies) return;
         const unsigned char* x_bytes = static_cast<const unsigned char*>(prm.x);
         const unsigned char* b_bytes = static_cast<const unsigned char*>(prm.b);
         if (shape.use_boxes && lane == 0) {
@@ -215,7 +218,7 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < shape.tiles; tile += gridDim.x) {
             // a fresh barrier counts as "previous phase complete", so the first lap does not wait
-            if (!mbar_wait(smem_addr(&empty[stage]), phase ^ 1u)) {
+            if (!mbar_wait(smem_addr(&empty[stage]), phase ^ 1u, shape.wait_limit_ns)) {
                 ok = false;
                 break;
             }
@@ -261,7 +264,7 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
                     stage = shape.stages - 1;
                     phase ^= 1u;
                 }
-                if (!mbar_wait(smem_addr(&full[stage]), phase)) break;
+                if (!mbar_wait(smem_addr(&full[stage]), phase, shape.wait_limit_ns)) break;
             }
         }
         return;
@@ -316,7 +319,7 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
     bool dead = false;
     BlockCursor cursor;
     for (int64_t tile = blockIdx.x; tile < shape.tiles; tile += gridDim.x) {
-        if (!dead && !__all_sync(0xFFFFFFFFu, mbar_wait(smem_addr(&full[stage]), phase))) {
+        if (!dead && !__all_sync(0xFFFFFFFFu, mbar_wait(smem_addr(&full[stage]), phase, shape.wait_limit_ns))) {
             report_timeout(prm, 2);
             *abort_flag = 1;
             dead = true;
@@ -384,8 +387,13 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
             }
         }
         if (in_place) {
-            // tell the store warp (dead warps too, so that it never waits for nothing)
-            asm volatile("bar.arrive %0, %1;" ::"r"(1 + stage), "r"(consumer_threads + 32u) : "memory");
+            // Tell the store warp.  A warp that gave up still takes part, and waits for the meeting to
+            // complete: it no longer waits for data, and must not run ahead of the store warp and be counted
+            // twice on one barrier.
+            if (dead)
+                asm volatile("bar.sync %0, %1;" ::"r"(1 + stage), "r"(consumer_threads + 32u) : "memory");
+            else
+                asm volatile("bar.arrive %0, %1;" ::"r"(1 + stage), "r"(consumer_threads + 32u) : "memory");
         } else if (out_tiles) {
             // One meeting of the compute warps per tile.  Before it the leader sees the previous tile's
             // stores finish reading their buffer, so after it (a) the other buffer is free for the next
@@ -466,6 +474,8 @@ bool shape_for(const FusedParams& prm, const FusedTuning& tune, int vec, int g, 
     while (stages > 2 && kSmemHeaderBytes + (size_t)stages * sh.stage_bytes + out_total > smem_limit) --stages;
     if (stages < 2 || kSmemHeaderBytes + (size_t)stages * sh.stage_bytes + out_total > smem_limit) return false;
     sh.stages = stages;
+    sh.wait_limit_ns = tune.wait_limit_ms > 0 ? (uint64_t)tune.wait_limit_ms * 1000000ull : kDefaultWaitLimitNs;
+    sh.withhold_copies = tune.withhold_copies;
     sh.out_offset = (uint32_t)stages * sh.stage_bytes;
     out->threads = (warps + (store_mode == 3 ? 2 : 1)) * 32;
     out->smem_bytes = kSmemHeaderBytes + (uint32_t)stages * sh.stage_bytes + (uint32_t)out_total;

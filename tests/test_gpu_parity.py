@@ -413,3 +413,32 @@ def test_full_size_sampled_columns(rps_mod, oracle, name):
         assert all((a == o).all() for a, o in zip(r.read_masks(t), oracle.masks(w.n, w.p, w.seed, t)))
     r.close()
     torch.cuda.empty_cache()
+
+
+# ------------------------------------------------------------------ bounded waits
+
+@pytest.mark.parametrize("store_mode", [1, 2, 3])
+def test_a_wait_that_runs_out_is_reported_and_harmless(rps_mod, store_mode):
+    """The staged kernel's waits are bounded.  With the copies withheld nothing ever lands, every compute
+    warp gives up after the (shortened) limit, the kernel ends by itself, the replicas are untouched, the
+    next read reports the error, and the device is as usable as before."""
+    w = TWINS["cfg2"].scaled(d=40_002, steps=1)
+    b = wl.make_targets(w)
+    x0 = np.random.default_rng(1).standard_normal(b.shape).astype(np.float32)
+    r = make(rps_mod, w, kernel=2, store_mode=store_mode, wait_limit_ms=20, withhold_copies=True)
+    r.set_targets(b)
+    r.write(x0)
+    r.step()
+    with pytest.raises(rps_mod.RPSError) as err:
+        r.read()
+    assert err.value.code == rps_mod.RPS_ECUDA and "gave up" in str(err.value)
+    torch.cuda.synchronize()
+    assert (r.x_dev[:, :w.d].cpu().numpy() == x0).all()
+    r.close()
+    # the same handle settings without the test aid work, on the same device, right after
+    r = make(rps_mod, w, kernel=2, store_mode=store_mode, wait_limit_ms=20)
+    r.set_targets(b)
+    r.write(x0)
+    r.step()
+    assert np.isfinite(r.read()).all()
+    r.close()

@@ -7,6 +7,8 @@ C ABI on buffers it owns and checks that two consecutive steps give the same
 replicas as the ordinary handle-based path.  It lives in its own file, collected
 last, so a failure here cannot hide the results of the other tests.
 """
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -41,13 +43,16 @@ def test_static_step_matches_the_bound_step_twice_in_a_row(name, d):
     tdtype = torch.float32 if w.dtype == "f32" else torch.bfloat16
     x_dev = torch.zeros((w.n, pitch), dtype=tdtype, device="cuda")
     b_dev = ref.b_dev.clone()
+    # tensors of earlier tests may still be waiting for the garbage collector: let them go first, so that
+    # the only thing that could change the allocator's count below is the call under test
+    gc.collect()
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
     for t in range(2):
         binding.step_static(x_dev, b_dev, n=w.n, d=w.d, dtype=w.dtype, p=w.p, gamma=w.gamma, sigma=w.sigma,
                             seed=w.seed, t=t)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == before
+        assert torch.cuda.memory_allocated() <= before        # nothing was allocated on our behalf
         got = x_dev[:, :w.d].contiguous()
         got = (got.view(torch.int16) if w.dtype == "bf16" else got).cpu().numpy()
         if w.dtype == "bf16":
