@@ -359,3 +359,72 @@ int rps_oracle_diag(int n, int64_t d, int dtype, const void* x, const void* b, d
     *consensus = cons;
     return 0;
 }
+
+/*
+ * The comparison method of Section 5 ("Comparison with Gradient Averaging"): the same unreliable
+ * Reduce-Scatter / All-Gather, but what travels is the stochastic gradient instead of the model.
+ *
+ *   g^(i)      = grad F_i(x^(i); xi)
+ *   gtilde^(j) = 1/|N^(j)| * sum_{k in N^(j)} g^(k,j)
+ *   x^(i,j)    = x^(i,j) - gamma * gtilde^(j)   if worker i received it,
+ *                x^(i,j) - gamma * g^(i,j)      otherwise (it applies its own gradient).
+ *
+ * The paper gives no formulas for it; this is the reading in which a worker that misses the average
+ * still takes an SGD step.  Its point: a drop leaves a difference between replicas that nothing ever
+ * removes, because the model is the sum of all earlier gradients.  Masks, noise and rounding are those
+ * of rps_oracle_step.
+ */
+int rps_oracle_step_gradavg(int n, int64_t d, int dtype, void* x, const void* b, double gamma, double sigma,
+                            double p, uint64_t seed, uint64_t t, int self_delivery, int assign,
+                            const uint64_t* forced_up, const uint64_t* forced_down)
+{
+    if (n < 1 || n > 64 || d < 1) return -1;
+    uint64_t up[64], down[64];
+    int32_t cnt[64];
+    if (forced_up && forced_down) {
+        for (int j = 0; j < n; ++j) {
+            up[j] = forced_up[j];
+            down[j] = forced_down[j];
+            cnt[j] = 0;
+            for (int i = 0; i < n; ++i) cnt[j] += (int)((up[j] >> i) & 1);
+            if (cnt[j] == 0) down[j] = 0;
+        }
+    } else if (rps_oracle_masks(n, p, seed, t, self_delivery, assign, up, down, cnt, NULL) != 0) {
+        return -1;
+    }
+    const double lr = (double)(float)gamma;
+    const double s = (double)(float)sigma;
+    const int64_t block = rps_oracle_block_size(n, d);
+    double xs[64], grad[64];
+    for (int64_t c = 0; c < d; ++c) {
+        const int j = (int)(c / block);
+        for (int i = 0; i < n; ++i) {
+            xs[i] = load_elem(dtype, x, (int64_t)i * d + c);
+            grad[i] = xs[i] - load_elem(dtype, b, (int64_t)i * d + c);
+            if (s != 0.0) grad[i] += s * rps_oracle_noise(seed, t, i, c);
+        }
+        double gtilde = 0.0;
+        if (cnt[j] > 0) {
+            double sum = 0.0;
+            for (int k = 0; k < n; ++k)
+                if ((up[j] >> k) & 1) sum += grad[k];
+            gtilde = sum / (double)cnt[j];
+        }
+        for (int i = 0; i < n; ++i) {
+            double applied = ((down[j] >> i) & 1) ? gtilde : grad[i];
+            store_elem(dtype, x, (int64_t)i * d + c, xs[i] - lr * applied);
+        }
+    }
+    return 0;
+}
+
+int rps_oracle_run_gradavg(int n, int64_t d, int dtype, void* x, const void* b, double gamma, double sigma,
+                           double p, uint64_t seed, uint64_t t0, int64_t steps, int self_delivery, int assign)
+{
+    for (int64_t k = 0; k < steps; ++k) {
+        int rc = rps_oracle_step_gradavg(n, d, dtype, x, b, gamma, sigma, p, seed, t0 + (uint64_t)k,
+                                         self_delivery, assign, NULL, NULL);
+        if (rc != 0) return rc;
+    }
+    return 0;
+}

@@ -68,6 +68,10 @@ def _load():
                                    ctypes.c_double, ctypes.c_double, ctypes.c_uint64, ctypes.c_uint64,
                                    ctypes.c_int64, ctypes.c_int, ctypes.c_int]
     lib.rps_oracle_run.restype = ctypes.c_int
+    lib.rps_oracle_step_gradavg.argtypes = lib.rps_oracle_step.argtypes
+    lib.rps_oracle_step_gradavg.restype = ctypes.c_int
+    lib.rps_oracle_run_gradavg.argtypes = lib.rps_oracle_run.argtypes
+    lib.rps_oracle_run_gradavg.restype = ctypes.c_int
     lib.rps_oracle_step_columns.argtypes = [ctypes.c_int, ctypes.c_int64, ctypes.c_int, ctypes.c_int64, i64p,
                                             vp, vp, ctypes.c_double, ctypes.c_double, ctypes.c_double,
                                             ctypes.c_uint64, ctypes.c_uint64, ctypes.c_int, ctypes.c_int]
@@ -131,8 +135,9 @@ def block_size(n: int, d: int) -> int:
 
 def step(x: np.ndarray, b: np.ndarray, *, dtype: str, gamma: float, sigma: float, p: float, seed: int, t: int,
          self_delivery: bool = True, assign: int = ASSIGN_FIXED,
-         forced_up: Optional[np.ndarray] = None, forced_down: Optional[np.ndarray] = None) -> None:
-    """One iteration of Algorithm 1, in place on ``x``."""
+         forced_up: Optional[np.ndarray] = None, forced_down: Optional[np.ndarray] = None,
+         average_gradients: bool = False) -> None:
+    """One iteration of Algorithm 1 (or of its gradient-averaging comparison), in place on ``x``."""
     n, d = _check_state(x, b, dtype)
     u64p = ctypes.POINTER(ctypes.c_uint64)
     fu = fd = None
@@ -144,18 +149,21 @@ def step(x: np.ndarray, b: np.ndarray, *, dtype: str, gamma: float, sigma: float
         if fu_a.shape != (n,) or fd_a.shape != (n,):
             raise ValueError("forced masks must have n entries")
         fu, fd = fu_a.ctypes.data_as(u64p), fd_a.ctypes.data_as(u64p)
-    rc = _load().rps_oracle_step(n, d, _DTYPE[dtype], x.ctypes.data, b.ctypes.data, gamma, sigma, p, seed, t,
-                                 int(self_delivery), assign, fu, fd)
+    fn = _load().rps_oracle_step_gradavg if average_gradients else _load().rps_oracle_step
+    rc = fn(n, d, _DTYPE[dtype], x.ctypes.data, b.ctypes.data, gamma, sigma, p, seed, t, int(self_delivery), assign,
+            fu, fd)
     if rc != 0:
         raise ValueError("rps_oracle_step rejected its arguments")
 
 
 def run(x: np.ndarray, b: np.ndarray, *, dtype: str, gamma: float, sigma: float, p: float, seed: int,
-        t0: int, steps: int, self_delivery: bool = True, assign: int = ASSIGN_FIXED) -> None:
+        t0: int, steps: int, self_delivery: bool = True, assign: int = ASSIGN_FIXED,
+        average_gradients: bool = False) -> None:
     """``steps`` iterations of Algorithm 1 starting at step ``t0``, in place on ``x``."""
     n, d = _check_state(x, b, dtype)
-    rc = _load().rps_oracle_run(n, d, _DTYPE[dtype], x.ctypes.data, b.ctypes.data, gamma, sigma, p, seed, t0,
-                                steps, int(self_delivery), assign)
+    fn = _load().rps_oracle_run_gradavg if average_gradients else _load().rps_oracle_run
+    rc = fn(n, d, _DTYPE[dtype], x.ctypes.data, b.ctypes.data, gamma, sigma, p, seed, t0, steps, int(self_delivery),
+            assign)
     if rc != 0:
         raise ValueError("rps_oracle_run rejected its arguments")
 
