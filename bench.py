@@ -211,7 +211,7 @@ def run_cuda(args):
         w = w.scaled(d=args.d)
     b = wl.make_targets(w)
     r = binding.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma, kernel=args.kernel,
-                    workers_per_lane=args.workers_per_lane, stages=args.stages, consumer_warps=args.consumer_warps, copy_mode=args.copy_mode, slice_bytes=args.slice_bytes, store_mode=args.store_mode)
+                    workers_per_lane=args.workers_per_lane, stages=args.stages, consumer_warps=args.consumer_warps, copy_mode=args.copy_mode, slice_bytes=args.slice_bytes, store_mode=args.store_mode, average_gradients=args.average_gradients)
     r.set_targets(b)
     stream = r.stream
     bytes_per_step = w.bytes_per_step
@@ -251,7 +251,8 @@ def run_cuda(args):
     fused_avg_ms = fused_ms / max(fused_n, 1)
     achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
     traffic = None
-    default_shape = not (args.kernel or args.workers_per_lane or args.stages or args.consumer_warps or args.copy_mode or args.slice_bytes or args.store_mode)
+    default_shape = not (args.kernel or args.workers_per_lane or args.stages or args.consumer_warps or args.copy_mode or args.slice_bytes or args.store_mode
+                         or args.average_gradients)
     if default_shape and NCU_TRAFFIC["kernel_digest"] == kernel_digest():
         traffic = NCU_TRAFFIC["bytes_per_launch"].get(w.name)
 
@@ -265,6 +266,7 @@ def run_cuda(args):
             "n": w.n, "d": w.d, "p": w.p, "replicas": "one independent job per GPU, no collective",
             "kernel_shape": {"kernel": args.kernel, "workers_per_lane": args.workers_per_lane, "stages": args.stages,
                              "consumer_warps": args.consumer_warps, "copy_mode": args.copy_mode, "slice_bytes": args.slice_bytes, "store_mode": args.store_mode},
+            "average": "gradients" if args.average_gradients else "models",
             "l2": "inputs larger than L2 (x and b are %.0f MB each)" % (row_bytes / 1e6),
             "algorithmic_bytes_per_step": bytes_per_step,
             "hbm_gbs_whole_step": bytes_per_step / (total_ms / args.steps * 1e-3) / 1e9,
@@ -356,6 +358,8 @@ def main(argv=None):
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--consumer-warps", type=int, default=0)
     ap.add_argument("--slice-bytes", type=int, default=0, help="staged kernel, bf16: 16 or 8 bytes per lane and row")
+    ap.add_argument("--average-gradients", action="store_true",
+                    help="time the gradient-averaging comparison of Section 5 instead of RPS (model averaging)")
     ap.add_argument("--store-mode", type=int, default=0, help="staged kernel: 1 register stores, 2 TMA stores")
     ap.add_argument("--copy-mode", type=int, default=0, help="staged kernel: 1 bulk copy per row, 2 TMA boxes")
     args = ap.parse_args(argv)

@@ -60,6 +60,16 @@ typedef enum rps_dtype { RPS_F32 = 0, RPS_BF16 = 1 } rps_dtype;
  *                   replacement") and as the lemmas of the supplement assume. */
 typedef enum rps_assign { RPS_ASSIGN_FIXED = 0, RPS_ASSIGN_PERM = 1 } rps_assign;
 
+/* What the workers exchange.
+ * RPS_AVERAGE_MODELS:    the models v after the local SGD step: the RPS algorithm (Algorithm 1).
+ * RPS_AVERAGE_GRADIENTS: the stochastic gradients, over the same unreliable Reduce-Scatter / All-Gather
+ *                        (Section 5, "Comparison with Gradient Averaging"): the server of block j averages
+ *                        the gradients that arrived; a worker that receives the average applies it,
+ *                        x <- x - gamma * gtilde, any other worker applies its own gradient.  A drop then
+ *                        leaves a difference between replicas that never decays, which is the paper's
+ *                        argument for averaging models. */
+typedef enum rps_average { RPS_AVERAGE_MODELS = 0, RPS_AVERAGE_GRADIENTS = 1 } rps_average;
+
 typedef struct rps_options {
     int32_t dtype;         /* rps_dtype, default RPS_F32                                   */
     int32_t assign;        /* rps_assign, default RPS_ASSIGN_FIXED                         */
@@ -96,6 +106,7 @@ typedef struct rps_options {
     int32_t withhold_copies;  /* kernel 2, test aid for that time-out path: 1 = the producer warp
                                  issues no copies, so the compute warps' waits run out, x is
                                  left unchanged and the error is reported; 0 otherwise       */
+    int32_t average;          /* rps_average, default RPS_AVERAGE_MODELS                        */
 } rps_options;
 
 /*

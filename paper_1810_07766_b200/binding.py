@@ -38,7 +38,7 @@ class rps_options(ctypes.Structure):
                 ("workers_per_lane", ctypes.c_int32), ("stages", ctypes.c_int32), ("consumer_warps", ctypes.c_int32),
                 ("copy_mode", ctypes.c_int32), ("slice_bytes", ctypes.c_int32),
                 ("store_mode", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32),
-                ("withhold_copies", ctypes.c_int32)]
+                ("withhold_copies", ctypes.c_int32), ("average", ctypes.c_int32)]
 
 
 class RPSError(RuntimeError):
@@ -114,7 +114,7 @@ class RPS:
     def __init__(self, n: int, d: int, p: float, gamma: float, seed: int, *, dtype: str = "f32", sigma: float = 0.0,
                  assign: int = RPS_ASSIGN_FIXED, self_delivery: bool = True, mask_window: int = 32,
                  kernel: int = 0, workers_per_lane: int = 0, stages: int = 0, consumer_warps: int = 0,
-                 row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0, wait_limit_ms: int = 0, withhold_copies: bool = False, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+                 row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0, wait_limit_ms: int = 0, withhold_copies: bool = False, average_gradients: bool = False, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         if not torch.cuda.is_available():
@@ -130,6 +130,7 @@ class RPS:
         opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps = kernel, workers_per_lane, stages, consumer_warps
         opt.row_skew_lines, opt.copy_mode, opt.slice_bytes = row_skew_lines, copy_mode, slice_bytes
         opt.store_mode, opt.wait_limit_ms, opt.withhold_copies = store_mode, wait_limit_ms, int(withhold_copies)
+        opt.average = int(average_gradients)
         self._check(self._lib.rps_configure(self._h, ctypes.byref(opt)), "rps_configure")
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
         self.pitch = int(self._lib.rps_pitch(self._h))

@@ -181,6 +181,7 @@ int run_fused(rps_handle* h, const rps::StepMasks* masks)
     prm.n = h->n;
     prm.narrow = h->d < ((int64_t)1 << 31);
     prm.error = h->error_word();
+    prm.average_gradients = h->opt.average == RPS_AVERAGE_GRADIENTS;
     rps::set_sgd_scalars(prm, h->gamma, h->sigma);
     prm.t_lo = (uint32_t)h->t;
     prm.t_hi = (uint32_t)(h->t >> 32);
@@ -251,6 +252,7 @@ int rps_default_options(rps_options* opt)
     opt->store_mode = 0;
     opt->wait_limit_ms = 0;
     opt->withhold_copies = 0;
+    opt->average = RPS_AVERAGE_MODELS;
     return RPS_OK;
 }
 
@@ -324,6 +326,8 @@ int rps_configure(rps_handle* h, const rps_options* opt)
         return fail(h, RPS_EINVAL, "consumer_warps must be 0 (auto) or 1..24");
     if (opt->slice_bytes != 0 && opt->slice_bytes != 8 && opt->slice_bytes != 16)
         return fail(h, RPS_EINVAL, "slice_bytes must be 0 (auto), 8 or 16");
+    if (opt->average != RPS_AVERAGE_MODELS && opt->average != RPS_AVERAGE_GRADIENTS)
+        return fail(h, RPS_EINVAL, "unknown average");
     if (opt->wait_limit_ms < 0 || opt->wait_limit_ms > 10000)
         return fail(h, RPS_EINVAL, "wait_limit_ms must be 0 (default) or 1..10000");
     if (opt->withhold_copies != 0 && opt->withhold_copies != 1)

@@ -168,20 +168,10 @@ struct RowVec<__nv_bfloat16, 4> {
     }
 };
 
-// Local SGD step of one lane: WPT workers (starting at the even worker w_first) x
-// VEC consecutive columns starting at column c, evaluated as
-//   v = x - gamma * ((x - b) + sigma * xi) = keep * x + gamma * b - (gamma * sigma) * xi,  keep = 1 - gamma.
-// One Philox draw serves a worker pair on four columns.
+// Subtracts (gamma * sigma) * xi from v: one Philox draw per worker pair and four columns.
 template <int VEC, int WPT>
-__device__ __forceinline__ void local_sgd(const float (&xv)[WPT][VEC], const float (&bv)[WPT][VEC],
-                                          float (&v)[WPT][VEC], int64_t c, int w_first, const FusedParams& prm)
+__device__ __forceinline__ void add_gradient_noise(float (&v)[WPT][VEC], int64_t c, int w_first, const FusedParams& prm)
 {
-    static_assert(WPT % 2 == 0 && VEC % 4 == 0, "noise draws cover worker pairs and 4 columns");
-#pragma unroll
-    for (int w = 0; w < WPT; ++w)
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) v[w][e] = fmaf(prm.gamma, bv[w][e], prm.keep * xv[w][e]);
-    if (!prm.noisy) return;
 #pragma unroll
     for (int w = 0; w < WPT; w += 2) {
 #pragma unroll
@@ -199,6 +189,30 @@ __device__ __forceinline__ void local_sgd(const float (&xv)[WPT][VEC], const flo
             }
         }
     }
+}
+
+// Local SGD step of one lane: WPT workers (starting at the even worker w_first) x
+// VEC consecutive columns starting at column c, evaluated as
+//   v = x - gamma * ((x - b) + sigma * xi) = keep * x + gamma * b - (gamma * sigma) * xi,  keep = 1 - gamma.
+// One Philox draw serves a worker pair on four columns.  GRAD: leave the update v - x in v instead.
+template <int VEC, int WPT, bool GRAD>
+__device__ __forceinline__ void local_sgd(const float (&xv)[WPT][VEC], const float (&bv)[WPT][VEC],
+                                          float (&v)[WPT][VEC], int64_t c, int w_first, const FusedParams& prm)
+{
+    static_assert(WPT % 2 == 0 && VEC % 4 == 0, "noise draws cover worker pairs and 4 columns");
+#pragma unroll
+    for (int w = 0; w < WPT; ++w)
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) v[w][e] = fmaf(prm.gamma, bv[w][e], prm.keep * xv[w][e]);
+    if (GRAD) {
+        // gradient averaging exchanges the update u = v - x = -gamma * g instead of the model (x is
+        // taken off before the noise goes in, so that its registers are free by then)
+#pragma unroll
+        for (int w = 0; w < WPT; ++w)
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) v[w][e] -= xv[w][e];
+    }
+    if (prm.noisy) add_gradient_noise<VEC, WPT>(v, c, w_first, prm);
 }
 
 // s += v where `take` is set, as one predicated add (no branch, no select); a value that is

@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(256) rps_mask_kernel(const MaskParams prm)
 // read once.  (The staged form in rps_staged.cu does the same arithmetic with
 // the loads decoupled from the warps through shared memory.)
 // --------------------------------------------------------------------------
-template <typename T, int VEC, int WPT, int G, int THREADS>
+template <typename T, int VEC, int WPT, int G, int THREADS, bool GRAD>
 __global__ void __launch_bounds__(THREADS) rps_fused_direct_kernel(const FusedParams prm)
 {
     constexpr int LPG = 32 / G;
@@ -116,9 +116,23 @@ __global__ void __launch_bounds__(THREADS) rps_fused_direct_kernel(const FusedPa
                 RowVec<T, VEC>::unpack(raw_x, xv[w]);
                 RowVec<T, VEC>::unpack(raw_b, bv[w]);
             }
-            local_sgd<VEC, WPT>(xv, bv, v, c, w_first, prm);
+            local_sgd<VEC, WPT, GRAD>(xv, bv, v, c, w_first, prm);
         }
         const uint32_t live_bits = average_and_select<VEC, WPT, G>(v, c, col_live, w_first, masks, cursor, prm);
+        if (GRAD) {
+            // v holds the update each worker applies (the average one where it arrived): x_{t+1} = x + update
+            const int64_t c_read = col_live ? c : 0;
+#pragma unroll
+            for (int w = 0; w < WPT; ++w) {
+                const int row = w_first + w < n ? w_first + w : n - 1;
+                float xv[VEC];
+                RowVec<T, VEC>::unpack(__ldcs(reinterpret_cast<const typename RowVec<T, VEC>::Raw*>(
+                                           x + (int64_t)row * prm.pitch + c_read)),
+                                       xv);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) v[w][e] += xv[e];
+            }
+        }
         T* dst = x + (int64_t)w_first * prm.pitch + c;  // this lane's slice of its first worker's row
         if (live_bits == (1u << VEC) - 1u) {
 #pragma unroll
@@ -203,7 +217,7 @@ namespace {
 
 constexpr int kThreads = 256;
 
-template <typename T, int VEC, int WPT, int G>
+template <typename T, int VEC, int WPT, int G, bool GRAD = false>
 cudaError_t launch_direct_as(const FusedParams& prm, int sm_count, cudaStream_t stream)
 {
     constexpr int warp_cols = (32 / G) * VEC;
@@ -213,7 +227,7 @@ cudaError_t launch_direct_as(const FusedParams& prm, int sm_count, cudaStream_t 
     if (per_sm == 0) {
         int occ = 0;
         cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-            &occ, rps_fused_direct_kernel<T, VEC, WPT, G, kThreads>, kThreads, 0);
+            &occ, rps_fused_direct_kernel<T, VEC, WPT, G, kThreads, GRAD>, kThreads, 0);
         if (err != cudaSuccess) return err;
         per_sm = occ < 1 ? 1 : occ;
     }
@@ -221,7 +235,7 @@ cudaError_t launch_direct_as(const FusedParams& prm, int sm_count, cudaStream_t 
     int64_t grid = (int64_t)sm_count * per_sm;
     if (grid > ctas_needed) grid = ctas_needed;
     if (grid < 1) grid = 1;
-    rps_fused_direct_kernel<T, VEC, WPT, G, kThreads><<<(unsigned)grid, kThreads, 0, stream>>>(prm);
+    rps_fused_direct_kernel<T, VEC, WPT, G, kThreads, GRAD><<<(unsigned)grid, kThreads, 0, stream>>>(prm);
     return cudaGetLastError();
 }
 
@@ -229,6 +243,15 @@ template <typename T, int VEC>
 cudaError_t launch_direct_for_n(const FusedParams& prm, int wpt, int sm_count, cudaStream_t stream)
 {
     const int n = prm.n;
+    if (prm.average_gradients) {
+        // the gradient-averaging comparison is built in one family of shapes only
+        if (n <= 2) return launch_direct_as<T, VEC, 2, 1, true>(prm, sm_count, stream);
+        if (n <= 4) return launch_direct_as<T, VEC, 4, 1, true>(prm, sm_count, stream);
+        if (n <= 8) return launch_direct_as<T, VEC, 4, 2, true>(prm, sm_count, stream);
+        if (n <= 16) return launch_direct_as<T, VEC, 4, 4, true>(prm, sm_count, stream);
+        if (n <= 32) return launch_direct_as<T, VEC, 4, 8, true>(prm, sm_count, stream);
+        return launch_direct_as<T, VEC, 4, 16, true>(prm, sm_count, stream);
+    }
     if (wpt == 4) {
         if (n <= 4) return launch_direct_as<T, VEC, 4, 1>(prm, sm_count, stream);
         if (n <= 8) return launch_direct_as<T, VEC, 4, 2>(prm, sm_count, stream);

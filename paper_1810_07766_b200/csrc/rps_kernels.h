@@ -48,6 +48,7 @@ struct FusedParams {
     float gamma;
     float noise_scale;  // -2 ln 2 * (gamma * sigma)^2
     int32_t noisy;      // sigma != 0
+    int32_t average_gradients;  // 1: the updates -gamma*g are averaged and applied to x (Section 5's comparison)
     uint32_t t_lo, t_hi;
     uint32_t key0, key1;
     uint32_t round_key[10][2];  // Philox round keys: key + r * (0x9E3779B9, 0xBB67AE85)

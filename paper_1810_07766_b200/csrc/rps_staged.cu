@@ -163,7 +163,7 @@ constexpr int max_consumer_warps(int wpt, int vec, int elem)
     return wpt >= 8 ? ((elem == 2 && vec == 4) ? 20 : 12) : kMaxConsumerWarps;
 }
 
-template <typename T, int VEC, int WPT, int G>
+template <typename T, int VEC, int WPT, int G, bool GRAD>
 __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) + 2) * 32)
     rps_fused_staged_kernel(const FusedParams prm, const StagedShape shape, const __grid_constant__ CUtensorMap map_x,
                             const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out)
@@ -307,6 +307,8 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
     const uint32_t lane_off =
         (uint32_t)(col_in_tile / shape.box_cols) * shape.box_bytes + (uint32_t)(col_in_tile % shape.box_cols) * elem;
     const bool out_tiles = shape.store_mode == 2, in_place = shape.store_mode == 3;
+    // the stage is read a second time after the average when updates rather than models are averaged
+    const bool hold_stage = in_place || GRAD;
     const uint32_t lane_out_off = out_tiles ? (uint32_t)(col_in_tile / shape.out_box_cols) * shape.out_box_bytes +
                                                   (uint32_t)(col_in_tile % shape.out_box_cols) * elem
                                             : 0u;
@@ -345,14 +347,30 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
                     RowVec<T, VEC>::unpack(raw_x, xv[w]);
                     RowVec<T, VEC>::unpack(raw_b, bv[w]);
                 }
-                if (!in_place) {
+                if (!hold_stage) {
                     // this warp has read everything it needs from the stage: hand it back to the producer
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_addr(&empty[stage]));
                 }
-                local_sgd<VEC, WPT>(xv, bv, v, c, w_first, prm);
+                local_sgd<VEC, WPT, GRAD>(xv, bv, v, c, w_first, prm);
             }
             const uint32_t live_bits = average_and_select<VEC, WPT, G>(v, c, col_live, w_first, masks, cursor, prm);
+            if (GRAD) {
+                // v holds the update each worker applies (the average one where it arrived): x_{t+1} = x + update
+#pragma unroll
+                for (int w = 0; w < WPT; ++w) {
+                    const int row = w_first + w < n ? w_first + w : n - 1;
+                    float xv[VEC];
+                    RowVec<T, VEC>::unpack(
+                        *reinterpret_cast<const typename RowVec<T, VEC>::Raw*>(base + (size_t)row * shape.row_bytes), xv);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) v[w][e] += xv[e];
+                }
+                if (!in_place) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_addr(&empty[stage]));
+                }
+            }
             if (in_place) {
                 // every lane overwrites exactly the slices of x it read; columns past d are clipped by
                 // the tensor store
@@ -533,10 +551,10 @@ bool encode_rows(CUtensorMap* map, const void* base, bool bf16, const FusedParam
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <typename T, int VEC, int WPT, int G>
+template <typename T, int VEC, int WPT, int G, bool GRAD = false>
 cudaError_t launch_staged_as(const FusedParams& prm, const FusedTuning& tune, int sm_count, cudaStream_t stream)
 {
-    auto kernel = rps_fused_staged_kernel<T, VEC, WPT, G>;
+    auto kernel = rps_fused_staged_kernel<T, VEC, WPT, G, GRAD>;
     static size_t smem_limit = 0;   // opt-in shared memory per CTA of this device
     static uint32_t smem_granted = 0;
     static int occ_threads = 0, occ_per_sm = 0;
@@ -587,6 +605,15 @@ cudaError_t launch_staged_for_n(const FusedParams& prm, const FusedTuning& tune,
     const int n = prm.n;
     // workers per lane: asked for, or 8 where that halves the shuffle stages and pays for its
     // registers (bf16 replicas, or more than 32 workers), else 4
+    if (prm.average_gradients) {
+        // the gradient-averaging comparison is built in one family of shapes only
+        if (n <= 2) return launch_staged_as<T, VEC, 2, 1, true>(prm, tune, sm_count, stream);
+        if (n <= 4) return launch_staged_as<T, VEC, 4, 1, true>(prm, tune, sm_count, stream);
+        if (n <= 8) return launch_staged_as<T, VEC, 4, 2, true>(prm, tune, sm_count, stream);
+        if (n <= 16) return launch_staged_as<T, VEC, 4, 4, true>(prm, tune, sm_count, stream);
+        if (n <= 32) return launch_staged_as<T, VEC, 4, 8, true>(prm, tune, sm_count, stream);
+        return launch_staged_as<T, VEC, 4, 16, true>(prm, tune, sm_count, stream);
+    }
     int wpt = tune.workers_per_lane;
     if (wpt == 0) wpt = (n > 4 && (sizeof(T) == 2 || n > 32)) ? 8 : 4;
     if (wpt == 8) {
@@ -618,7 +645,7 @@ cudaError_t launch_fused_staged(const FusedParams& prm, const FusedTuning& tune,
 {
     // TMA coordinates are 32-bit: rows of 2^31 elements or more go through the direct kernel
     if (prm.pitch >= ((int64_t)1 << 31)) return launch_fused_direct(prm, tune, bf16, sm_count, stream);
-    if (bf16 && tune.slice_bytes == 8) {
+    if (bf16 && tune.slice_bytes == 8 && !prm.average_gradients) {
         // narrow bf16 slices exist for 8 workers per lane only
         const int n = prm.n;
         if (n <= 8) return launch_staged_as<__nv_bfloat16, 4, 8, 1>(prm, tune, sm_count, stream);

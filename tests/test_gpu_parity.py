@@ -442,3 +442,28 @@ def test_a_wait_that_runs_out_is_reported_and_harmless(rps_mod, store_mode):
     r.step()
     assert np.isfinite(r.read()).all()
     r.close()
+
+
+# ------------------------------------------------------------------ gradient averaging (Section 5's comparison)
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg4", "cfg5"])
+def test_gradient_averaging_parity(rps_mod, oracle, name):
+    w = TWINS[name].scaled(d=TWINS[name].d // 2 + (1 if name != "cfg5" else 0), steps=6)
+    b = wl.make_targets(w)
+    want = wl.make_initial(w)
+    oracle.run(want, b, dtype=w.dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps,
+               average_gradients=True)
+    tol = BF16_TOL if w.dtype == "bf16" else 6 * STEP_TOL
+    for kernel, store_mode, copy_mode in ((0, 0, 0), (1, 0, 0), (2, 1, 1), (2, 2, 2), (2, 3, 0)):
+        r = make(rps_mod, w, average_gradients=True, kernel=kernel, store_mode=store_mode, copy_mode=copy_mode)
+        r.set_targets(b)
+        r.step_n(w.steps)
+        assert_close(w, r.read(), want, tol)
+        r.close()
+    # and it is a different method: model averaging from the same inputs ends elsewhere
+    r = make(rps_mod, w)
+    r.set_targets(b)
+    r.step_n(w.steps)
+    other = r.read()
+    r.close()
+    assert np.abs(wl.as_float64(w, other) - wl.as_float64(w, want)).max() > 1e-3
