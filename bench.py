@@ -168,6 +168,24 @@ def timed_steps(torch, stream, fn, device):
     return max_over_ranks(start.elapsed_time(stop), device)
 
 
+def in_situ_copy_gbs(torch, device) -> float:
+    """Read+write bytes per second of a plain device copy of 1 GiB on this GPU, now (best of 6): the same
+    kind of measurement as the recorded peak, taken in this process, because the machine's GPUs differ."""
+    a = torch.empty(1 << 29, dtype=torch.bfloat16, device=device)
+    c = torch.empty_like(a)
+    best = float("inf")
+    for _ in range(6):
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        c.copy_(a)
+        stop.record()
+        torch.cuda.synchronize(device)
+        best = min(best, start.elapsed_time(stop))
+    del a, c
+    torch.cuda.empty_cache()
+    return 2 * (1 << 30) / (best * 1e-3) / 1e9
+
+
 def oracle_baseline(w, b, seconds_hint="one step"):
     """The CPU oracle, as it stands, on one full-size step of the workload (single thread)."""
     import oracle
@@ -247,6 +265,7 @@ def run_cuda(args):
                "call": "rps_step_host (pinned host x and b)"}
     row_bytes = w.n * w.d * w.elem_bytes
 
+    copy_gbs = in_situ_copy_gbs(torch, device)
     peak, peak_kind = measured_peak_gbs()
     fused_avg_ms = fused_ms / max(fused_n, 1)
     achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
@@ -278,7 +297,8 @@ def run_cuda(args):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": fused_kernel_name(args, w),
                      "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n,
-                     "mask_kernel_ms_per_launch": mask_ms / max(mask_n, 1), "mask_launches_timed": mask_n},
+                     "mask_kernel_ms_per_launch": mask_ms / max(mask_n, 1), "mask_launches_timed": mask_n,
+                     "in_situ_copy_gbs": copy_gbs, "frac_of_in_situ_copy": achieved / copy_gbs},
     }
     r.close()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

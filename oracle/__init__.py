@@ -13,6 +13,7 @@ from .rps_oracle import (  # noqa: F401
     double_to_bf16,
     masks,
     noise,
+    philox4x32,
     philox4x32_10,
     run,
     step,

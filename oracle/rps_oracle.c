@@ -42,7 +42,7 @@
 /* two fixed odd constants, and mixes the high halves with the other counter   */
 /* words and the round key; the key grows by a Weyl constant between rounds.   */
 /* ------------------------------------------------------------------------- */
-void rps_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+void rps_oracle_philox4x32(const uint32_t ctr[4], const uint32_t key[2], int rounds, uint32_t out[4])
 {
     const uint64_t mult_a = 0xD2511F53u;
     const uint64_t mult_b = 0xCD9E8D57u;
@@ -50,7 +50,7 @@ void rps_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint
     const uint32_t weyl_b = 0xBB67AE85u;
     uint32_t c[4] = {ctr[0], ctr[1], ctr[2], ctr[3]};
     uint32_t k[2] = {key[0], key[1]};
-    for (int round = 0; round < 10; ++round) {
+    for (int round = 0; round < rounds; ++round) {
         uint64_t prod_a = mult_a * (uint64_t)c[0];
         uint64_t prod_b = mult_b * (uint64_t)c[2];
         uint32_t next[4];
@@ -65,16 +65,32 @@ void rps_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint
     memcpy(out, c, sizeof c);
 }
 
+void rps_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    rps_oracle_philox4x32(ctr, key, 10, out);
+}
+
 /* Counter layout shared by convention with the CUDA library (each side has its
  * own code for it): words 0,1 = step t; word 3's low byte tags the stream.     */
 enum { STREAM_UP = 0, STREAM_DOWN = 1, STREAM_NOISE = 2, STREAM_PERM = 3 };
 
-static void philox_draw(uint64_t seed, uint64_t t, uint32_t w2, uint32_t w3, uint32_t out[4])
+static void philox_draw_rounds(uint64_t seed, uint64_t t, uint32_t w2, uint32_t w3, int rounds, uint32_t out[4])
 {
     uint32_t ctr[4] = {(uint32_t)t, (uint32_t)(t >> 32), w2, w3};
     uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
-    rps_oracle_philox4x32_10(ctr, key, out);
+    rps_oracle_philox4x32(ctr, key, rounds, out);
 }
+
+/* Drop masks and the server draw use the standard ten rounds. */
+static void philox_draw(uint64_t seed, uint64_t t, uint32_t w2, uint32_t w3, uint32_t out[4])
+{
+    philox_draw_rounds(seed, t, w2, w3, 10, out);
+}
+
+/* The gradient noise uses Philox4x32 with seven rounds, the fewest with which the generator's authors
+ * report it passing their statistical test batteries (ten is their default, with a safety margin).
+ * The paper asks of the noise only zero mean and bounded variance (Assumption 1). */
+#define RPS_ORACLE_NOISE_ROUNDS 7
 
 /* ------------------------------------------------------------------------- */
 /* Unreliable channel (Section 3): every message is lost independently with    */
@@ -146,7 +162,8 @@ int rps_oracle_masks(int n, double p, uint64_t seed, uint64_t t, int self_delive
 
 /* ------------------------------------------------------------------------- */
 /* Gradient noise xi(t, i, c): a standard normal per (step, worker, column).   */
-/* One Philox draw (four 32-bit words) serves a pair of workers (2k, 2k+1) on   */
+/* One 7-round Philox draw (four 32-bit words) serves a pair of workers (2k,     */
+/* 2k+1) on                                                                     */
 /* four consecutive columns 4q..4q+3.  Each word gives one Box-Muller pair:     */
 /* its low 16 bits are the radius uniform, its high 16 bits the angle uniform,  */
 /* both taken at bin centres (k + 1/2) / 2^16 so that neither is 0 or 1.       */
@@ -157,7 +174,8 @@ double rps_oracle_noise(uint64_t seed, uint64_t t, int i, int64_t c)
     uint32_t r[4];
     int64_t q = c / 4;
     int e = (int)(c % 4);
-    philox_draw(seed, t, (uint32_t)q, (uint32_t)STREAM_NOISE | ((uint32_t)(i / 2) << 8), r);
+    philox_draw_rounds(seed, t, (uint32_t)q, (uint32_t)STREAM_NOISE | ((uint32_t)(i / 2) << 8),
+                       RPS_ORACLE_NOISE_ROUNDS, r);
     uint32_t word = r[(i % 2) * 2 + e / 2];
     double u_radius = ((double)(word & 0xFFFFu) + 0.5) / 65536.0;
     double u_angle = ((double)(word >> 16) + 0.5) / 65536.0;

@@ -49,6 +49,8 @@ def _load():
     vp = ctypes.c_void_p
     lib.rps_oracle_philox4x32_10.argtypes = [u32p, u32p, u32p]
     lib.rps_oracle_philox4x32_10.restype = None
+    lib.rps_oracle_philox4x32.argtypes = [u32p, u32p, ctypes.c_int, u32p]
+    lib.rps_oracle_philox4x32.restype = None
     lib.rps_oracle_masks.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_uint64, ctypes.c_uint64,
                                      ctypes.c_int, ctypes.c_int, u64p, u64p, i32p, i32p]
     lib.rps_oracle_masks.restype = ctypes.c_int
@@ -97,6 +99,14 @@ def philox4x32_10(ctr, key) -> Tuple[int, int, int, int]:
     k = (ctypes.c_uint32 * 2)(*[int(v) & 0xFFFFFFFF for v in key])
     out = (ctypes.c_uint32 * 4)()
     _load().rps_oracle_philox4x32_10(c, k, out)
+    return tuple(int(v) for v in out)
+
+
+def philox4x32(ctr, key, rounds: int) -> Tuple[int, int, int, int]:
+    c = (ctypes.c_uint32 * 4)(*[int(v) & 0xFFFFFFFF for v in ctr])
+    k = (ctypes.c_uint32 * 2)(*[int(v) & 0xFFFFFFFF for v in key])
+    out = (ctypes.c_uint32 * 4)()
+    _load().rps_oracle_philox4x32(c, k, rounds, out)
     return tuple(int(v) for v in out)
 
 

@@ -206,3 +206,16 @@ def test_noise_box_muller_partners_share_a_radius(oracle):
 def test_noise_is_a_pure_function(oracle):
     assert oracle.noise(1, 2, 3, 4) == oracle.noise(1, 2, 3, 4)
     assert oracle.noise(1, 2, 3, 4) != oracle.noise(1, 2 + (1 << 32), 3, 4)
+
+
+def test_round_count_is_honoured(oracle):
+    """Ten rounds are seven rounds followed by three more under the advanced key: ties the reduced-round
+    generator of the gradient noise to the known-answer vectors of the ten-round one."""
+    weyl = (0x9E3779B9, 0xBB67AE85)
+    for ctr, key, want in read_kat():
+        assert list(oracle.philox4x32(ctr, key, 10)) == want
+        mid = oracle.philox4x32(ctr, key, 7)
+        later_key = [(key[0] + 7 * weyl[0]) & 0xFFFFFFFF, (key[1] + 7 * weyl[1]) & 0xFFFFFFFF]
+        assert list(oracle.philox4x32(mid, later_key, 3)) == want
+        assert list(mid) != want and list(oracle.philox4x32(ctr, key, 6)) != list(mid)
+    assert oracle.philox4x32([1, 2, 3, 4], [5, 6], 0) == (1, 2, 3, 4)
