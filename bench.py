@@ -43,7 +43,7 @@ NCU_TRAFFIC = {
 def kernel_digest() -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_1810_07766_b200", "csrc")
-    for name in ("rps_device.cuh", "rps_kernels.cu", "rps_staged.cu"):
+    for name in ("rps_device.cuh", "rps_direct.cuh", "rps_kernels.cu", "rps_staged.cuh", "rps_staged.cu"):
         with open(os.path.join(csrc, name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -231,6 +231,9 @@ def run_cuda(args):
     r = binding.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma, kernel=args.kernel,
                     workers_per_lane=args.workers_per_lane, stages=args.stages, consumer_warps=args.consumer_warps, copy_mode=args.copy_mode, slice_bytes=args.slice_bytes, store_mode=args.store_mode, average_gradients=args.average_gradients)
     r.set_targets(b)
+    if args.track:
+        # every step of the run also records the distance to the optimum and the consensus error
+        r.track(2 * max(args.warmup, 3) + 2 * args.steps + args.warmup + 64)
     stream = r.stream
     bytes_per_step = w.bytes_per_step
 
@@ -271,7 +274,7 @@ def run_cuda(args):
     achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
     traffic = None
     default_shape = not (args.kernel or args.workers_per_lane or args.stages or args.consumer_warps or args.copy_mode or args.slice_bytes or args.store_mode
-                         or args.average_gradients)
+                         or args.average_gradients or args.track)
     if default_shape and NCU_TRAFFIC["kernel_digest"] == kernel_digest():
         traffic = NCU_TRAFFIC["bytes_per_launch"].get(w.name)
 
@@ -286,6 +289,7 @@ def run_cuda(args):
             "kernel_shape": {"kernel": args.kernel, "workers_per_lane": args.workers_per_lane, "stages": args.stages,
                              "consumer_warps": args.consumer_warps, "copy_mode": args.copy_mode, "slice_bytes": args.slice_bytes, "store_mode": args.store_mode},
             "average": "gradients" if args.average_gradients else "models",
+            "tracked": bool(args.track),
             "l2": "inputs larger than L2 (x and b are %.0f MB each)" % (row_bytes / 1e6),
             "algorithmic_bytes_per_step": bytes_per_step,
             "hbm_gbs_whole_step": bytes_per_step / (total_ms / args.steps * 1e-3) / 1e9,
@@ -380,6 +384,8 @@ def main(argv=None):
     ap.add_argument("--slice-bytes", type=int, default=0, help="staged kernel, bf16: 16 or 8 bytes per lane and row")
     ap.add_argument("--average-gradients", action="store_true",
                     help="time the gradient-averaging comparison of Section 5 instead of RPS (model averaging)")
+    ap.add_argument("--track", action="store_true",
+                    help="time tracked steps: distance to the optimum and consensus error as a by-product of the pass")
     ap.add_argument("--store-mode", type=int, default=0, help="staged kernel: 1 register stores, 2 TMA stores")
     ap.add_argument("--copy-mode", type=int, default=0, help="staged kernel: 1 bulk copy per row, 2 TMA boxes")
     args = ap.parse_args(argv)

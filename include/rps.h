@@ -217,6 +217,33 @@ int rps_read_masks(rps_handle* h, uint64_t t, uint64_t* up, uint64_t* down, int3
 int rps_diag(rps_handle* h, double* dist2_to_opt, double* consensus);
 
 /*
+ * rps_track: the same two quantities as rps_diag, as a by-product of the fused pass itself (no extra
+ * read of x or b): the step measures what it leaves behind from the values it holds in registers,
+ * so a run can follow the distance to the optimum (Section 5 plots convergence against the optimum;
+ * Lemma 3 bounds the consensus error) at every step.
+ *   trace_dev : device array of 2 * capacity doubles, 16-byte aligned, owned by the caller, who keeps
+ *               it alive until tracking is switched off or the handle destroyed.  Cleared here
+ *               (asynchronously, on the bound stream).
+ *   capacity  : number of steps to record; later steps run untracked.
+ * The k-th step enqueued after this call (k = 0 .. capacity-1; rps_step, rps_step_n, rps_step_forced,
+ * rps_step_host alike) adds into trace_dev[2k] the value ||xbar - mean_i b_i||^2 and into
+ * trace_dev[2k+1] the value sum_i ||x^(i) - xbar||^2 of the state x_{t+1} it produces (for bf16
+ * replicas: of the rounded values it stores).  fp32 arithmetic relative to a per-column pivot
+ * within a tile of columns, fp64 across tiles; the order of the fp64 additions is not fixed, so the
+ * last bits vary from run to run.  Tracked steps run in the lane shape with 4 workers per lane
+ * whatever workers_per_lane says.  trace_dev == NULL or capacity == 0 switches tracking off.
+ * Errors: RPS_ESTATE before rps_bind, RPS_EINVAL for a negative capacity or a misaligned pointer.
+ */
+int rps_track(rps_handle* h, double* trace_dev, int64_t capacity);
+
+/*
+ * rps_read_trace: synchronises and copies the entries recorded so far (at most max_entries) to
+ * trace_host_out as pairs {dist2_to_opt, consensus}; *entries receives how many pairs were
+ * written.  RPS_ESTATE when tracking is off.
+ */
+int rps_read_trace(rps_handle* h, double* trace_host_out, int64_t max_entries, int64_t* entries);
+
+/*
  * Per-kernel device timing.  rps_profile(h, 1) makes every later kernel launch of
  * this handle be bracketed by CUDA events on the bound stream; rps_profile_read
  * synchronises and returns the summed device time and launch count of the fused

@@ -26,7 +26,8 @@ _DTYPE = {"f32": RPS_F32, "bf16": RPS_BF16}
 SYMBOLS = (
     "rps_create", "rps_destroy", "rps_default_options", "rps_configure", "rps_pitch", "rps_scratch_bytes",
     "rps_bind", "rps_set_targets", "rps_write", "rps_set_step", "rps_get_step", "rps_step", "rps_step_n",
-    "rps_step_forced", "rps_step_host", "rps_read", "rps_read_masks", "rps_diag", "rps_profile",
+    "rps_step_forced", "rps_step_host", "rps_read", "rps_read_masks", "rps_diag", "rps_track", "rps_read_trace",
+    "rps_profile",
     "rps_profile_read", "rps_launch_count", "rps_last_error", "rps_version", "rps_step_static",
 )
 
@@ -80,6 +81,8 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         "rps_read": (cint, [vp, vp]),
         "rps_read_masks": (cint, [vp, u64, u64p, u64p, i32p, i32p]),
         "rps_diag": (cint, [vp, dblp, dblp]),
+        "rps_track": (cint, [vp, vp, i64]),
+        "rps_read_trace": (cint, [vp, vp, i64, i64p]),
         "rps_profile": (cint, [vp, cint]),
         "rps_profile_read": (cint, [vp, dblp, i64p, dblp, i64p]),
         "rps_launch_count": (i64, [vp]),
@@ -234,6 +237,24 @@ class RPS:
         a, c = ctypes.c_double(), ctypes.c_double()
         self._check(self._lib.rps_diag(self._h, ctypes.byref(a), ctypes.byref(c)), "rps_diag")
         return a.value, c.value
+
+    def track(self, capacity: int) -> None:
+        """Records {dist2_to_opt, consensus} of the state each of the next `capacity` steps leaves behind, as a
+        by-product of the fused pass (rps_track); 0 switches tracking off."""
+        self.trace_dev = torch.zeros((capacity, 2), dtype=torch.float64, device=self.device) if capacity > 0 else None
+        ptr = self.trace_dev.data_ptr() if capacity > 0 else None
+        with torch.cuda.device(self.device):
+            self._check(self._lib.rps_track(self._h, ptr, capacity), "rps_track")
+
+    def read_trace(self) -> np.ndarray:
+        """The recorded pairs so far as a float64 array [steps][2] (synchronises)."""
+        held = getattr(self, "trace_dev", None)
+        out = np.zeros((held.shape[0] if held is not None else 1, 2), dtype=np.float64)
+        count = ctypes.c_int64()
+        with torch.cuda.device(self.device):
+            self._check(self._lib.rps_read_trace(self._h, out.ctypes.data, out.shape[0], ctypes.byref(count)),
+                        "rps_read_trace")
+        return out[:count.value]
 
     def profile(self, enable: bool) -> None:
         self._check(self._lib.rps_profile(self._h, int(enable)), "rps_profile")

@@ -63,6 +63,10 @@ struct rps_handle {
     double ms[2] = {0.0, 0.0};
     int64_t timed[2] = {0, 0};
     rps::StepMasks staged{};  // host copy of caller-given masks
+    // tracked steps (rps_track)
+    double* trace = nullptr;
+    int64_t trace_capacity = 0;
+    int64_t trace_used = 0;
     std::string error;
 
     size_t elem() const { return opt.dtype == RPS_BF16 ? 2 : 4; }
@@ -182,12 +186,18 @@ int run_fused(rps_handle* h, const rps::StepMasks* masks)
     prm.narrow = h->d < ((int64_t)1 << 31);
     prm.error = h->error_word();
     prm.average_gradients = h->opt.average == RPS_AVERAGE_GRADIENTS;
+    prm.inv_n = 1.0f / (float)h->n;
+    const bool tracked = h->trace != nullptr && h->trace_used < h->trace_capacity;
+    prm.trace = tracked ? h->trace + 2 * h->trace_used : nullptr;
     rps::set_sgd_scalars(prm, h->gamma, h->sigma);
     prm.t_lo = (uint32_t)h->t;
     prm.t_hi = (uint32_t)(h->t >> 32);
     rps::set_philox_key(prm, h->seed);
     int rc = timed_launch(h, 0, [&] { return rps::launch_fused(prm, h->tuning(), h->opt.dtype == RPS_BF16, h->sm_count, h->stream); });
-    if (rc == RPS_OK) h->t += 1;
+    if (rc == RPS_OK) {
+        h->t += 1;
+        if (tracked) h->trace_used += 1;
+    }
     return rc;
 }
 
@@ -500,6 +510,39 @@ int rps_diag(rps_handle* h, double* dist2_to_opt, double* consensus)
     RPS_CUDA(h, cudaStreamSynchronize(h->stream));
     if (dist2_to_opt) *dist2_to_opt = host[0];
     if (consensus) *consensus = host[1];
+    return RPS_OK;
+}
+
+int rps_track(rps_handle* h, double* trace_dev, int64_t capacity)
+{
+    int rc = need_bound(h);
+    if (rc != RPS_OK) return rc;
+    if (capacity < 0) return fail(h, RPS_EINVAL, "capacity is negative");
+    if (capacity > ((int64_t)1 << 40)) return fail(h, RPS_EINVAL, "capacity is larger than 2^40 steps");
+    if ((uintptr_t)trace_dev % 16 != 0) return fail(h, RPS_EINVAL, "trace_dev must be 16-byte aligned");
+    h->trace = nullptr;
+    h->trace_capacity = 0;
+    h->trace_used = 0;
+    if (trace_dev == nullptr || capacity == 0) return RPS_OK;
+    RPS_CUDA(h, cudaMemsetAsync(trace_dev, 0, (size_t)capacity * 2 * sizeof(double), h->stream));
+    h->trace = trace_dev;
+    h->trace_capacity = capacity;
+    return RPS_OK;
+}
+
+int rps_read_trace(rps_handle* h, double* trace_host_out, int64_t max_entries, int64_t* entries)
+{
+    int rc = need_bound(h);
+    if (rc != RPS_OK) return rc;
+    if (h->trace == nullptr) return fail(h, RPS_ESTATE, "tracking is off (rps_track)");
+    if (!trace_host_out || !entries || max_entries < 0) return fail(h, RPS_EINVAL, "bad output arguments");
+    const int64_t count = h->trace_used < max_entries ? h->trace_used : max_entries;
+    if (count > 0)
+        RPS_CUDA(h, cudaMemcpyAsync(trace_host_out, h->trace, (size_t)count * 2 * sizeof(double),
+                                    cudaMemcpyDeviceToHost, h->stream));
+    rc = finish(h);
+    if (rc != RPS_OK) return rc;
+    *entries = count;
     return RPS_OK;
 }
 

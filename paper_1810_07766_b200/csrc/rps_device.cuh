@@ -335,4 +335,101 @@ __device__ __forceinline__ void store_ragged(T* dst, const float (&vals)[VEC], u
         if ((live_bits >> e) & 1u) dst[e] = RowVec<T, VEC>::narrow(vals[e]);
 }
 
+// s = fma(v, v, s) where `take` is set (one predicated instruction, like add_if).
+__device__ __forceinline__ void add_square_if(float& s, float v, uint32_t take)
+{
+    asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p fma.rn.f32 %0, %1, %1, %0;\n\t}" : "+f"(s) : "f"(v), "r"(take));
+}
+
+// The values a lane is about to store, as they will read back: rounded to T and widened again
+// (nothing to do for fp32 replicas).
+template <typename T, int VEC>
+__device__ __forceinline__ void as_stored(float (&vals)[VEC])
+{
+    if (sizeof(T) != sizeof(float)) RowVec<T, VEC>::unpack(RowVec<T, VEC>::pack(vals), vals);
+}
+
+// By-product of a tracked step: what the step leaves behind, measured on the values that are in
+// registers anyway (no extra pass over x):
+//   dist2 = || mean_i x^(i) - mean_i b_i ||^2   squared distance of the averaged model to the optimum of
+//                                               the quadratic objective,
+//   cons  = sum_i || x^(i) - mean_k x^(k) ||^2  the consensus error (the quantity Lemma 3 bounds).
+// Per column, relative to the pivot a = worker 0's new value (so that nothing large is squared and
+// subtracted):  D = sum_i (x_i - a),  Q = sum_i (x_i - a)^2;  mean x = a + D/n;  cons = Q - D^2/n.
+// fp32 within a tile of columns, fp64 across tiles.  All lanes of a warp call targets() and models()
+// together; `present` has bit w set iff worker w_first + w exists.
+template <int VEC, int WPT, int G>
+struct Tracker {
+    double dist2 = 0.0, cons = 0.0;
+    float bsum[VEC];  // this lane's part of sum_i b_i of the tile in flight
+
+    static __device__ __forceinline__ uint32_t present_workers(int w_first, int n)
+    {
+        const int left = n - w_first;
+        return left >= WPT ? (1u << WPT) - 1u : (left > 0 ? (1u << left) - 1u : 0u);
+    }
+
+    __device__ __forceinline__ void targets(const float (&bv)[WPT][VEC], uint32_t present)
+    {
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) bsum[e] = 0.0f;
+#pragma unroll
+        for (int w = 0; w < WPT; ++w)
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) add_if(bsum[e], bv[w][e], (present >> w) & 1u);
+    }
+
+    // v: x_{t+1} of this lane's workers and columns as stored; live_bits: which of the VEC columns exist
+    __device__ __forceinline__ void models(const float (&v)[WPT][VEC], uint32_t present, uint32_t live_bits, float inv_n)
+    {
+        constexpr int LPG = 32 / G;
+        const int lane = threadIdx.x & 31;
+        const bool first_group = lane < LPG;  // holds worker 0; speaks for the column
+        float q = 0.0f, dd = 0.0f;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            const uint32_t live = (live_bits >> e) & 1u;
+            const float a = __shfl_sync(0xFFFFFFFFu, v[0][e], lane & (LPG - 1));
+            float dsum = 0.0f;
+#pragma unroll
+            for (int w = 0; w < WPT; ++w) {
+                const uint32_t take = (present >> w) & live;
+                const float dev = v[w][e] - a;
+                add_if(dsum, dev, take);
+                add_square_if(q, dev, take);
+            }
+            dsum = sum_over_groups<G>(dsum);
+            const float btot = sum_over_groups<G>(bsum[e]);
+            if (first_group && live) {
+                const float gap = fmaf(dsum - btot, inv_n, a);  // mean x - mean b of this column
+                dd = fmaf(gap, gap, dd);
+                q = fmaf(-dsum * inv_n, dsum, q);
+            }
+        }
+        dist2 += (double)dd;
+        cons += (double)q;
+    }
+
+    // Adds this warp's sums to the CTA's pair in shared memory (zeroed before the first call); the
+    // last of `warps` warps to arrive adds the CTA's pair to out[0], out[1].  Nobody waits for anybody.
+    __device__ __forceinline__ void flush(double* cta_pair, int* cta_arrivals, int warps, double* out)
+    {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            dist2 += __shfl_xor_sync(0xFFFFFFFFu, dist2, off);
+            cons += __shfl_xor_sync(0xFFFFFFFFu, cons, off);
+        }
+        if ((threadIdx.x & 31) == 0) {
+            atomicAdd(&cta_pair[0], dist2);
+            atomicAdd(&cta_pair[1], cons);
+            __threadfence_block();
+            if (atomicAdd(cta_arrivals, 1) == warps - 1) {
+                __threadfence_block();
+                atomicAdd(&out[0], *reinterpret_cast<volatile double*>(&cta_pair[0]));
+                atomicAdd(&out[1], *reinterpret_cast<volatile double*>(&cta_pair[1]));
+            }
+        }
+    }
+};
+
 }  // namespace rps

@@ -38,6 +38,7 @@ struct FusedParams {
     const void* b;  // [n][pitch] targets of the quadratic objective
     const StepMasks* masks;
     int32_t* error;      // device word set non-zero when a bounded wait gave up (may be NULL)
+    double* trace;       // tracked step: [2] sums this launch adds to (see Tracker), zeroed beforehand; else NULL
     int64_t pitch;       // row pitch in elements
     int64_t d;           // model size
     int64_t block_cols;  // ceil(d / n): columns per parameter-server block
@@ -49,6 +50,7 @@ struct FusedParams {
     float noise_scale;  // -2 ln 2 * (gamma * sigma)^2
     int32_t noisy;      // sigma != 0
     int32_t average_gradients;  // 1: the updates -gamma*g are averaged and applied to x (Section 5's comparison)
+    float inv_n;                // 1 / n
     uint32_t t_lo, t_hi;
     uint32_t key0, key1;
     uint32_t round_key[10][2];  // Philox round keys: key + r * (0x9E3779B9, 0xBB67AE85)
@@ -76,6 +78,14 @@ cudaError_t launch_fused_direct(const FusedParams& prm, const FusedTuning& tune,
                                 cudaStream_t stream);
 cudaError_t launch_fused_staged(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
                                 cudaStream_t stream);
+// The optional forms of the fused step, built in one family of lane shapes, each group in a
+// translation unit of its own: gradient averaging (prm.average_gradients) and tracked steps
+// (prm.trace != NULL, with either kind of averaging).
+cudaError_t launch_staged_gradavg(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
+                                  cudaStream_t stream);
+cudaError_t launch_staged_tracked(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
+                                  cudaStream_t stream);
+cudaError_t launch_direct_tracked(const FusedParams& prm, bool bf16, int sm_count, cudaStream_t stream);
 cudaError_t launch_diag(const DiagParams& prm, bool bf16, int sm_count, cudaStream_t stream);
 
 }  // namespace rps

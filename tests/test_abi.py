@@ -75,6 +75,9 @@ def test_options_pitch_and_state_errors(lib):
         assert lib.rps_step(h) == -2
         assert lib.rps_step_n(h, 3) == -2
         assert lib.rps_read(h, None) == -2
+        assert lib.rps_track(h, None, 4) == -2
+        count = ctypes.c_int64()
+        assert lib.rps_read_trace(h, None, 0, ctypes.byref(count)) == -2
         assert b"rps_bind" in lib.rps_last_error(h)
         assert lib.rps_bind(h, None, None, 0, None, 0, None) == -1
         t = ctypes.c_uint64()
