@@ -6,6 +6,7 @@ this package.  It never imports the CUDA package and shares no code with it.
 from .rps_oracle import (  # noqa: F401
     ASSIGN_FIXED,
     ASSIGN_PERM,
+    alpha_mc,
     bf16_to_double,
     block_size,
     build,

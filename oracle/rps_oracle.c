@@ -23,6 +23,9 @@
  *                        (Assumption 1), so its exact values are a convention of
  *                        this build: parity unpinned by the paper for that part
  *   bf16 rounding        library conversion on random inputs
+ *   alpha_mc             exact alpha_1, alpha_2 from all drop patterns on tiny n (within the
+ *                        sampling error), 0 and 1 at p = 0 and p = 1, a second route to the
+ *                        same per-sample value through counts of arrivals and receivers
  */
 #define _GNU_SOURCE
 #include <math.h>
@@ -444,5 +447,77 @@ int rps_oracle_run_gradavg(int n, int64_t d, int dtype, void* x, const void* b, 
                                          self_delivery, assign, NULL, NULL);
         if (rc != 0) return rc;
     }
+    return 0;
+}
+
+/*
+ * Monte-Carlo estimate of the constants alpha_1 and alpha_2 of Eqs. (4) and (5),
+ *   E[W W^T]     = alpha_1 I + (1 - alpha_1) A_n,     E[W A_n W^T] = alpha_2 I + (1 - alpha_2) A_n,
+ * with A_n = 1 1^T / n and W = W_t^(j) the matrix of Eq. (3): X_{t+1}^(j) = V_t^(j) W_t^(j), column k
+ * of W holding the weights with which worker k's new block j mixes the workers' v.  A matrix of
+ * the form a I + (1 - a) A_n has a = (its diagonal entry) - (its off-diagonal entry), so each
+ * sampled W contributes mean(diag M) - mean(offdiag M) for M = W W^T and M = W A_n W^T, and the
+ * estimate is the mean over the n blocks of `steps` consecutive steps from t0.  Every matrix is
+ * formed entry by entry and multiplied out with plain loops.  Needs n >= 2.
+ */
+int rps_oracle_alpha_mc(int n, double p, uint64_t seed, uint64_t t0, int64_t steps, int self_delivery, int assign,
+                        double* alpha1, double* alpha2)
+{
+    if (n < 2 || n > 64 || steps < 1) return -1;
+    uint64_t up[64], down[64];
+    int32_t cnt[64], server[64];
+    double* w = (double*)malloc(sizeof(double) * n * n * 4);
+    if (!w) return -2;
+    double* wa = w + n * n;   /* W A_n        */
+    double* m1 = wa + n * n;  /* W W^T        */
+    double* m2 = m1 + n * n;  /* W A_n W^T    */
+    double sum1 = 0.0, sum2 = 0.0;
+    for (int64_t s = 0; s < steps; ++s) {
+        if (rps_oracle_masks(n, p, seed, t0 + (uint64_t)s, self_delivery, assign, up, down, cnt, server) != 0) {
+            free(w);
+            return -1;
+        }
+        for (int j = 0; j < n; ++j) {
+            /* W[m][k]: weight of v^(m) in x_{t+1}^(k) for block j */
+            for (int m = 0; m < n; ++m)
+                for (int k = 0; k < n; ++k) {
+                    const int received = (int)((down[j] >> k) & 1u);
+                    const int arrived = (int)((up[j] >> m) & 1u);
+                    w[m * n + k] = received ? (arrived ? 1.0 / cnt[j] : 0.0) : (m == k ? 1.0 : 0.0);
+                }
+            for (int m = 0; m < n; ++m)
+                for (int k = 0; k < n; ++k) {
+                    double acc = 0.0;
+                    for (int l = 0; l < n; ++l) acc += w[m * n + l] * (1.0 / n);
+                    wa[m * n + k] = acc;
+                }
+            for (int m = 0; m < n; ++m)
+                for (int k = 0; k < n; ++k) {
+                    double a1 = 0.0, a2 = 0.0;
+                    for (int l = 0; l < n; ++l) {
+                        a1 += w[m * n + l] * w[k * n + l];
+                        a2 += wa[m * n + l] * w[k * n + l];
+                    }
+                    m1[m * n + k] = a1;
+                    m2[m * n + k] = a2;
+                }
+            double d1 = 0.0, o1 = 0.0, d2 = 0.0, o2 = 0.0;
+            for (int m = 0; m < n; ++m)
+                for (int k = 0; k < n; ++k) {
+                    if (m == k) {
+                        d1 += m1[m * n + k];
+                        d2 += m2[m * n + k];
+                    } else {
+                        o1 += m1[m * n + k];
+                        o2 += m2[m * n + k];
+                    }
+                }
+            sum1 += d1 / n - o1 / ((double)n * (n - 1));
+            sum2 += d2 / n - o2 / ((double)n * (n - 1));
+        }
+    }
+    free(w);
+    *alpha1 = sum1 / ((double)steps * n);
+    *alpha2 = sum2 / ((double)steps * n);
     return 0;
 }

@@ -80,6 +80,9 @@ def _load():
     lib.rps_oracle_step_columns.restype = ctypes.c_int
     lib.rps_oracle_diag.argtypes = [ctypes.c_int, ctypes.c_int64, ctypes.c_int, vp, vp, f64p, f64p]
     lib.rps_oracle_diag.restype = ctypes.c_int
+    lib.rps_oracle_alpha_mc.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_uint64, ctypes.c_uint64,
+                                        ctypes.c_int64, ctypes.c_int, ctypes.c_int, f64p, f64p]
+    lib.rps_oracle_alpha_mc.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -201,3 +204,15 @@ def diag(x: np.ndarray, b: np.ndarray, *, dtype: str) -> Tuple[float, float]:
     c = ctypes.c_double()
     _load().rps_oracle_diag(n, d, _DTYPE[dtype], x.ctypes.data, b.ctypes.data, ctypes.byref(a), ctypes.byref(c))
     return a.value, c.value
+
+
+def alpha_mc(n: int, p: float, seed: int, t0: int, steps: int, self_delivery: bool = True,
+             assign: int = ASSIGN_FIXED) -> Tuple[float, float]:
+    """Monte-Carlo (alpha_1, alpha_2) of Eqs. (4), (5) over the n blocks of ``steps`` steps from ``t0``."""
+    a1 = ctypes.c_double()
+    a2 = ctypes.c_double()
+    rc = _load().rps_oracle_alpha_mc(n, p, seed, t0, steps, int(self_delivery), assign, ctypes.byref(a1),
+                                     ctypes.byref(a2))
+    if rc != 0:
+        raise ValueError("rps_oracle_alpha_mc rejected its arguments")
+    return a1.value, a2.value
