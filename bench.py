@@ -31,19 +31,25 @@ UNIT = "replica-params/s"
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one fused-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) from
-# the ncu capture summarised under profiles/, keyed by workload; valid only for the kernel
-# sources whose digest is recorded with it.
+# the ncu captures summarised under profiles/, keyed by workload; valid only for the kernel
+# sources whose digest is recorded with it.  "bytes_per_launch": mean of 10 consecutive launches
+# of this benchmark at full size with the caches left as the launch before left them (one-pass
+# capture), which is the state the timed steps run in: a step starts on the columns that the step
+# before it touched last, so part of x and b is still in L2 and the traffic is below the
+# algorithmic bytes.  "cold_bytes_per_launch": one launch alone with the caches flushed first
+# (cfg3 and cfg5 from captures at d/4 and d/8, scaled by 4 and 8).
 NCU_TRAFFIC = {
-    "kernel_digest": "ab25329539aedc19",
-    # cfg3 and cfg5 come from captures at d/4 and d/8, scaled (traffic is proportional to d)
-    "bytes_per_launch": {"cfg2": 1023694080, "cfg3": 4727221248, "cfg4": 1488895128, "cfg5": 6058887168},
+    "kernel_digest": "3be8d0ef4408324f",
+    "bytes_per_launch": {"cfg2": 964367104, "cfg3": 4810349773, "cfg4": 1433042816, "cfg5": 6385079219},
+    "cold_bytes_per_launch": {"cfg2": 1022745856, "cfg3": 4713916416, "cfg4": 1490735016, "cfg5": 6073657344},
 }
 
 
 def kernel_digest() -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_1810_07766_b200", "csrc")
-    for name in ("rps_device.cuh", "rps_direct.cuh", "rps_kernels.cu", "rps_staged.cuh", "rps_staged.cu"):
+    # the fused kernels, their arithmetic and the choice of the default shape
+    for name in ("rps_device.cuh", "rps_direct.cuh", "rps_staged.cuh", "rps_staged.cu"):
         with open(os.path.join(csrc, name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -229,7 +235,7 @@ def run_cuda(args):
         w = w.scaled(d=args.d)
     b = wl.make_targets(w)
     r = binding.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma, kernel=args.kernel,
-                    workers_per_lane=args.workers_per_lane, stages=args.stages, consumer_warps=args.consumer_warps, copy_mode=args.copy_mode, slice_bytes=args.slice_bytes, store_mode=args.store_mode, average_gradients=args.average_gradients)
+                    workers_per_lane=args.workers_per_lane, stages=args.stages, consumer_warps=args.consumer_warps, copy_mode=args.copy_mode, slice_bytes=args.slice_bytes, store_mode=args.store_mode, average_gradients=args.average_gradients, traversal=args.traversal, l2_policy=args.l2_policy)
     r.set_targets(b)
     if args.track:
         # every step of the run also records the distance to the optimum and the consensus error
@@ -237,19 +243,21 @@ def run_cuda(args):
     stream = r.stream
     bytes_per_step = w.bytes_per_step
 
-    # pass 1 (untimed for `value`): every launch bracketed by events -> per-kernel durations
-    r.step_n(max(args.warmup, 3))
-    r.profile(True)
-    r.step_n(args.steps)
-    fused_ms, fused_n, mask_ms, mask_n = r.profile_read()
-    r.profile(False)
-
-    # pass 2: W warm-up steps, then exactly K timed steps
-    r.step_n(args.warmup)
-    launches_before = r.launch_count()
+    # the clocks are sampled from here to the end of the timed steps: an NVML query takes milliseconds, so
+    # the timed region alone (tens of milliseconds) would yield a single sample
     with ClockSampler(local_rank) as clocks:
+        # pass 1 (untimed for `value`): every launch bracketed by events -> per-kernel durations
+        r.step_n(max(args.warmup, 3))
+        r.profile(True)
+        r.step_n(args.steps)
+        fused_ms, fused_n, mask_ms, mask_n = r.profile_read()
+        r.profile(False)
+
+        # pass 2: W warm-up steps, then exactly K timed steps
+        r.step_n(args.warmup)
+        launches_before = r.launch_count()
         total_ms = timed_steps(torch, stream, lambda: r.step_n(args.steps), device)
-    gpu_launches = r.launch_count() - launches_before
+        gpu_launches = r.launch_count() - launches_before
 
     # pass 3: end to end through the host-buffer call: H2D of x and b, the step, D2H of x, every step
     e2e = None
@@ -272,11 +280,12 @@ def run_cuda(args):
     peak, peak_kind = measured_peak_gbs()
     fused_avg_ms = fused_ms / max(fused_n, 1)
     achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
-    traffic = None
+    traffic = traffic_cold = None
     default_shape = not (args.kernel or args.workers_per_lane or args.stages or args.consumer_warps or args.copy_mode or args.slice_bytes or args.store_mode
-                         or args.average_gradients or args.track)
+                         or args.average_gradients or args.track or args.traversal or args.l2_policy)
     if default_shape and NCU_TRAFFIC["kernel_digest"] == kernel_digest():
         traffic = NCU_TRAFFIC["bytes_per_launch"].get(w.name)
+        traffic_cold = NCU_TRAFFIC["cold_bytes_per_launch"].get(w.name)
 
     line = {
         "metric": METRIC, "value": world * w.n * w.d * args.steps / (total_ms * 1e-3), "unit": UNIT,
@@ -287,7 +296,8 @@ def run_cuda(args):
                         f"seed={w.seed}; quadratic objective, b_i ~ N({'mu_i' if w.hetero else '0'},1)",
             "n": w.n, "d": w.d, "p": w.p, "replicas": "one independent job per GPU, no collective",
             "kernel_shape": {"kernel": args.kernel, "workers_per_lane": args.workers_per_lane, "stages": args.stages,
-                             "consumer_warps": args.consumer_warps, "copy_mode": args.copy_mode, "slice_bytes": args.slice_bytes, "store_mode": args.store_mode},
+                             "consumer_warps": args.consumer_warps, "copy_mode": args.copy_mode, "slice_bytes": args.slice_bytes, "store_mode": args.store_mode,
+                             "traversal": args.traversal, "l2_policy": args.l2_policy},
             "average": "gradients" if args.average_gradients else "models",
             "tracked": bool(args.track),
             "l2": "inputs larger than L2 (x and b are %.0f MB each)" % (row_bytes / 1e6),
@@ -299,7 +309,7 @@ def run_cuda(args):
         "e2e": e2e,
         "gpu_launches": gpu_launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": fused_kernel_name(args, w),
+                     "traffic": traffic, "traffic_cold_cache": traffic_cold, "peak_kind": f"of {peak_kind}", "kernel": fused_kernel_name(args, w),
                      "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n,
                      "mask_kernel_ms_per_launch": mask_ms / max(mask_n, 1), "mask_launches_timed": mask_n,
                      "in_situ_copy_gbs": copy_gbs, "frac_of_in_situ_copy": achieved / copy_gbs},
@@ -384,6 +394,9 @@ def main(argv=None):
     ap.add_argument("--slice-bytes", type=int, default=0, help="staged kernel, bf16: 16 or 8 bytes per lane and row")
     ap.add_argument("--average-gradients", action="store_true",
                     help="time the gradient-averaging comparison of Section 5 instead of RPS (model averaging)")
+    ap.add_argument("--traversal", type=int, default=0,
+                    help="0: odd steps walk the columns downwards (default); 1: every step upwards")
+    ap.add_argument("--l2-policy", type=int, default=0, help="staged kernel: 1 plain loads, 2 targets evict-first")
     ap.add_argument("--track", action="store_true",
                     help="time tracked steps: distance to the optimum and consensus error as a by-product of the pass")
     ap.add_argument("--store-mode", type=int, default=0, help="staged kernel: 1 register stores, 2 TMA stores")

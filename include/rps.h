@@ -107,6 +107,14 @@ typedef struct rps_options {
                                  issues no copies, so the compute warps' waits run out, x is
                                  left unchanged and the error is reported; 0 otherwise       */
     int32_t average;          /* rps_average, default RPS_AVERAGE_MODELS                        */
+    /* How consecutive steps share the L2 cache; neither changes any result. */
+    int32_t traversal;        /* 0 (default): even steps walk the columns upwards, odd steps
+                                 downwards, so a step starts on the part of x and b that the step
+                                 before it touched last and that is still in L2; 1: always upwards */
+    int32_t l2_policy;        /* kernel 2: 1 = plain loads; 2 = the targets b are loaded with the
+                                 L2 evict-first hint, which leaves the cache to the lines of x
+                                 (a retained line of x saves a read and a write-back, one of b
+                                 only a read); 0 = the library's choice                        */
 } rps_options;
 
 /*
@@ -215,6 +223,18 @@ int rps_read_masks(rps_handle* h, uint64_t t, uint64_t* up, uint64_t* down, int3
  * Synchronises.  Either output may be NULL.
  */
 int rps_diag(rps_handle* h, double* dist2_to_opt, double* consensus);
+
+/*
+ * rps_estimate_alpha: Monte-Carlo estimate of the constants of Eqs. (4) and (5),
+ *   E[W W^T] = alpha_1 I + (1 - alpha_1) A_n,   E[W A_n W^T] = alpha_2 I + (1 - alpha_2) A_n,
+ * (W = W_t^(j) of Eq. 3, A_n = 1 1^T / n), which Figures 2 and 3 plot and whose difference beta
+ * sets the rate of Theorem 1.  Runs the mask generator for steps t0 .. t0+steps-1 of this handle's
+ * streams (n, p, seed, assign, self_delivery) and averages, over the n blocks of every step, the
+ * value (mean diagonal) - (mean off-diagonal) of W W^T and of W A_n W^T, computed on the device from
+ * the counts of arrivals and receivers.  Does not touch x, b or the step counter.  Synchronises.
+ * RPS_EINVAL for n < 2 (no off-diagonal entries) or steps < 1.
+ */
+int rps_estimate_alpha(rps_handle* h, uint64_t t0, int64_t steps, double* alpha1, double* alpha2);
 
 /*
  * rps_track: the same two quantities as rps_diag, as a by-product of the fused pass itself (no extra

@@ -26,7 +26,8 @@ _DTYPE = {"f32": RPS_F32, "bf16": RPS_BF16}
 SYMBOLS = (
     "rps_create", "rps_destroy", "rps_default_options", "rps_configure", "rps_pitch", "rps_scratch_bytes",
     "rps_bind", "rps_set_targets", "rps_write", "rps_set_step", "rps_get_step", "rps_step", "rps_step_n",
-    "rps_step_forced", "rps_step_host", "rps_read", "rps_read_masks", "rps_diag", "rps_track", "rps_read_trace",
+    "rps_step_forced", "rps_step_host", "rps_read", "rps_read_masks", "rps_diag", "rps_estimate_alpha", "rps_track",
+    "rps_read_trace",
     "rps_profile",
     "rps_profile_read", "rps_launch_count", "rps_last_error", "rps_version", "rps_step_static",
 )
@@ -39,7 +40,8 @@ class rps_options(ctypes.Structure):
                 ("workers_per_lane", ctypes.c_int32), ("stages", ctypes.c_int32), ("consumer_warps", ctypes.c_int32),
                 ("copy_mode", ctypes.c_int32), ("slice_bytes", ctypes.c_int32),
                 ("store_mode", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32),
-                ("withhold_copies", ctypes.c_int32), ("average", ctypes.c_int32)]
+                ("withhold_copies", ctypes.c_int32), ("average", ctypes.c_int32),
+                ("traversal", ctypes.c_int32), ("l2_policy", ctypes.c_int32)]
 
 
 class RPSError(RuntimeError):
@@ -81,6 +83,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         "rps_read": (cint, [vp, vp]),
         "rps_read_masks": (cint, [vp, u64, u64p, u64p, i32p, i32p]),
         "rps_diag": (cint, [vp, dblp, dblp]),
+        "rps_estimate_alpha": (cint, [vp, u64, i64, dblp, dblp]),
         "rps_track": (cint, [vp, vp, i64]),
         "rps_read_trace": (cint, [vp, vp, i64, i64p]),
         "rps_profile": (cint, [vp, cint]),
@@ -117,7 +120,7 @@ class RPS:
     def __init__(self, n: int, d: int, p: float, gamma: float, seed: int, *, dtype: str = "f32", sigma: float = 0.0,
                  assign: int = RPS_ASSIGN_FIXED, self_delivery: bool = True, mask_window: int = 32,
                  kernel: int = 0, workers_per_lane: int = 0, stages: int = 0, consumer_warps: int = 0,
-                 row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0, wait_limit_ms: int = 0, withhold_copies: bool = False, average_gradients: bool = False, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+                 row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0, wait_limit_ms: int = 0, withhold_copies: bool = False, average_gradients: bool = False, traversal: int = 0, l2_policy: int = 0, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         if not torch.cuda.is_available():
@@ -134,6 +137,7 @@ class RPS:
         opt.row_skew_lines, opt.copy_mode, opt.slice_bytes = row_skew_lines, copy_mode, slice_bytes
         opt.store_mode, opt.wait_limit_ms, opt.withhold_copies = store_mode, wait_limit_ms, int(withhold_copies)
         opt.average = int(average_gradients)
+        opt.traversal, opt.l2_policy = traversal, l2_policy
         self._check(self._lib.rps_configure(self._h, ctypes.byref(opt)), "rps_configure")
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
         self.pitch = int(self._lib.rps_pitch(self._h))
@@ -237,6 +241,13 @@ class RPS:
         a, c = ctypes.c_double(), ctypes.c_double()
         self._check(self._lib.rps_diag(self._h, ctypes.byref(a), ctypes.byref(c)), "rps_diag")
         return a.value, c.value
+
+    def estimate_alpha(self, t0: int, steps: int) -> Tuple[float, float]:
+        """Monte-Carlo (alpha_1, alpha_2) of Eqs. (4), (5) from the drop masks of ``steps`` steps from ``t0``."""
+        a1, a2 = ctypes.c_double(), ctypes.c_double()
+        self._check(self._lib.rps_estimate_alpha(self._h, t0, steps, ctypes.byref(a1), ctypes.byref(a2)),
+                    "rps_estimate_alpha")
+        return a1.value, a2.value
 
     def track(self, capacity: int) -> None:
         """Records {dist2_to_opt, consensus} of the state each of the next `capacity` steps leaves behind, as a

@@ -81,7 +81,7 @@ struct rps_handle {
     rps::FusedTuning tuning() const
     {
         return rps::FusedTuning{opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps, opt.copy_mode, opt.slice_bytes, opt.store_mode,
-                                 opt.wait_limit_ms, opt.withhold_copies};
+                                 opt.wait_limit_ms, opt.withhold_copies, opt.traversal, opt.l2_policy};
     }
     rps::StepMasks* window() const { return reinterpret_cast<rps::StepMasks*>(scratch + kDiagBytes); }
     rps::StepMasks* probe() const { return window() + opt.mask_window; }
@@ -187,6 +187,7 @@ int run_fused(rps_handle* h, const rps::StepMasks* masks)
     prm.error = h->error_word();
     prm.average_gradients = h->opt.average == RPS_AVERAGE_GRADIENTS;
     prm.inv_n = 1.0f / (float)h->n;
+    prm.descending = h->opt.traversal == 0 && (h->t & 1u) != 0;
     const bool tracked = h->trace != nullptr && h->trace_used < h->trace_capacity;
     prm.trace = tracked ? h->trace + 2 * h->trace_used : nullptr;
     rps::set_sgd_scalars(prm, h->gamma, h->sigma);
@@ -263,6 +264,8 @@ int rps_default_options(rps_options* opt)
     opt->wait_limit_ms = 0;
     opt->withhold_copies = 0;
     opt->average = RPS_AVERAGE_MODELS;
+    opt->traversal = 0;
+    opt->l2_policy = 0;
     return RPS_OK;
 }
 
@@ -344,6 +347,8 @@ int rps_configure(rps_handle* h, const rps_options* opt)
         return fail(h, RPS_EINVAL, "withhold_copies must be 0 or 1");
     if (opt->store_mode < 0 || opt->store_mode > 3) return fail(h, RPS_EINVAL, "store_mode must be 0 (auto) or 1..3");
     if (opt->copy_mode < 0 || opt->copy_mode > 2) return fail(h, RPS_EINVAL, "copy_mode must be 0 (auto), 1 or 2");
+    if (opt->traversal != 0 && opt->traversal != 1) return fail(h, RPS_EINVAL, "traversal must be 0 or 1");
+    if (opt->l2_policy < 0 || opt->l2_policy > 2) return fail(h, RPS_EINVAL, "l2_policy must be 0 (auto), 1 or 2");
     h->opt = *opt;
     h->sigma = (float)opt->sigma;
     return RPS_OK;
@@ -510,6 +515,33 @@ int rps_diag(rps_handle* h, double* dist2_to_opt, double* consensus)
     RPS_CUDA(h, cudaStreamSynchronize(h->stream));
     if (dist2_to_opt) *dist2_to_opt = host[0];
     if (consensus) *consensus = host[1];
+    return RPS_OK;
+}
+
+int rps_estimate_alpha(rps_handle* h, uint64_t t0, int64_t steps, double* alpha1, double* alpha2)
+{
+    int rc = need_bound(h);
+    if (rc != RPS_OK) return rc;
+    if (h->n < 2) return fail(h, RPS_EINVAL, "alpha needs at least 2 workers");
+    if (steps < 1 || !alpha1 || !alpha2) return fail(h, RPS_EINVAL, "steps must be positive and the outputs non-NULL");
+    RPS_CUDA(h, cudaMemsetAsync(h->diag_acc(), 0, 2 * sizeof(double), h->stream));
+    h->window_valid = false;  // the window of pre-generated masks is reused as sample storage
+    const int64_t window = h->opt.mask_window;
+    for (int64_t done = 0; done < steps; done += window) {
+        const int chunk = (int)(steps - done < window ? steps - done : window);
+        rc = generate_masks(h, h->window(), t0 + (uint64_t)done, chunk);
+        if (rc != RPS_OK) return rc;
+        rps::AlphaParams prm{h->window(), h->diag_acc(), h->n};
+        cudaError_t err = rps::launch_alpha(prm, chunk, h->stream);
+        if (err != cudaSuccess) return cuda_fail(h, "alpha kernel launch", err);
+        h->launches += 1;
+    }
+    double host[2] = {0.0, 0.0};
+    RPS_CUDA(h, cudaMemcpyAsync(host, h->diag_acc(), sizeof host, cudaMemcpyDeviceToHost, h->stream));
+    RPS_CUDA(h, cudaStreamSynchronize(h->stream));
+    const double samples = (double)steps * (double)h->n;
+    *alpha1 = host[0] / samples;
+    *alpha2 = host[1] / samples;
     return RPS_OK;
 }
 

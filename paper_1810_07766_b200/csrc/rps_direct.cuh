@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(THREADS) rps_fused_direct_kernel(const FusedPa
     }
     // odd steps take the tiles from the last to the first: a step starts on the columns that the step
     // before it touched last, which are still in L2
-    const bool descending = (prm.t_lo & 1u) != 0;
+    const bool descending = prm.descending != 0;
     for (int64_t turn = (int64_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5); turn < tiles;
          turn += warps_total) {
         const int64_t tile = descending ? tiles - 1 - turn : turn;

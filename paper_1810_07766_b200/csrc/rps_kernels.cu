@@ -126,8 +126,58 @@ __global__ void __launch_bounds__(256) rps_diag_kernel(const DiagParams prm)
 }
 
 // --------------------------------------------------------------------------
+// Monte-Carlo estimate of alpha_1 and alpha_2 (Eqs. 4 and 5) from generated drop masks.  For block j
+// of one step let N be the set of workers whose copy arrived (c of them) and R the number of workers
+// that receive the average.  Column k of W_t^(j) (Eq. 3) is the uniform average over N if k receives
+// and the unit vector e_k otherwise, hence
+//   (W W^T)[m][m']     = R [m in N][m' in N] / c^2 + [m = m'][m does not receive]
+//   (W A_n W^T)[m][m'] = s_m s_m' / n,   s_m = R [m in N] / c + [m does not receive]   (row sums of W).
+// Both matrices have all entries summing to n, so with their traces T the sample of
+// alpha = (mean diagonal) - (mean off-diagonal) is T/n - (n - T)/(n (n - 1)).  One CTA per step,
+// one thread per block; sums in fp64.
+// --------------------------------------------------------------------------
+__global__ void __launch_bounds__(kMaxWorkers) rps_alpha_kernel(const AlphaParams prm)
+{
+    const StepMasks* rec = prm.masks + blockIdx.x;
+    const int n = prm.n;
+    const int j = threadIdx.x;
+    double a1 = 0.0, a2 = 0.0;
+    if (j < n) {
+        const uint64_t up = rec->up[j], down = rec->down[j];
+        const int c = rec->cnt[j];
+        const int receivers = __popcll(down);
+        const double share = c > 0 ? (double)receivers / (double)c : 0.0;  // R / c; no average exists when c = 0
+        const double trace1 = share + (double)(n - receivers);
+        const int in_and_recv = __popcll(up & down);     // s = R/c
+        const int in_not_recv = __popcll(up & ~down);    // s = R/c + 1
+        const int out_not_recv = n - __popcll(up | down);  // s = 1 (outside N and receiving: s = 0)
+        const double trace2 =
+            ((double)in_and_recv * share * share + (double)in_not_recv * (share + 1.0) * (share + 1.0) +
+             (double)out_not_recv) / (double)n;
+        const double off = 1.0 / ((double)n * (double)(n - 1));
+        a1 = trace1 / n - ((double)n - trace1) * off;
+        a2 = trace2 / n - ((double)n - trace2) * off;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        a1 += __shfl_xor_sync(0xFFFFFFFFu, a1, o);
+        a2 += __shfl_xor_sync(0xFFFFFFFFu, a2, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicAdd(prm.out, a1);
+        atomicAdd(prm.out + 1, a2);
+    }
+}
+
+// --------------------------------------------------------------------------
 // Launch wrappers
 // --------------------------------------------------------------------------
+cudaError_t launch_alpha(const AlphaParams& prm, int steps, cudaStream_t stream)
+{
+    rps_alpha_kernel<<<steps, kMaxWorkers, 0, stream>>>(prm);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_masks(const MaskParams& prm, int steps, cudaStream_t stream)
 {
     rps_mask_kernel<<<steps, 256, 0, stream>>>(prm);

@@ -31,6 +31,8 @@ struct FusedTuning {
     int32_t store_mode;        // staged kernel: 1 stores from registers, 2 TMA stores from an output tile, 3 TMA stores in place
     int32_t wait_limit_ms;     // staged kernel: bound of every mbarrier wait (0 = 2000 ms)
     int32_t withhold_copies;   // staged kernel, test aid: issue no copies so that the bounded waits run out
+    int32_t traversal;         // 0 odd steps walk the tiles downwards, 1 always upwards
+    int32_t l2_policy;         // staged kernel: 1 plain loads, 2 targets loaded with the L2 evict-first hint
 };
 
 struct FusedParams {
@@ -50,6 +52,7 @@ struct FusedParams {
     float noise_scale;  // -2 ln 2 * (gamma * sigma)^2
     int32_t noisy;      // sigma != 0
     int32_t average_gradients;  // 1: the updates -gamma*g are averaged and applied to x (Section 5's comparison)
+    int32_t descending;         // 1: take the tiles from the last to the first (odd steps, see FusedTuning::traversal)
     float inv_n;                // 1 / n
     uint32_t t_lo, t_hi;
     uint32_t key0, key1;
@@ -71,6 +74,13 @@ struct DiagParams {
     int32_t n;
 };
 
+struct AlphaParams {
+    const StepMasks* masks;  // one record per step
+    double* out;             // [2] sums over all blocks of all records, added to
+    int32_t n;
+};
+
+cudaError_t launch_alpha(const AlphaParams& prm, int steps, cudaStream_t stream);
 cudaError_t launch_masks(const MaskParams& prm, int steps, cudaStream_t stream);
 cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
                          cudaStream_t stream);

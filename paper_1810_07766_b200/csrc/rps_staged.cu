@@ -11,9 +11,9 @@ cudaError_t launch_staged_for_n(const FusedParams& prm, const FusedTuning& tune,
 {
     const int n = prm.n;
     // workers per lane: asked for, or 8 where that halves the shuffle stages and pays for its
-    // registers (bf16 replicas, or more than 32 workers), else 4
+    // registers (bf16 replicas, or more than 8 workers), else 4
     int wpt = tune.workers_per_lane;
-    if (wpt == 0) wpt = (n > 4 && (sizeof(T) == 2 || n > 32)) ? 8 : 4;
+    if (wpt == 0) wpt = (n > 4 && (sizeof(T) == 2 || n > 8)) ? 8 : 4;
     if (wpt == 8) {
         if (n <= 8) return launch_staged_as<T, VEC, 8, 1>(prm, tune, sm_count, stream);
         if (n <= 16) return launch_staged_as<T, VEC, 8, 2>(prm, tune, sm_count, stream);

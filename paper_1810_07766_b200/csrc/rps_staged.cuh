@@ -45,6 +45,7 @@ constexpr uint32_t kSmemHeaderBytes = 128 + 2 * kMaxWorkers * 8 + kMaxWorkers * 
 constexpr uint32_t kAbortFlagOffset = kSmemHeaderBytes - 128;
 constexpr int kOutBuffers = 2;
 constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;
+constexpr int kDefaultL2Policy = 1;
 static_assert(kSmemHeaderBytes % 128 == 0, "tile data must start on a 128-byte boundary");
 
 struct StagedShape {
@@ -75,6 +76,7 @@ struct StagedShape {
     // 1: the tiles are taken from the last to the first.  Odd steps run this way, so that a step starts
     // on the columns the step before it touched last, which are still in L2 (and still dirty there).
     int32_t descending;
+    int32_t evict_first_targets;  // 1: b is loaded with the L2 evict-first hint
 
     __device__ __forceinline__ int64_t tile_of_turn(int64_t turn) const { return descending ? tiles - 1 - turn : turn; }
 };
@@ -151,6 +153,34 @@ __device__ __forceinline__ void bulk_load_row(uint32_t dst_smem, const void* src
                      dst_smem),
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
+}
+
+// The same two copies carrying an L2 cache policy (made by createpolicy).
+__device__ __forceinline__ void tma_load_box(uint32_t dst_smem, const CUtensorMap* map, int32_t column, int32_t row,
+                                             uint32_t bar, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, "
+        "%3}], [%4], %5;" ::"r"(dst_smem),
+        "l"(map), "r"(column), "r"(row), "r"(bar), "l"(policy)
+        : "memory");
+}
+
+__device__ __forceinline__ void bulk_load_row(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar,
+                                              uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+            dst_smem),
+        "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+        : "memory");
+}
+
+__device__ __forceinline__ uint64_t l2_evict_first_policy()
+{
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
 }
 
 // TMA tensor store shared -> global of one box; the unit clips what lies outside the tensor (columns >= d).
@@ -230,6 +260,7 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
         }
+        const uint64_t targets_policy = l2_evict_first_policy();
         int stage = 0;
         uint32_t phase = 0;
         int64_t issued = 0;
@@ -252,7 +283,11 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
                     for (int k = 0; k < shape.boxes_per_tile; ++k) {
                         const int32_t col = (int32_t)c0 + k * shape.box_cols;
                         tma_load_box(dst + (uint32_t)k * shape.box_bytes, &map_x, col, 0, bar);
-                        tma_load_box(dst + shape.array_bytes + (uint32_t)k * shape.box_bytes, &map_b, col, 0, bar);
+                        if (shape.evict_first_targets)
+                            tma_load_box(dst + shape.array_bytes + (uint32_t)k * shape.box_bytes, &map_b, col, 0, bar,
+                                         targets_policy);
+                        else
+                            tma_load_box(dst + shape.array_bytes + (uint32_t)k * shape.box_bytes, &map_b, col, 0, bar);
                     }
                 }
             } else {
@@ -265,7 +300,11 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
                 for (int i = lane; i < n; i += 32) {
                     const int64_t at = ((int64_t)i * prm.pitch + c0) * elem;
                     bulk_load_row(dst + (uint32_t)i * shape.row_bytes, x_bytes + at, bytes, bar);
-                    bulk_load_row(dst + shape.array_bytes + (uint32_t)i * shape.row_bytes, b_bytes + at, bytes, bar);
+                    if (shape.evict_first_targets)
+                        bulk_load_row(dst + shape.array_bytes + (uint32_t)i * shape.row_bytes, b_bytes + at, bytes, bar,
+                                      targets_policy);
+                    else
+                        bulk_load_row(dst + shape.array_bytes + (uint32_t)i * shape.row_bytes, b_bytes + at, bytes, bar);
                 }
             }
             ++issued;
@@ -524,7 +563,8 @@ bool shape_for(const FusedParams& prm, const FusedTuning& tune, int vec, int g, 
     sh.stages = stages;
     sh.wait_limit_ns = tune.wait_limit_ms > 0 ? (uint64_t)tune.wait_limit_ms * 1000000ull : kDefaultWaitLimitNs;
     sh.withhold_copies = tune.withhold_copies;
-    sh.descending = (int32_t)(prm.t_lo & 1u);
+    sh.descending = prm.descending;
+    sh.evict_first_targets = (tune.l2_policy != 0 ? tune.l2_policy : kDefaultL2Policy) == 2;
     sh.out_offset = (uint32_t)stages * sh.stage_bytes;
     out->threads = (warps + (store_mode == 3 ? 2 : 1)) * 32;
     out->smem_bytes = kSmemHeaderBytes + (uint32_t)stages * sh.stage_bytes + (uint32_t)out_total;

@@ -98,6 +98,8 @@ extern "C" int rps_step_static(int n, int64_t d, int dtype, void* x_dev, const v
     rps::set_sgd_scalars(fp, (float)gamma, (float)sigma);
     fp.t_lo = (uint32_t)t;
     fp.t_hi = (uint32_t)(t >> 32);
+    fp.descending = (int32_t)(t & 1u);  // as rps_step does: odd steps walk the columns downwards
+    fp.inv_n = 1.0f / (float)n;
     rps::set_philox_key(fp, seed);
     if (rps::launch_fused(fp, rps::FusedTuning{}, dtype == RPS_BF16, st->sm_count, stream) != cudaSuccess)
         return RPS_ECUDA;

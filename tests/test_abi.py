@@ -59,13 +59,15 @@ def test_options_pitch_and_state_errors(lib):
         assert (opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps) == (0, 0, 0, 0)
         assert opt.row_skew_lines == -1 and opt.copy_mode == 0 and opt.slice_bytes == 0 and opt.store_mode == 0
         assert opt.wait_limit_ms == 0 and opt.withhold_copies == 0 and opt.average == 0
+        assert opt.traversal == 0 and opt.l2_policy == 0
         assert lib.rps_scratch_bytes(h) == 256 + 34 * 1792
         opt.dtype = 1
         assert lib.rps_configure(h, ctypes.byref(opt)) == 0
         assert lib.rps_pitch(h) == 11_174_080                      # rounded up to 64 bf16, plus one skew line
         for field, value in (("dtype", 7), ("assign", 2), ("self_delivery", 3), ("mask_window", 0),
                              ("mask_window", 257), ("sigma", -1.0), ("kernel", 3), ("workers_per_lane", 3), ("stages", 1),
-                             ("stages", 9), ("consumer_warps", 25), ("slice_bytes", 4), ("store_mode", 4), ("wait_limit_ms", -1), ("withhold_copies", 2), ("average", 2), ("row_skew_lines", -2), ("copy_mode", 3)):
+                             ("stages", 9), ("consumer_warps", 25), ("slice_bytes", 4), ("store_mode", 4), ("wait_limit_ms", -1), ("withhold_copies", 2), ("average", 2), ("row_skew_lines", -2), ("copy_mode", 3),
+                             ("traversal", 2), ("l2_policy", 3)):
             bad = rps_options()
             lib.rps_default_options(ctypes.byref(bad))
             setattr(bad, field, value)
@@ -76,6 +78,8 @@ def test_options_pitch_and_state_errors(lib):
         assert lib.rps_step_n(h, 3) == -2
         assert lib.rps_read(h, None) == -2
         assert lib.rps_track(h, None, 4) == -2
+        a1, a2 = ctypes.c_double(), ctypes.c_double()
+        assert lib.rps_estimate_alpha(h, 0, 10, ctypes.byref(a1), ctypes.byref(a2)) == -2
         count = ctypes.c_int64()
         assert lib.rps_read_trace(h, None, 0, ctypes.byref(count)) == -2
         assert b"rps_bind" in lib.rps_last_error(h)

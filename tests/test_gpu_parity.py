@@ -467,3 +467,21 @@ def test_gradient_averaging_parity(rps_mod, oracle, name):
     other = r.read()
     r.close()
     assert np.abs(wl.as_float64(w, other) - wl.as_float64(w, want)).max() > 1e-3
+
+
+# ------------------------------------------------------------------ cache-related options change no bit
+
+def test_traversal_and_l2_policy_do_not_change_results(rps_mod):
+    """Walking the columns downwards on odd steps, or hinting the L2 cache, only moves work in time."""
+    for dtype, n, d in (("f32", 8, 300_010), ("f32", 32, 100_005), ("bf16", 64, 65_536)):
+        w = wl.Workload("cache", n=n, d=d, dtype=dtype, p=0.1, gamma=0.05, sigma=0.1, seed=11, steps=5)
+        b = wl.make_targets(w)
+        out = []
+        for kernel, traversal, l2_policy in ((2, 0, 0), (2, 1, 1), (2, 0, 2), (2, 1, 2), (1, 0, 0), (1, 1, 0)):
+            r = make(rps_mod, w, kernel=kernel, workers_per_lane=4, traversal=traversal, l2_policy=l2_policy)
+            r.set_targets(b)
+            r.step_n(w.steps)
+            out.append(r.read().view(np.uint16 if dtype == "bf16" else np.uint32))
+            r.close()
+        for other in out[1:]:
+            assert (other == out[0]).all()
