@@ -225,6 +225,7 @@ def run_cuda(args):
 
         dist.init_process_group("nccl", device_id=device)
     build.build()
+    import numpy as np
 
     w = wl.WORKLOADS[args.workload]
     if args.p is not None:
@@ -234,14 +235,25 @@ def run_cuda(args):
     if args.d is not None:
         w = w.scaled(d=args.d)
     b = wl.make_targets(w)
+    # --shard: the ranks cut ONE model by columns (no exchange: columns never interact); default: one whole
+    # model per rank.  `cols` is what this rank holds, `jobs` how many models the ranks process together.
+    begin, cols, jobs = 0, w.d, world
+    if args.shard and world > 1:
+        begin, cols = binding.shard_columns(w.d, world, rank)
+        if cols == 0:
+            raise SystemExit("--shard: the model is too short for this many ranks")
+        b = np.ascontiguousarray(b[:, begin:begin + cols])
+        jobs = 1
+    sharded = jobs != world
     r = binding.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma, kernel=args.kernel,
+                    shard_begin=begin if sharded else 0, shard_cols=cols if sharded else 0, launch_overlap=args.launch_overlap,
                     workers_per_lane=args.workers_per_lane, stages=args.stages, consumer_warps=args.consumer_warps, copy_mode=args.copy_mode, slice_bytes=args.slice_bytes, store_mode=args.store_mode, average_gradients=args.average_gradients, traversal=args.traversal, l2_policy=args.l2_policy)
     r.set_targets(b)
     if args.track:
         # every step of the run also records the distance to the optimum and the consensus error
         r.track(2 * max(args.warmup, 3) + 2 * args.steps + args.warmup + 64)
     stream = r.stream
-    bytes_per_step = w.bytes_per_step
+    bytes_per_step = w.bytes_per_step * cols // w.d
 
     # the clocks are sampled from here to the end of the timed steps: an NVML query takes milliseconds, so
     # the timed region alone (tens of milliseconds) would yield a single sample
@@ -262,19 +274,17 @@ def run_cuda(args):
     # pass 3: end to end through the host-buffer call: H2D of x and b, the step, D2H of x, every step
     e2e = None
     if not args.skip_e2e:
-        import numpy as np
-
         tdtype = torch.float32 if w.dtype == "f32" else torch.int16  # bf16 bit patterns travel as 16-bit words
-        x_host = torch.zeros((w.n, w.d), dtype=tdtype).pin_memory()
+        x_host = torch.zeros((w.n, cols), dtype=tdtype).pin_memory()
         b_host = torch.from_numpy(b if w.dtype == "f32" else b.view(np.int16)).pin_memory()
         e2e_steps = max(1, min(args.steps, args.e2e_steps))
         for _ in range(2):
             r.step_host(x_host, b_host)
         e2e_ms = timed_steps(torch, stream, lambda: [r.step_host(x_host, b_host) for _ in range(e2e_steps)], device)
-        e2e = {"value": world * w.n * w.d * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
-               "h2d_bytes_per_step": 2 * w.n * w.d * w.elem_bytes, "d2h_bytes_per_step": w.n * w.d * w.elem_bytes,
+        e2e = {"value": jobs * w.n * w.d * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
+               "h2d_bytes_per_step": 2 * w.n * cols * w.elem_bytes, "d2h_bytes_per_step": w.n * cols * w.elem_bytes,
                "call": "rps_step_host (pinned host x and b)"}
-    row_bytes = w.n * w.d * w.elem_bytes
+    row_bytes = w.n * cols * w.elem_bytes
 
     copy_gbs = in_situ_copy_gbs(torch, device)
     peak, peak_kind = measured_peak_gbs()
@@ -282,22 +292,25 @@ def run_cuda(args):
     achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
     traffic = traffic_cold = None
     default_shape = not (args.kernel or args.workers_per_lane or args.stages or args.consumer_warps or args.copy_mode or args.slice_bytes or args.store_mode
-                         or args.average_gradients or args.track or args.traversal or args.l2_policy)
+                         or args.average_gradients or args.track or args.traversal or args.l2_policy or args.launch_overlap or sharded)
     if default_shape and NCU_TRAFFIC["kernel_digest"] == kernel_digest():
         traffic = NCU_TRAFFIC["bytes_per_launch"].get(w.name)
         traffic_cold = NCU_TRAFFIC["cold_bytes_per_launch"].get(w.name)
 
     line = {
-        "metric": METRIC, "value": world * w.n * w.d * args.steps / (total_ms * 1e-3), "unit": UNIT,
+        "metric": METRIC, "value": jobs * w.n * w.d * args.steps / (total_ms * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {
             "workload": f"{w.name}: n={w.n} workers, d={w.d} {w.dtype}, p={w.p}, gamma={w.gamma}, sigma={w.sigma}, "
                         f"seed={w.seed}; quadratic objective, b_i ~ N({'mu_i' if w.hetero else '0'},1)",
-            "n": w.n, "d": w.d, "p": w.p, "replicas": "one independent job per GPU, no collective",
+            "n": w.n, "d": w.d, "p": w.p,
+            "replicas": ("one model cut by columns over the GPUs, no collective" if sharded
+                         else "one independent job per GPU, no collective"),
             "kernel_shape": {"kernel": args.kernel, "workers_per_lane": args.workers_per_lane, "stages": args.stages,
                              "consumer_warps": args.consumer_warps, "copy_mode": args.copy_mode, "slice_bytes": args.slice_bytes, "store_mode": args.store_mode,
-                             "traversal": args.traversal, "l2_policy": args.l2_policy},
+                             "traversal": args.traversal, "l2_policy": args.l2_policy,
+                             "launch_overlap": args.launch_overlap},
             "average": "gradients" if args.average_gradients else "models",
             "tracked": bool(args.track),
             "l2": "inputs larger than L2 (x and b are %.0f MB each)" % (row_bytes / 1e6),
@@ -397,6 +410,11 @@ def main(argv=None):
     ap.add_argument("--traversal", type=int, default=0,
                     help="0: odd steps walk the columns downwards (default); 1: every step upwards")
     ap.add_argument("--l2-policy", type=int, default=0, help="staged kernel: 1 plain loads, 2 targets evict-first")
+    ap.add_argument("--launch-overlap", type=int, default=0,
+                    help="staged kernel: 1 plain launches, 2 programmatic stream serialization (default)")
+    ap.add_argument("--shard", action="store_true",
+                    help="with --gpus N > 1: cut one model by columns over the ranks (strong scaling) instead of "
+                         "running one whole model per rank")
     ap.add_argument("--track", action="store_true",
                     help="time tracked steps: distance to the optimum and consensus error as a by-product of the pass")
     ap.add_argument("--store-mode", type=int, default=0, help="staged kernel: 1 register stores, 2 TMA stores")

@@ -115,6 +115,21 @@ typedef struct rps_options {
                                  L2 evict-first hint, which leaves the cache to the lines of x
                                  (a retained line of x saves a read and a write-back, one of b
                                  only a read); 0 = the library's choice                        */
+    int32_t launch_overlap;   /* kernel 2: 2 = the fused kernel is launched with programmatic stream
+                                 serialization: its CTAs may be placed and set up while the kernel
+                                 before it in the stream drains, and wait (griddepcontrol.wait) for
+                                 that kernel to complete before they read anything it may have
+                                 written; 1 = plain launches; 0 = the library's choice          */
+    /* Column shard.  Columns never interact (block j of every worker meets only block j of the
+     * others, and masks and noise are pure functions of (seed, t, block, worker, column)), so a
+     * model can be cut by columns over several handles, on one GPU or on several, with no
+     * exchange between them: each handle holds columns [shard_begin, shard_begin + shard_cols)
+     * of all n workers and produces bit for bit what a handle holding the whole model produces
+     * for those columns.  The device and host arrays of a shard handle are [n][shard_cols]
+     * (pitch from rps_pitch); d of rps_create stays the size of the whole model, which fixes the
+     * blocks.  shard_cols = 0 (default): the whole model.  shard_begin must be a multiple of 64. */
+    int64_t shard_begin;
+    int64_t shard_cols;
 } rps_options;
 
 /*
@@ -202,6 +217,10 @@ int rps_step_forced(rps_handle* h, const uint64_t* up, const uint64_t* down);
  * x_host (and b_host unless NULL, in which case the resident targets are used)
  * to the device, runs rps_step, copies the new replicas back into x_host and
  * synchronises.  Pinned host memory makes the copies fast; pageable works.
+ * Because columns never interact, a large model goes through in up to 8 pieces of
+ * columns: the upload of one piece overlaps the step and the download of the piece
+ * before it (two internal copy streams and a few events, created on the first call
+ * and released by rps_destroy; no device memory).  The result is that of rps_step.
  */
 int rps_step_host(rps_handle* h, void* x_host, const void* b_host);
 

@@ -21,7 +21,7 @@
  *   noise                distribution tests against a library normal CDF; the
  *                        paper fixes only zero mean and bounded variance
  *                        (Assumption 1), so its exact values are a convention of
- *                        this build: parity unpinned by the paper for that part
+ *                        this implementation: parity unpinned by the paper for that part
  *   bf16 rounding        library conversion on random inputs
  *   alpha_mc             exact alpha_1, alpha_2 from all drop patterns on tiny n (within the
  *                        sampling error), 0 and 1 at p = 0 and p = 1, a second route to the

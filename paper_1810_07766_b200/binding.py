@@ -41,7 +41,21 @@ class rps_options(ctypes.Structure):
                 ("copy_mode", ctypes.c_int32), ("slice_bytes", ctypes.c_int32),
                 ("store_mode", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32),
                 ("withhold_copies", ctypes.c_int32), ("average", ctypes.c_int32),
-                ("traversal", ctypes.c_int32), ("l2_policy", ctypes.c_int32)]
+                ("traversal", ctypes.c_int32), ("l2_policy", ctypes.c_int32), ("launch_overlap", ctypes.c_int32),
+                ("shard_begin", ctypes.c_int64), ("shard_cols", ctypes.c_int64)]
+
+
+def shard_columns(d: int, world: int, rank: int, align: int = 64) -> Tuple[int, int]:
+    """(shard_begin, shard_cols) of rank ``rank`` when a model of ``d`` columns is cut over ``world`` handles:
+    contiguous ranges that cover [0, d) once, each starting at a multiple of ``align`` columns, sizes within one
+    unit of ``align`` of each other (ranks past the end of a very short model get no columns: (d, 0))."""
+    if not (0 <= rank < world) or d < 1 or align < 1:
+        raise ValueError("need 0 <= rank < world, d >= 1, align >= 1")
+    units = -(-d // align)                      # whole or partial units of `align` columns
+    first = (units * rank) // world
+    last = (units * (rank + 1)) // world
+    begin, end = min(first * align, d), min(last * align, d)
+    return begin, end - begin
 
 
 class RPSError(RuntimeError):
@@ -120,12 +134,13 @@ class RPS:
     def __init__(self, n: int, d: int, p: float, gamma: float, seed: int, *, dtype: str = "f32", sigma: float = 0.0,
                  assign: int = RPS_ASSIGN_FIXED, self_delivery: bool = True, mask_window: int = 32,
                  kernel: int = 0, workers_per_lane: int = 0, stages: int = 0, consumer_warps: int = 0,
-                 row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0, wait_limit_ms: int = 0, withhold_copies: bool = False, average_gradients: bool = False, traversal: int = 0, l2_policy: int = 0, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+                 row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0, wait_limit_ms: int = 0, withhold_copies: bool = False, average_gradients: bool = False, traversal: int = 0, l2_policy: int = 0, launch_overlap: int = 0, shard_begin: int = 0, shard_cols: int = 0, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         if not torch.cuda.is_available():
             raise RuntimeError("the RPS library needs a CUDA device; there is no CPU path")
         self.n, self.d, self.dtype = int(n), int(d), dtype
+        self.cols = int(shard_cols) if shard_cols else int(d)  # columns this handle holds: its shard, or the model
         rc = self._lib.rps_create(n, d, p, gamma, seed, ctypes.byref(self._h))
         if rc != RPS_OK:
             raise RPSError(rc, "rps_create", self._lib.rps_last_error(None).decode())
@@ -137,7 +152,8 @@ class RPS:
         opt.row_skew_lines, opt.copy_mode, opt.slice_bytes = row_skew_lines, copy_mode, slice_bytes
         opt.store_mode, opt.wait_limit_ms, opt.withhold_copies = store_mode, wait_limit_ms, int(withhold_copies)
         opt.average = int(average_gradients)
-        opt.traversal, opt.l2_policy = traversal, l2_policy
+        opt.traversal, opt.l2_policy, opt.launch_overlap = traversal, l2_policy, launch_overlap
+        opt.shard_begin, opt.shard_cols = shard_begin, shard_cols
         self._check(self._lib.rps_configure(self._h, ctypes.byref(opt)), "rps_configure")
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
         self.pitch = int(self._lib.rps_pitch(self._h))
@@ -172,10 +188,10 @@ class RPS:
             pass
 
     def _host_array(self) -> np.ndarray:
-        return np.empty((self.n, self.d), dtype=np.float32 if self.dtype == "f32" else np.uint16)
+        return np.empty((self.n, self.cols), dtype=np.float32 if self.dtype == "f32" else np.uint16)
 
     def _expect(self, a, name: str) -> None:
-        want = (self.n, self.d)
+        want = (self.n, self.cols)
         if tuple(a.shape) != want:
             raise ValueError(f"{name} must have shape {want}")
         size = a.element_size() if isinstance(a, torch.Tensor) else a.dtype.itemsize

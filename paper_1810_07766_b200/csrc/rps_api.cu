@@ -28,6 +28,8 @@ namespace {
 
 constexpr size_t kDiagBytes = 256;   // two fp64 accumulators, then the kernels' error word, padded
 constexpr size_t kErrorOffset = 64;
+constexpr int kHostChunks = 8;                       // rps_step_host cuts the columns into at most this many pieces
+constexpr int64_t kHostChunkMinBytes = 4 << 20;      // ... of at least this many bytes of x each
 thread_local std::string g_create_error;
 
 struct TimedLaunch {
@@ -63,6 +65,10 @@ struct rps_handle {
     double ms[2] = {0.0, 0.0};
     int64_t timed[2] = {0, 0};
     rps::StepMasks staged{};  // host copy of caller-given masks
+    // rps_step_host: copy streams and the events that chain upload -> kernel -> download of each piece
+    cudaStream_t up_stream = nullptr, down_stream = nullptr;
+    cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
+    cudaEvent_t ev_up[kHostChunks] = {}, ev_done[kHostChunks] = {};
     // tracked steps (rps_track)
     double* trace = nullptr;
     int64_t trace_capacity = 0;
@@ -70,10 +76,12 @@ struct rps_handle {
     std::string error;
 
     size_t elem() const { return opt.dtype == RPS_BF16 ? 2 : 4; }
+    // columns held by this handle: the whole model, or its shard
+    int64_t cols() const { return opt.shard_cols > 0 ? opt.shard_cols : d; }
     int64_t pitch() const
     {
         const int64_t per_line = 128 / (int64_t)elem();
-        const int64_t lines = (d + per_line - 1) / per_line;
+        const int64_t lines = (cols() + per_line - 1) / per_line;
         return (lines + rps_row_skew_lines(lines, opt.row_skew_lines)) * per_line;
     }
     double* diag_acc() const { return reinterpret_cast<double*>(scratch); }
@@ -81,7 +89,7 @@ struct rps_handle {
     rps::FusedTuning tuning() const
     {
         return rps::FusedTuning{opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps, opt.copy_mode, opt.slice_bytes, opt.store_mode,
-                                 opt.wait_limit_ms, opt.withhold_copies, opt.traversal, opt.l2_policy};
+                                 opt.wait_limit_ms, opt.withhold_copies, opt.traversal, opt.l2_policy, opt.launch_overlap};
     }
     rps::StepMasks* window() const { return reinterpret_cast<rps::StepMasks*>(scratch + kDiagBytes); }
     rps::StepMasks* probe() const { return window() + opt.mask_window; }
@@ -173,14 +181,18 @@ int generate_masks(rps_handle* h, rps::StepMasks* out, uint64_t t0, int steps)
     return timed_launch(h, 1, [&] { return rps::launch_masks(prm, steps, h->stream); });
 }
 
-int run_fused(rps_handle* h, const rps::StepMasks* masks)
+// Launches the fused kernel of step h->t on columns [begin, begin + cols) of this handle's arrays (a
+// multiple-of-64 begin), without advancing the step: a step may be issued in several pieces.
+int launch_fused_window(rps_handle* h, const rps::StepMasks* masks, int64_t begin, int64_t cols)
 {
     rps::FusedParams prm{};
-    prm.x = h->x;
-    prm.b = h->b;
+    prm.x = static_cast<char*>(h->x) + (size_t)begin * h->elem();
+    prm.b = static_cast<const char*>(h->b) + (size_t)begin * h->elem();
     prm.masks = masks;
     prm.pitch = h->pitch();
-    prm.d = h->d;
+    prm.d = cols;
+    prm.col_offset = (h->opt.shard_cols > 0 ? h->opt.shard_begin : 0) + begin;
+    prm.cols_in_row = h->pitch() - begin;
     prm.block_cols = (h->d + h->n - 1) / h->n;
     prm.n = h->n;
     prm.narrow = h->d < ((int64_t)1 << 31);
@@ -194,18 +206,40 @@ int run_fused(rps_handle* h, const rps::StepMasks* masks)
     prm.t_lo = (uint32_t)h->t;
     prm.t_hi = (uint32_t)(h->t >> 32);
     rps::set_philox_key(prm, h->seed);
-    int rc = timed_launch(h, 0, [&] { return rps::launch_fused(prm, h->tuning(), h->opt.dtype == RPS_BF16, h->sm_count, h->stream); });
-    if (rc == RPS_OK) {
-        h->t += 1;
-        if (tracked) h->trace_used += 1;
+    return timed_launch(h, 0, [&] { return rps::launch_fused(prm, h->tuning(), h->opt.dtype == RPS_BF16, h->sm_count, h->stream); });
+}
+
+void advance_step(rps_handle* h)
+{
+    if (h->trace != nullptr && h->trace_used < h->trace_capacity) h->trace_used += 1;
+    h->t += 1;
+}
+
+// The mask record of step h->t, generating the next window of records when the step is outside the current one.
+int masks_of_step(rps_handle* h, const rps::StepMasks** out)
+{
+    const uint64_t window = (uint64_t)h->opt.mask_window;
+    if (!h->window_valid || h->t < h->window_t0 || h->t - h->window_t0 >= window) {
+        int rc = generate_masks(h, h->window(), h->t, (int)window);
+        if (rc != RPS_OK) return rc;
+        h->window_valid = true;
+        h->window_t0 = h->t;
     }
+    *out = h->window() + (h->t - h->window_t0);
+    return RPS_OK;
+}
+
+int run_fused(rps_handle* h, const rps::StepMasks* masks)
+{
+    int rc = launch_fused_window(h, masks, 0, h->cols());
+    if (rc == RPS_OK) advance_step(h);
     return rc;
 }
 
 int copy_rows(rps_handle* h, void* dst, size_t dst_pitch_bytes, const void* src, size_t src_pitch_bytes,
               cudaMemcpyKind kind)
 {
-    const size_t row_bytes = (size_t)h->d * h->elem();
+    const size_t row_bytes = (size_t)h->cols() * h->elem();
     if (dst_pitch_bytes < ((size_t)1 << 31) && src_pitch_bytes < ((size_t)1 << 31)) {
         RPS_CUDA(h, cudaMemcpy2DAsync(dst, dst_pitch_bytes, src, src_pitch_bytes, row_bytes, (size_t)h->n, kind,
                                       h->stream));
@@ -221,12 +255,12 @@ int copy_rows(rps_handle* h, void* dst, size_t dst_pitch_bytes, const void* src,
 
 int upload(rps_handle* h, void* dev, const void* host)
 {
-    return copy_rows(h, dev, (size_t)h->pitch() * h->elem(), host, (size_t)h->d * h->elem(), cudaMemcpyHostToDevice);
+    return copy_rows(h, dev, (size_t)h->pitch() * h->elem(), host, (size_t)h->cols() * h->elem(), cudaMemcpyHostToDevice);
 }
 
 int download(rps_handle* h, void* host, const void* dev)
 {
-    return copy_rows(h, host, (size_t)h->d * h->elem(), dev, (size_t)h->pitch() * h->elem(), cudaMemcpyDeviceToHost);
+    return copy_rows(h, host, (size_t)h->cols() * h->elem(), dev, (size_t)h->pitch() * h->elem(), cudaMemcpyDeviceToHost);
 }
 
 // Drains the stream and reports a kernel that gave up on a bounded wait.
@@ -266,6 +300,9 @@ int rps_default_options(rps_options* opt)
     opt->average = RPS_AVERAGE_MODELS;
     opt->traversal = 0;
     opt->l2_policy = 0;
+    opt->launch_overlap = 0;
+    opt->shard_begin = 0;
+    opt->shard_cols = 0;
     return RPS_OK;
 }
 
@@ -314,6 +351,20 @@ int rps_destroy(rps_handle* h)
         cudaEventDestroy(tl.start);
         cudaEventDestroy(tl.stop);
     }
+    if (h->up_stream) {
+        cudaStreamSynchronize(h->up_stream);
+        cudaStreamDestroy(h->up_stream);
+    }
+    if (h->down_stream) {
+        cudaStreamSynchronize(h->down_stream);
+        cudaStreamDestroy(h->down_stream);
+    }
+    if (h->ev_begin) cudaEventDestroy(h->ev_begin);
+    if (h->ev_end) cudaEventDestroy(h->ev_end);
+    for (int k = 0; k < kHostChunks; ++k) {
+        if (h->ev_up[k]) cudaEventDestroy(h->ev_up[k]);
+        if (h->ev_done[k]) cudaEventDestroy(h->ev_done[k]);
+    }
     delete h;
     return RPS_OK;
 }
@@ -349,6 +400,12 @@ int rps_configure(rps_handle* h, const rps_options* opt)
     if (opt->copy_mode < 0 || opt->copy_mode > 2) return fail(h, RPS_EINVAL, "copy_mode must be 0 (auto), 1 or 2");
     if (opt->traversal != 0 && opt->traversal != 1) return fail(h, RPS_EINVAL, "traversal must be 0 or 1");
     if (opt->l2_policy < 0 || opt->l2_policy > 2) return fail(h, RPS_EINVAL, "l2_policy must be 0 (auto), 1 or 2");
+    if (opt->launch_overlap < 0 || opt->launch_overlap > 2)
+        return fail(h, RPS_EINVAL, "launch_overlap must be 0 (auto), 1 or 2");
+    if (opt->shard_cols < 0 || opt->shard_begin < 0) return fail(h, RPS_EINVAL, "shard_begin and shard_cols must not be negative");
+    if (opt->shard_cols == 0 && opt->shard_begin != 0) return fail(h, RPS_EINVAL, "shard_begin without shard_cols");
+    if (opt->shard_cols > 0 && (opt->shard_begin % 64 != 0 || opt->shard_begin > h->d - opt->shard_cols))
+        return fail(h, RPS_EINVAL, "a shard starts at a multiple of 64 and ends inside the model");
     h->opt = *opt;
     h->sigma = (float)opt->sigma;
     return RPS_OK;
@@ -414,14 +471,9 @@ int rps_step(rps_handle* h)
 {
     int rc = need_bound(h);
     if (rc != RPS_OK) return rc;
-    const uint64_t window = (uint64_t)h->opt.mask_window;
-    if (!h->window_valid || h->t < h->window_t0 || h->t - h->window_t0 >= window) {
-        rc = generate_masks(h, h->window(), h->t, (int)window);
-        if (rc != RPS_OK) return rc;
-        h->window_valid = true;
-        h->window_t0 = h->t;
-    }
-    return run_fused(h, h->window() + (h->t - h->window_t0));
+    const rps::StepMasks* masks = nullptr;
+    if ((rc = masks_of_step(h, &masks)) != RPS_OK) return rc;
+    return run_fused(h, masks);
 }
 
 int rps_step_n(rps_handle* h, int64_t T)
@@ -462,10 +514,61 @@ int rps_step_host(rps_handle* h, void* x_host, const void* b_host)
     int rc = need_bound(h);
     if (rc != RPS_OK) return rc;
     if (!x_host) return fail(h, RPS_EINVAL, "x_host is NULL");
-    if ((rc = upload(h, h->x, x_host)) != RPS_OK) return rc;
-    if (b_host && (rc = upload(h, h->b, b_host)) != RPS_OK) return rc;
-    if ((rc = rps_step(h)) != RPS_OK) return rc;
-    if ((rc = download(h, x_host, h->x)) != RPS_OK) return rc;
+    // Columns never interact, so the step is issued in pieces: piece k is uploaded on one copy stream,
+    // stepped on the bound stream and downloaded on another copy stream, and the upload of piece k + 1
+    // runs while piece k is on its way back (PCIe carries both directions at once).
+    const int64_t cols = h->cols();
+    const int64_t row_bytes = cols * (int64_t)h->elem();
+    int pieces = (int)(row_bytes * h->n / kHostChunkMinBytes);
+    if (pieces > kHostChunks) pieces = kHostChunks;
+    if (pieces < 2 || h->pitch() >= ((int64_t)1 << 31)) {
+        if ((rc = upload(h, h->x, x_host)) != RPS_OK) return rc;
+        if (b_host && (rc = upload(h, h->b, b_host)) != RPS_OK) return rc;
+        if ((rc = rps_step(h)) != RPS_OK) return rc;
+        if ((rc = download(h, x_host, h->x)) != RPS_OK) return rc;
+        return finish(h);
+    }
+    if (h->up_stream == nullptr) {
+        RPS_CUDA(h, cudaStreamCreateWithFlags(&h->up_stream, cudaStreamNonBlocking));
+        RPS_CUDA(h, cudaStreamCreateWithFlags(&h->down_stream, cudaStreamNonBlocking));
+        RPS_CUDA(h, cudaEventCreateWithFlags(&h->ev_begin, cudaEventDisableTiming));
+        RPS_CUDA(h, cudaEventCreateWithFlags(&h->ev_end, cudaEventDisableTiming));
+        for (int k = 0; k < kHostChunks; ++k) {
+            RPS_CUDA(h, cudaEventCreateWithFlags(&h->ev_up[k], cudaEventDisableTiming));
+            RPS_CUDA(h, cudaEventCreateWithFlags(&h->ev_done[k], cudaEventDisableTiming));
+        }
+    }
+    const rps::StepMasks* masks = nullptr;
+    if ((rc = masks_of_step(h, &masks)) != RPS_OK) return rc;
+    // the uploads overwrite what earlier work on the bound stream may still be using
+    RPS_CUDA(h, cudaEventRecord(h->ev_begin, h->stream));
+    RPS_CUDA(h, cudaStreamWaitEvent(h->up_stream, h->ev_begin, 0));
+    RPS_CUDA(h, cudaStreamWaitEvent(h->down_stream, h->ev_begin, 0));
+    const size_t es = h->elem();
+    const size_t dev_pitch = (size_t)h->pitch() * es, host_pitch = (size_t)cols * es;
+    const int64_t units = (cols + 63) / 64;  // pieces start at multiples of 64 columns
+    for (int k = 0; k < pieces; ++k) {
+        const int64_t begin = units * k / pieces * 64;
+        const int64_t end = k + 1 == pieces ? cols : units * (k + 1) / pieces * 64;
+        if (end <= begin) continue;
+        const size_t width = (size_t)(end - begin) * es, at = (size_t)begin * es;
+        RPS_CUDA(h, cudaMemcpy2DAsync(static_cast<char*>(h->x) + at, dev_pitch, static_cast<const char*>(x_host) + at,
+                                      host_pitch, width, (size_t)h->n, cudaMemcpyHostToDevice, h->up_stream));
+        if (b_host)
+            RPS_CUDA(h, cudaMemcpy2DAsync(static_cast<char*>(h->b) + at, dev_pitch,
+                                          static_cast<const char*>(b_host) + at, host_pitch, width, (size_t)h->n,
+                                          cudaMemcpyHostToDevice, h->up_stream));
+        RPS_CUDA(h, cudaEventRecord(h->ev_up[k], h->up_stream));
+        RPS_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_up[k], 0));
+        if ((rc = launch_fused_window(h, masks, begin, end - begin)) != RPS_OK) return rc;
+        RPS_CUDA(h, cudaEventRecord(h->ev_done[k], h->stream));
+        RPS_CUDA(h, cudaStreamWaitEvent(h->down_stream, h->ev_done[k], 0));
+        RPS_CUDA(h, cudaMemcpy2DAsync(static_cast<char*>(x_host) + at, host_pitch, static_cast<const char*>(h->x) + at,
+                                      dev_pitch, width, (size_t)h->n, cudaMemcpyDeviceToHost, h->down_stream));
+    }
+    advance_step(h);
+    RPS_CUDA(h, cudaEventRecord(h->ev_end, h->down_stream));
+    RPS_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_end, 0));
     return finish(h);
 }
 
@@ -506,7 +609,7 @@ int rps_diag(rps_handle* h, double* dist2_to_opt, double* consensus)
     prm.b = h->b;
     prm.out = h->diag_acc();
     prm.pitch = h->pitch();
-    prm.d = h->d;
+    prm.d = h->cols();  // a shard reports its own columns' part of both sums
     prm.n = h->n;
     cudaError_t err = rps::launch_diag(prm, h->opt.dtype == RPS_BF16, h->sm_count, h->stream);
     if (err != cudaSuccess) return cuda_fail(h, "diagnostic kernel launch", err);

@@ -184,7 +184,7 @@ __device__ __forceinline__ void add_gradient_noise(float (&v)[WPT][VEC], int64_t
     for (int w = 0; w < WPT; w += 2) {
 #pragma unroll
         for (int q = 0; q < VEC / 4; ++q) {
-            const Philox4 r = philox4x32_keyed<kNoiseRounds>(prm.t_lo, prm.t_hi, (uint32_t)(c >> 2) + q,
+            const Philox4 r = philox4x32_keyed<kNoiseRounds>(prm.t_lo, prm.t_hi, (uint32_t)((c + prm.col_offset) >> 2) + q,
                                                              kStreamNoise | ((uint32_t)((w_first + w) >> 1) << 8),
                                                              prm.round_key);
             const uint32_t words[4] = {r.x, r.y, r.z, r.w};
@@ -239,11 +239,13 @@ __device__ __forceinline__ float sum_over_groups(float s)
     return s;
 }
 
-// Block (parameter server) of column c: columns are cut into n blocks of
-// block_cols = ceil(d / n) columns (Step 0, model partitioning).
+// Block (parameter server) of local column c: the model's columns are cut into n blocks of
+// block_cols = ceil(d / n) columns (Step 0, model partitioning); x and b may be a window of the
+// model that starts at its column col_offset.
 __device__ __forceinline__ int block_of(int64_t c, const FusedParams& prm)
 {
-    return prm.narrow ? (int)((uint32_t)c / (uint32_t)prm.block_cols) : (int)(c / prm.block_cols);
+    const int64_t g = c + prm.col_offset;
+    return prm.narrow ? (int)((uint32_t)g / (uint32_t)prm.block_cols) : (int)(g / prm.block_cols);
 }
 
 // What a lane needs to know about the masks: the words of block j, shifted so
@@ -257,13 +259,13 @@ struct MaskView {
 // Remembers the block a lane was last in: lanes walk the columns upwards, so the block
 // index is recomputed (one division) only when a lane crosses into a new block.
 struct BlockCursor {
-    int64_t begin = 0, end = 0;  // columns [begin, end) belong to block j; empty at first
+    int64_t begin = 0, end = 0;  // local columns [begin, end) belong to block j; empty at first
     int j = 0;
     __device__ __forceinline__ int locate(int64_t c, const FusedParams& prm)
     {
         if (c < begin || c >= end) {
             j = block_of(c, prm);
-            begin = (int64_t)j * prm.block_cols;
+            begin = (int64_t)j * prm.block_cols - prm.col_offset;
             end = begin + prm.block_cols;
         }
         return j;

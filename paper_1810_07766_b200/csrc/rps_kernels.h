@@ -33,6 +33,7 @@ struct FusedTuning {
     int32_t withhold_copies;   // staged kernel, test aid: issue no copies so that the bounded waits run out
     int32_t traversal;         // 0 odd steps walk the tiles downwards, 1 always upwards
     int32_t l2_policy;         // staged kernel: 1 plain loads, 2 targets loaded with the L2 evict-first hint
+    int32_t launch_overlap;    // staged kernel: 1 plain launch, 2 programmatic stream serialization
 };
 
 struct FusedParams {
@@ -42,10 +43,12 @@ struct FusedParams {
     int32_t* error;      // device word set non-zero when a bounded wait gave up (may be NULL)
     double* trace;       // tracked step: [2] sums this launch adds to (see Tracker), zeroed beforehand; else NULL
     int64_t pitch;       // row pitch in elements
-    int64_t d;           // model size
-    int64_t block_cols;  // ceil(d / n): columns per parameter-server block
+    int64_t d;           // columns to process: the model size, or the width of a window of its columns
+    int64_t col_offset;  // index in the whole model of column 0 of x and b (0 unless this is a window; a multiple of 64)
+    int64_t cols_in_row; // columns that may be read in a row from its first one (the pitch, less what precedes a window)
+    int64_t block_cols;  // ceil(model size / n): columns per parameter-server block
     int32_t n;
-    int32_t narrow;  // d < 2^31: block index by 32-bit division
+    int32_t narrow;  // model size < 2^31: block index by 32-bit division
     // v = keep * x + gamma * b - (gamma * sigma) * xi
     float keep;         // 1 - gamma
     float gamma;

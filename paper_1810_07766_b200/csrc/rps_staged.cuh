@@ -46,6 +46,7 @@ constexpr uint32_t kAbortFlagOffset = kSmemHeaderBytes - 128;
 constexpr int kOutBuffers = 2;
 constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;
 constexpr int kDefaultL2Policy = 1;
+constexpr int kDefaultLaunchOverlap = 2;
 static_assert(kSmemHeaderBytes % 128 == 0, "tile data must start on a 128-byte boundary");
 
 struct StagedShape {
@@ -231,6 +232,12 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // Launched with programmatic stream serialization this CTA may have been placed while the kernel before
+    // it in the stream was still draining.  Let the kernel after this one do the same, then wait for the one
+    // before to complete (its writes visible) before reading anything from global memory: the masks here, x
+    // and b in the producer.  Both are no-ops in a plain launch.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kAbortFlagOffset);
     if (threadIdx.x == 0) *abort_flag = 0;
     // tracked steps: the CTA's pair of sums and the count of warps that have added theirs
@@ -292,7 +299,7 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
                 }
             } else {
                 // one bulk copy per row and array, spread over the lanes; the last tile stops at the pitch
-                const int64_t cols_left = prm.pitch - c0;
+                const int64_t cols_left = prm.cols_in_row - c0;
                 const uint32_t cols = (uint32_t)(cols_left < shape.tile_cols ? cols_left : shape.tile_cols);
                 const uint32_t bytes = cols * elem;
                 if (lane == 0) mbar_arrive_expect_tx(bar, 2u * (uint32_t)n * bytes);
@@ -643,8 +650,8 @@ cudaError_t launch_staged_as(const FusedParams& prm, const FusedTuning& tune, in
     constexpr bool bf16 = sizeof(T) == 2;
     alignas(64) CUtensorMap map_x, map_b, map_out;
     const int map_box_cols = plan.shape.use_boxes ? plan.shape.box_cols : 16;  // unused by 1-D copies, but valid
-    if (!encode_rows(&map_x, prm.x, bf16, prm, map_box_cols, prm.pitch) ||
-        !encode_rows(&map_b, prm.b, bf16, prm, map_box_cols, prm.pitch) ||
+    if (!encode_rows(&map_x, prm.x, bf16, prm, map_box_cols, prm.cols_in_row) ||
+        !encode_rows(&map_b, prm.b, bf16, prm, map_box_cols, prm.cols_in_row) ||
         !encode_rows(&map_out, prm.x, bf16, prm, plan.shape.out_box_cols, prm.d))
         return cudaErrorInvalidValue;
     if (plan.smem_bytes > smem_granted) {
@@ -666,6 +673,19 @@ cudaError_t launch_staged_as(const FusedParams& prm, const FusedTuning& tune, in
     int64_t grid = (int64_t)sm_count * occ_per_sm;
     if (grid > plan.shape.tiles) grid = plan.shape.tiles;
     if (grid < 1) grid = 1;
+    if ((tune.launch_overlap != 0 ? tune.launch_overlap : kDefaultLaunchOverlap) == 2) {
+        cudaLaunchConfig_t config = {};
+        config.gridDim = dim3((unsigned)grid);
+        config.blockDim = dim3((unsigned)plan.threads);
+        config.dynamicSmemBytes = plan.smem_bytes;
+        config.stream = stream;
+        cudaLaunchAttribute attribute[1];
+        attribute[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attribute[0].val.programmaticStreamSerializationAllowed = 1;
+        config.attrs = attribute;
+        config.numAttrs = 1;
+        return cudaLaunchKernelEx(&config, kernel, prm, plan.shape, map_x, map_b, map_out);
+    }
     kernel<<<(unsigned)grid, plan.threads, plan.smem_bytes, stream>>>(prm, plan.shape, map_x, map_b, map_out);
     return cudaGetLastError();
 }

@@ -91,6 +91,8 @@ extern "C" int rps_step_static(int n, int64_t d, int dtype, void* x_dev, const v
     fp.masks = st->masks;
     fp.pitch = pitch;
     fp.d = d;
+    fp.col_offset = 0;
+    fp.cols_in_row = pitch;
     fp.block_cols = (d + n - 1) / n;
     fp.n = n;
     fp.narrow = d < ((int64_t)1 << 31);

@@ -60,6 +60,56 @@ def test_max_over_ranks_with_two_gloo_ranks():
     assert got == {0: 15.0, 1: 15.0}
 
 
+def _shard_rank_main(rank, world, port, results):
+    sys.path.insert(0, ROOT)
+    from paper_1810_07766_b200 import binding
+
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    try:
+        d = 4_000_037
+        mine = torch.tensor(binding.shard_columns(d, world, rank), dtype=torch.int64)
+        everyone = [torch.zeros(2, dtype=torch.int64) for _ in range(world)]
+        dist.all_gather(everyone, mine)
+        results.put((rank, [tuple(int(v) for v in e) for e in everyone]))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_column_shards_of_two_gloo_ranks_tile_the_model():
+    """Every rank derives its own column range from (d, world, rank) alone; together they cover the model once."""
+    ctx = mp.get_context("spawn")
+    results = ctx.Queue()
+    port = 31500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_shard_rank_main, args=(r, 2, port, results)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = dict(results.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=120)
+        assert p.exitcode == 0
+    assert got[0] == got[1]
+    (b0, c0), (b1, c1) = got[0]
+    assert b0 == 0 and b1 == c0 and b1 % 64 == 0 and c0 + c1 == 4_000_037 and abs(c0 - c1) < 128
+
+
+def test_shard_ranges_cover_the_model_once():
+    sys.path.insert(0, ROOT)
+    from paper_1810_07766_b200 import binding
+
+    for d in (1, 63, 64, 65, 1000, 4_000_037, 11_173_962):
+        for world in (1, 2, 3, 8, 64):
+            ranges = [binding.shard_columns(d, world, r) for r in range(world)]
+            at = 0
+            for begin, cols in ranges:
+                if cols:
+                    assert begin == at and begin % 64 == 0
+                    at += cols
+            assert at == d
+            sizes = [c for _, c in ranges if c]
+            assert max(sizes) - min(sizes) < 128
+
+
 def test_max_over_ranks_single_process_is_identity():
     sys.path.insert(0, ROOT)
     import bench

@@ -365,6 +365,42 @@ def test_step_host_equals_resident_step(rps_mod):
     r.close()
 
 
+@pytest.mark.parametrize("n,d,dtype", [(8, 600_011, "f32"), (64, 200_000, "bf16"), (16, 2_000_003, "f32")])
+def test_step_host_in_pieces_equals_resident_step(rps_mod, oracle, n, d, dtype):
+    """Large enough for the host-buffer step to go through in several pieces of columns (upload, step and
+    download overlapped): bit for bit the resident step, with and without uploading the targets every step,
+    tracked steps included; and within the step's tolerance of the oracle."""
+    w = wl.Workload("pieces", n=n, d=d, dtype=dtype, p=0.1, gamma=0.05, sigma=0.1, seed=40 + n, steps=3)
+    b = wl.make_targets(w)
+    bits = np.uint16 if dtype == "bf16" else np.uint32
+    r = make(rps_mod, w, kernel=2)
+    r.set_targets(b)
+    r.track(w.steps)
+    r.step_n(w.steps)
+    want = r.read()
+    want_trace = r.read_trace()
+    r.close()
+    tdtype = torch.float32 if dtype == "f32" else torch.int16
+    for resident_targets in (False, True):
+        r = make(rps_mod, w, kernel=2)
+        r.track(w.steps)
+        x_host = torch.zeros((n, d), dtype=tdtype).pin_memory()
+        b_host = torch.from_numpy(b if dtype == "f32" else b.view(np.int16)).pin_memory()
+        if resident_targets:
+            r.set_targets(b)
+        for _ in range(w.steps):
+            r.step_host(x_host, None if resident_targets else b_host)
+        assert r.get_step() == w.steps
+        got = x_host.numpy().view(bits)
+        assert (got == want.view(bits)).all()
+        assert (r.read().view(bits) == want.view(bits)).all()
+        assert np.allclose(r.read_trace(), want_trace, rtol=1e-9)
+        r.close()
+    ref = wl.make_initial(w)
+    oracle.run(ref, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps)
+    assert_close(w, want, ref, BF16_TOL if dtype == "bf16" else 3 * STEP_TOL)
+
+
 def test_profile_counts_launches(rps_mod):
     w = TWINS["cfg1"]
     r = make(rps_mod, w, mask_window=4)
@@ -472,13 +508,16 @@ def test_gradient_averaging_parity(rps_mod, oracle, name):
 # ------------------------------------------------------------------ cache-related options change no bit
 
 def test_traversal_and_l2_policy_do_not_change_results(rps_mod):
-    """Walking the columns downwards on odd steps, or hinting the L2 cache, only moves work in time."""
+    """Walking the columns downwards on odd steps, hinting the L2 cache, or letting a launch be set up while the
+    one before it drains, only moves work in time."""
     for dtype, n, d in (("f32", 8, 300_010), ("f32", 32, 100_005), ("bf16", 64, 65_536)):
         w = wl.Workload("cache", n=n, d=d, dtype=dtype, p=0.1, gamma=0.05, sigma=0.1, seed=11, steps=5)
         b = wl.make_targets(w)
         out = []
-        for kernel, traversal, l2_policy in ((2, 0, 0), (2, 1, 1), (2, 0, 2), (2, 1, 2), (1, 0, 0), (1, 1, 0)):
-            r = make(rps_mod, w, kernel=kernel, workers_per_lane=4, traversal=traversal, l2_policy=l2_policy)
+        for kernel, traversal, l2_policy, overlap in ((2, 0, 0, 0), (2, 1, 1, 1), (2, 0, 2, 2), (2, 1, 2, 2),
+                                                       (2, 0, 0, 2), (1, 0, 0, 0), (1, 1, 0, 2)):
+            r = make(rps_mod, w, kernel=kernel, workers_per_lane=4, traversal=traversal, l2_policy=l2_policy,
+                     launch_overlap=overlap)
             r.set_targets(b)
             r.step_n(w.steps)
             out.append(r.read().view(np.uint16 if dtype == "bf16" else np.uint32))
