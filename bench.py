@@ -45,6 +45,23 @@ NCU_TRAFFIC = {
 }
 
 
+# Lane instructions (warp instructions x 32) per replica-param and step of the temporally blocked kernel, from
+# ncu's smsp__inst_executed.sum of one launch of `bench.py --block-steps 16` (profiles/), keyed by workload.
+BLOCKED_LANE_INSTRUCTIONS = {
+    "kernel_digest": "unset",
+    "per_replica_param_step": {},
+}
+
+
+def blocked_kernel_digest() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_1810_07766_b200", "csrc")
+    for name in ("rps_device.cuh", "rps_blocked.cu"):
+        with open(os.path.join(csrc, name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
 def kernel_digest() -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_1810_07766_b200", "csrc")
@@ -246,7 +263,7 @@ def run_cuda(args):
         jobs = 1
     sharded = jobs != world
     r = binding.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma, kernel=args.kernel,
-                    shard_begin=begin if sharded else 0, shard_cols=cols if sharded else 0, launch_overlap=args.launch_overlap,
+                    shard_begin=begin if sharded else 0, shard_cols=cols if sharded else 0, launch_overlap=args.launch_overlap, block_steps=args.block_steps,
                     workers_per_lane=args.workers_per_lane, stages=args.stages, consumer_warps=args.consumer_warps, copy_mode=args.copy_mode, slice_bytes=args.slice_bytes, store_mode=args.store_mode, average_gradients=args.average_gradients, traversal=args.traversal, l2_policy=args.l2_policy)
     r.set_targets(b)
     if args.track:
@@ -292,7 +309,7 @@ def run_cuda(args):
     achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
     traffic = traffic_cold = None
     default_shape = not (args.kernel or args.workers_per_lane or args.stages or args.consumer_warps or args.copy_mode or args.slice_bytes or args.store_mode
-                         or args.average_gradients or args.track or args.traversal or args.l2_policy or args.launch_overlap or sharded)
+                         or args.average_gradients or args.track or args.traversal or args.l2_policy or args.launch_overlap or sharded or args.block_steps)
     if default_shape and NCU_TRAFFIC["kernel_digest"] == kernel_digest():
         traffic = NCU_TRAFFIC["bytes_per_launch"].get(w.name)
         traffic_cold = NCU_TRAFFIC["cold_bytes_per_launch"].get(w.name)
@@ -310,7 +327,7 @@ def run_cuda(args):
             "kernel_shape": {"kernel": args.kernel, "workers_per_lane": args.workers_per_lane, "stages": args.stages,
                              "consumer_warps": args.consumer_warps, "copy_mode": args.copy_mode, "slice_bytes": args.slice_bytes, "store_mode": args.store_mode,
                              "traversal": args.traversal, "l2_policy": args.l2_policy,
-                             "launch_overlap": args.launch_overlap},
+                             "launch_overlap": args.launch_overlap, "block_steps": args.block_steps},
             "average": "gradients" if args.average_gradients else "models",
             "tracked": bool(args.track),
             "l2": "inputs larger than L2 (x and b are %.0f MB each)" % (row_bytes / 1e6),
@@ -327,6 +344,27 @@ def run_cuda(args):
                      "mask_kernel_ms_per_launch": mask_ms / max(mask_n, 1), "mask_launches_timed": mask_n,
                      "in_situ_copy_gbs": copy_gbs, "frac_of_in_situ_copy": achieved / copy_gbs},
     }
+    if args.block_steps > 1:
+        # several steps per pass over x and b: the pass is bound by the arithmetic of a step, not by HBM.
+        # achieved = lane instructions executed per second (ncu's count per replica-param and step, recorded
+        # above with the digest of the kernel sources, x replica-params x steps per second); peak = one warp
+        # instruction of 32 lanes per scheduler and clock.
+        steps_per_launch = args.steps / max(fused_n, 1)
+        rp_steps_per_s = w.n * cols * steps_per_launch / (fused_avg_ms * 1e-3)
+        sm_count = torch.cuda.get_device_properties(device).multi_processor_count
+        mhz = line["clocks"].get("sm_max_mhz") or 1965
+        peak_alu = sm_count * 4 * 32 * mhz * 1e6 / 1e12
+        instr = None
+        if BLOCKED_LANE_INSTRUCTIONS["kernel_digest"] == blocked_kernel_digest():
+            instr = BLOCKED_LANE_INSTRUCTIONS["per_replica_param_step"].get(w.name)
+        alu = instr * rp_steps_per_s / 1e12 if instr else None
+        line["roofline"] = {"bound": "alu", "achieved": alu, "peak": peak_alu, "unit": "T lane-instructions/s",
+                            "frac": alu / peak_alu if alu else None, "traffic": None,
+                            "peak_kind": "derived: SMs x 4 schedulers x 32 lanes x max SM clock",
+                            "kernel": "rps_fused_blocked_kernel", "lane_instructions_per_replica_param_step": instr,
+                            "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n,
+                            "steps_per_launch": steps_per_launch,
+                            "hbm_gbs_algorithmic_per_launch": 3 * w.elem_bytes * w.n * cols / (fused_avg_ms * 1e-3) / 1e9}
     r.close()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = oracle_baseline(w, b)
@@ -412,6 +450,9 @@ def main(argv=None):
     ap.add_argument("--l2-policy", type=int, default=0, help="staged kernel: 1 plain loads, 2 targets evict-first")
     ap.add_argument("--launch-overlap", type=int, default=0,
                     help="staged kernel: 1 plain launches, 2 programmatic stream serialization (default)")
+    ap.add_argument("--block-steps", type=int, default=0,
+                    help="temporal blocking of rps_step_n: this many consecutive steps per pass over x and b (<= 32); "
+                         "the pass is then bound by arithmetic, not by HBM (off by default)")
     ap.add_argument("--shard", action="store_true",
                     help="with --gpus N > 1: cut one model by columns over the ranks (strong scaling) instead of "
                          "running one whole model per rank")

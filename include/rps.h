@@ -130,6 +130,15 @@ typedef struct rps_options {
      * blocks.  shard_cols = 0 (default): the whole model.  shard_begin must be a multiple of 64. */
     int64_t shard_begin;
     int64_t shard_cols;
+    /* Temporal blocking of rps_step_n.  With the quadratic objective of this library the gradient of
+     * a column needs only that column, so up to block_steps consecutive steps (2..mask_window) can be
+     * applied to a slice of x while it sits in registers: x and b are read once and x written once per
+     * block_steps steps, each step with its own masks and noise and with x rounded to the replica
+     * type as a store would.  The result equals that of single steps in the lane shape with 4 workers per lane
+     * bit for bit.  This is not the paper's setting (there a model's forward and backward pass sits
+     * between two synchronisations), so it is off by default (0 or 1); it applies to rps_step_n only,
+     * and only to untracked model averaging.                                                         */
+    int32_t block_steps;
 } rps_options;
 
 /*

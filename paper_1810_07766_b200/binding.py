@@ -42,7 +42,7 @@ class rps_options(ctypes.Structure):
                 ("store_mode", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32),
                 ("withhold_copies", ctypes.c_int32), ("average", ctypes.c_int32),
                 ("traversal", ctypes.c_int32), ("l2_policy", ctypes.c_int32), ("launch_overlap", ctypes.c_int32),
-                ("shard_begin", ctypes.c_int64), ("shard_cols", ctypes.c_int64)]
+                ("shard_begin", ctypes.c_int64), ("shard_cols", ctypes.c_int64), ("block_steps", ctypes.c_int32)]
 
 
 def shard_columns(d: int, world: int, rank: int, align: int = 64) -> Tuple[int, int]:
@@ -134,7 +134,7 @@ class RPS:
     def __init__(self, n: int, d: int, p: float, gamma: float, seed: int, *, dtype: str = "f32", sigma: float = 0.0,
                  assign: int = RPS_ASSIGN_FIXED, self_delivery: bool = True, mask_window: int = 32,
                  kernel: int = 0, workers_per_lane: int = 0, stages: int = 0, consumer_warps: int = 0,
-                 row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0, wait_limit_ms: int = 0, withhold_copies: bool = False, average_gradients: bool = False, traversal: int = 0, l2_policy: int = 0, launch_overlap: int = 0, shard_begin: int = 0, shard_cols: int = 0, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+                 row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0, wait_limit_ms: int = 0, withhold_copies: bool = False, average_gradients: bool = False, traversal: int = 0, l2_policy: int = 0, launch_overlap: int = 0, shard_begin: int = 0, shard_cols: int = 0, block_steps: int = 0, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         if not torch.cuda.is_available():
@@ -153,7 +153,7 @@ class RPS:
         opt.store_mode, opt.wait_limit_ms, opt.withhold_copies = store_mode, wait_limit_ms, int(withhold_copies)
         opt.average = int(average_gradients)
         opt.traversal, opt.l2_policy, opt.launch_overlap = traversal, l2_policy, launch_overlap
-        opt.shard_begin, opt.shard_cols = shard_begin, shard_cols
+        opt.shard_begin, opt.shard_cols, opt.block_steps = shard_begin, shard_cols, block_steps
         self._check(self._lib.rps_configure(self._h, ctypes.byref(opt)), "rps_configure")
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
         self.pitch = int(self._lib.rps_pitch(self._h))

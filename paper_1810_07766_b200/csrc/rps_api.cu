@@ -181,9 +181,8 @@ int generate_masks(rps_handle* h, rps::StepMasks* out, uint64_t t0, int steps)
     return timed_launch(h, 1, [&] { return rps::launch_masks(prm, steps, h->stream); });
 }
 
-// Launches the fused kernel of step h->t on columns [begin, begin + cols) of this handle's arrays (a
-// multiple-of-64 begin), without advancing the step: a step may be issued in several pieces.
-int launch_fused_window(rps_handle* h, const rps::StepMasks* masks, int64_t begin, int64_t cols)
+// The fused kernels' parameters for step h->t on columns [begin, begin + cols) of this handle's arrays.
+rps::FusedParams fused_params(rps_handle* h, const rps::StepMasks* masks, int64_t begin, int64_t cols)
 {
     rps::FusedParams prm{};
     prm.x = static_cast<char*>(h->x) + (size_t)begin * h->elem();
@@ -206,6 +205,14 @@ int launch_fused_window(rps_handle* h, const rps::StepMasks* masks, int64_t begi
     prm.t_lo = (uint32_t)h->t;
     prm.t_hi = (uint32_t)(h->t >> 32);
     rps::set_philox_key(prm, h->seed);
+    return prm;
+}
+
+// Launches the fused kernel of step h->t on columns [begin, begin + cols) of this handle's arrays (a
+// multiple-of-64 begin), without advancing the step: a step may be issued in several pieces.
+int launch_fused_window(rps_handle* h, const rps::StepMasks* masks, int64_t begin, int64_t cols)
+{
+    const rps::FusedParams prm = fused_params(h, masks, begin, cols);
     return timed_launch(h, 0, [&] { return rps::launch_fused(prm, h->tuning(), h->opt.dtype == RPS_BF16, h->sm_count, h->stream); });
 }
 
@@ -303,6 +310,7 @@ int rps_default_options(rps_options* opt)
     opt->launch_overlap = 0;
     opt->shard_begin = 0;
     opt->shard_cols = 0;
+    opt->block_steps = 0;
     return RPS_OK;
 }
 
@@ -406,6 +414,8 @@ int rps_configure(rps_handle* h, const rps_options* opt)
     if (opt->shard_cols == 0 && opt->shard_begin != 0) return fail(h, RPS_EINVAL, "shard_begin without shard_cols");
     if (opt->shard_cols > 0 && (opt->shard_begin % 64 != 0 || opt->shard_begin > h->d - opt->shard_cols))
         return fail(h, RPS_EINVAL, "a shard starts at a multiple of 64 and ends inside the model");
+    if (opt->block_steps < 0 || opt->block_steps > opt->mask_window)
+        return fail(h, RPS_EINVAL, "block_steps must be in 0..mask_window");
     h->opt = *opt;
     h->sigma = (float)opt->sigma;
     return RPS_OK;
@@ -479,6 +489,33 @@ int rps_step(rps_handle* h)
 int rps_step_n(rps_handle* h, int64_t T)
 {
     if (h && T < 0) return fail(h, RPS_EINVAL, "T is negative");
+    if (h && h->bound && h->opt.block_steps > 1 && h->opt.average == RPS_AVERAGE_MODELS) {
+        // temporal blocking: as many steps per launch as asked for and as the window of masks holds (a lone
+        // left-over step goes through the same kernel, so that the lane shape never changes within a run)
+        int64_t done = 0;
+        while (done < T) {
+            const bool tracked = h->trace != nullptr && h->trace_used < h->trace_capacity;
+            const rps::StepMasks* masks = nullptr;
+            int rc = masks_of_step(h, &masks);
+            if (rc != RPS_OK) return rc;
+            int64_t chunk = (int64_t)h->opt.mask_window - (int64_t)(h->t - h->window_t0);
+            if (chunk > h->opt.block_steps) chunk = h->opt.block_steps;
+            if (chunk > T - done) chunk = T - done;
+            if (tracked) {  // tracked steps run singly, in the same lane shape (4 workers per lane)
+                if ((rc = run_fused(h, masks)) != RPS_OK) return rc;
+                done += 1;
+                continue;
+            }
+            rps::FusedParams prm = fused_params(h, masks, 0, h->cols());
+            rc = timed_launch(h, 0, [&] {
+                return rps::launch_fused_blocked(prm, (int)chunk, h->opt.dtype == RPS_BF16, h->sm_count, h->stream);
+            });
+            if (rc != RPS_OK) return rc;
+            h->t += (uint64_t)chunk;
+            done += chunk;
+        }
+        return RPS_OK;
+    }
     for (int64_t k = 0; k < T; ++k) {
         int rc = rps_step(h);
         if (rc != RPS_OK) return rc;

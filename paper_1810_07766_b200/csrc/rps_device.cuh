@@ -176,15 +176,17 @@ struct RowVec<__nv_bfloat16, 4> {
 // instruction issue, turn into 8 % more throughput.
 constexpr int kNoiseRounds = 7;
 
-// Subtracts (gamma * sigma) * xi from v: one Philox draw per worker pair and four columns.
+// Subtracts (gamma * sigma) * xi from v: one Philox draw per worker pair and four columns, for step
+// t = (t_hi, t_lo).
 template <int VEC, int WPT>
-__device__ __forceinline__ void add_gradient_noise(float (&v)[WPT][VEC], int64_t c, int w_first, const FusedParams& prm)
+__device__ __forceinline__ void add_gradient_noise(float (&v)[WPT][VEC], int64_t c, int w_first, const FusedParams& prm,
+                                                   uint32_t t_lo, uint32_t t_hi)
 {
 #pragma unroll
     for (int w = 0; w < WPT; w += 2) {
 #pragma unroll
         for (int q = 0; q < VEC / 4; ++q) {
-            const Philox4 r = philox4x32_keyed<kNoiseRounds>(prm.t_lo, prm.t_hi, (uint32_t)((c + prm.col_offset) >> 2) + q,
+            const Philox4 r = philox4x32_keyed<kNoiseRounds>(t_lo, t_hi, (uint32_t)((c + prm.col_offset) >> 2) + q,
                                                              kStreamNoise | ((uint32_t)((w_first + w) >> 1) << 8),
                                                              prm.round_key);
             const uint32_t words[4] = {r.x, r.y, r.z, r.w};
@@ -221,7 +223,7 @@ __device__ __forceinline__ void local_sgd(const float (&xv)[WPT][VEC], const flo
 #pragma unroll
             for (int e = 0; e < VEC; ++e) v[w][e] -= xv[w][e];
     }
-    if (prm.noisy) add_gradient_noise<VEC, WPT>(v, c, w_first, prm);
+    if (prm.noisy) add_gradient_noise<VEC, WPT>(v, c, w_first, prm, prm.t_lo, prm.t_hi);
 }
 
 // s += v where `take` is set, as one predicated add (no branch, no select); a value that is

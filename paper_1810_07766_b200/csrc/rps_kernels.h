@@ -99,6 +99,9 @@ cudaError_t launch_staged_gradavg(const FusedParams& prm, const FusedTuning& tun
 cudaError_t launch_staged_tracked(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
                                   cudaStream_t stream);
 cudaError_t launch_direct_tracked(const FusedParams& prm, bool bf16, int sm_count, cudaStream_t stream);
+// `steps` consecutive steps from step (prm.t_hi, prm.t_lo) in one pass, with the mask records of those steps
+// at prm.masks[0 .. steps-1]; plain model averaging, untracked (rps_blocked.cu).
+cudaError_t launch_fused_blocked(const FusedParams& prm, int steps, bool bf16, int sm_count, cudaStream_t stream);
 cudaError_t launch_diag(const DiagParams& prm, bool bf16, int sm_count, cudaStream_t stream);
 
 }  // namespace rps

@@ -60,7 +60,7 @@ def test_options_pitch_and_state_errors(lib):
         assert opt.row_skew_lines == -1 and opt.copy_mode == 0 and opt.slice_bytes == 0 and opt.store_mode == 0
         assert opt.wait_limit_ms == 0 and opt.withhold_copies == 0 and opt.average == 0
         assert opt.traversal == 0 and opt.l2_policy == 0 and opt.launch_overlap == 0
-        assert opt.shard_begin == 0 and opt.shard_cols == 0
+        assert opt.shard_begin == 0 and opt.shard_cols == 0 and opt.block_steps == 0
         assert lib.rps_scratch_bytes(h) == 256 + 34 * 1792
         opt.dtype = 1
         assert lib.rps_configure(h, ctypes.byref(opt)) == 0
@@ -69,7 +69,8 @@ def test_options_pitch_and_state_errors(lib):
                              ("mask_window", 257), ("sigma", -1.0), ("kernel", 3), ("workers_per_lane", 3), ("stages", 1),
                              ("stages", 9), ("consumer_warps", 25), ("slice_bytes", 4), ("store_mode", 4), ("wait_limit_ms", -1), ("withhold_copies", 2), ("average", 2), ("row_skew_lines", -2), ("copy_mode", 3),
                              ("traversal", 2), ("l2_policy", 3), ("launch_overlap", 3),
-                             ("shard_cols", -1), ("shard_begin", 64), ("shard_cols", 11_173_963)):
+                             ("shard_cols", -1), ("shard_begin", 64), ("shard_cols", 11_173_963),
+                             ("block_steps", -1), ("block_steps", 33)):
             bad = rps_options()
             lib.rps_default_options(ctypes.byref(bad))
             setattr(bad, field, value)
