@@ -39,17 +39,17 @@ FALLBACK_HBM_GBS = 6650.0
 # algorithmic bytes.  "cold_bytes_per_launch": one launch alone with the caches flushed first
 # (cfg3 and cfg5 from captures at d/4 and d/8, scaled by 4 and 8).
 NCU_TRAFFIC = {
-    "kernel_digest": "3be8d0ef4408324f",
-    "bytes_per_launch": {"cfg2": 964367104, "cfg3": 4810349773, "cfg4": 1433042816, "cfg5": 6385079219},
-    "cold_bytes_per_launch": {"cfg2": 1022745856, "cfg3": 4713916416, "cfg4": 1490735016, "cfg5": 6073657344},
+    "kernel_digest": "f53f1dba271480c3",
+    "bytes_per_launch": {"cfg2": 959924941, "cfg3": 4802226586, "cfg4": 1429876250, "cfg5": 6407438387},
+    "cold_bytes_per_launch": {"cfg2": 1022663936, "cfg3": 4713299968, "cfg4": 1490523304, "cfg5": 6076841984},
 }
 
 
 # Lane instructions (warp instructions x 32) per replica-param and step of the temporally blocked kernel, from
 # ncu's smsp__inst_executed.sum of one launch of `bench.py --block-steps 16` (profiles/), keyed by workload.
 BLOCKED_LANE_INSTRUCTIONS = {
-    "kernel_digest": "unset",
-    "per_replica_param_step": {},
+    "kernel_digest": "89b9831650423752",
+    "per_replica_param_step": {"cfg2": 19.33, "cfg3": 20.47, "cfg4": 20.98, "cfg5": 20.56},
 }
 
 
