@@ -62,6 +62,11 @@ def blocked_kernel_digest() -> str:
     return h.hexdigest()[:16]
 
 
+# rps_options fields that shape the kernels without changing what is computed (command-line flags of the same names)
+SHAPE_OPTIONS = ("kernel", "workers_per_lane", "stages", "consumer_warps", "copy_mode", "slice_bytes", "store_mode",
+                 "traversal", "l2_policy", "launch_overlap", "block_steps")
+
+
 def kernel_digest() -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_1810_07766_b200", "csrc")
@@ -154,7 +159,8 @@ class ClockSampler:
 # ----------------------------------------------------------------------------- multi-rank plumbing
 
 def dist_env():
-    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    env = os.environ
+    return int(env.get("RANK", "0")), int(env.get("LOCAL_RANK", "0")), int(env.get("WORLD_SIZE", "1"))
 
 
 def max_over_ranks(value: float, device=None) -> float:
@@ -262,9 +268,11 @@ def run_cuda(args):
         b = np.ascontiguousarray(b[:, begin:begin + cols])
         jobs = 1
     sharded = jobs != world
-    r = binding.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma, kernel=args.kernel,
-                    shard_begin=begin if sharded else 0, shard_cols=cols if sharded else 0, launch_overlap=args.launch_overlap, block_steps=args.block_steps,
-                    workers_per_lane=args.workers_per_lane, stages=args.stages, consumer_warps=args.consumer_warps, copy_mode=args.copy_mode, slice_bytes=args.slice_bytes, store_mode=args.store_mode, average_gradients=args.average_gradients, traversal=args.traversal, l2_policy=args.l2_policy)
+    # the kernel-shape options, all 0 = the library's choice
+    shape = {name: getattr(args, name) for name in SHAPE_OPTIONS}
+    r = binding.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma,
+                    average_gradients=args.average_gradients, shard_begin=begin if sharded else 0,
+                    shard_cols=cols if sharded else 0, **shape)
     r.set_targets(b)
     if args.track:
         # every step of the run also records the distance to the optimum and the consensus error
@@ -308,8 +316,7 @@ def run_cuda(args):
     fused_avg_ms = fused_ms / max(fused_n, 1)
     achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
     traffic = traffic_cold = None
-    default_shape = not (args.kernel or args.workers_per_lane or args.stages or args.consumer_warps or args.copy_mode or args.slice_bytes or args.store_mode
-                         or args.average_gradients or args.track or args.traversal or args.l2_policy or args.launch_overlap or sharded or args.block_steps)
+    default_shape = not (any(shape.values()) or args.average_gradients or args.track or sharded)
     if default_shape and NCU_TRAFFIC["kernel_digest"] == kernel_digest():
         traffic = NCU_TRAFFIC["bytes_per_launch"].get(w.name)
         traffic_cold = NCU_TRAFFIC["cold_bytes_per_launch"].get(w.name)
@@ -317,17 +324,15 @@ def run_cuda(args):
     line = {
         "metric": METRIC, "value": jobs * w.n * w.d * args.steps / (total_ms * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
-        "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
+        "dtype": w.dtype, "data": "synthetic",
         "config": {
             "workload": f"{w.name}: n={w.n} workers, d={w.d} {w.dtype}, p={w.p}, gamma={w.gamma}, sigma={w.sigma}, "
                         f"seed={w.seed}; quadratic objective, b_i ~ N({'mu_i' if w.hetero else '0'},1)",
             "n": w.n, "d": w.d, "p": w.p,
             "replicas": ("one model cut by columns over the GPUs, no collective" if sharded
                          else "one independent job per GPU, no collective"),
-            "kernel_shape": {"kernel": args.kernel, "workers_per_lane": args.workers_per_lane, "stages": args.stages,
-                             "consumer_warps": args.consumer_warps, "copy_mode": args.copy_mode, "slice_bytes": args.slice_bytes, "store_mode": args.store_mode,
-                             "traversal": args.traversal, "l2_policy": args.l2_policy,
-                             "launch_overlap": args.launch_overlap, "block_steps": args.block_steps},
+            "kernel_shape": shape,
             "average": "gradients" if args.average_gradients else "models",
             "tracked": bool(args.track),
             "l2": "inputs larger than L2 (x and b are %.0f MB each)" % (row_bytes / 1e6),
@@ -339,7 +344,8 @@ def run_cuda(args):
         "e2e": e2e,
         "gpu_launches": gpu_launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "traffic_cold_cache": traffic_cold, "peak_kind": f"of {peak_kind}", "kernel": fused_kernel_name(args, w),
+                     "traffic": traffic, "traffic_cold_cache": traffic_cold, "peak_kind": f"of {peak_kind}",
+                     "kernel": fused_kernel_name(args, w),
                      "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n,
                      "mask_kernel_ms_per_launch": mask_ms / max(mask_n, 1), "mask_launches_timed": mask_n,
                      "in_situ_copy_gbs": copy_gbs, "frac_of_in_situ_copy": achieved / copy_gbs},
@@ -364,7 +370,7 @@ def run_cuda(args):
                             "kernel": "rps_fused_blocked_kernel", "lane_instructions_per_replica_param_step": instr,
                             "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n,
                             "steps_per_launch": steps_per_launch,
-                            "hbm_gbs_algorithmic_per_launch": 3 * w.elem_bytes * w.n * cols / (fused_avg_ms * 1e-3) / 1e9}
+                            "hbm_gbs_moved_per_launch": 3 * w.elem_bytes * w.n * cols / (fused_avg_ms * 1e-3) / 1e9}
     r.close()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = oracle_baseline(w, b)

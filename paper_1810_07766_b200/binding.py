@@ -133,8 +133,12 @@ class RPS:
 
     def __init__(self, n: int, d: int, p: float, gamma: float, seed: int, *, dtype: str = "f32", sigma: float = 0.0,
                  assign: int = RPS_ASSIGN_FIXED, self_delivery: bool = True, mask_window: int = 32,
+                 average_gradients: bool = False, shard_begin: int = 0, shard_cols: int = 0, block_steps: int = 0,
                  kernel: int = 0, workers_per_lane: int = 0, stages: int = 0, consumer_warps: int = 0,
-                 row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0, wait_limit_ms: int = 0, withhold_copies: bool = False, average_gradients: bool = False, traversal: int = 0, l2_policy: int = 0, launch_overlap: int = 0, shard_begin: int = 0, shard_cols: int = 0, block_steps: int = 0, device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+                 row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0,
+                 traversal: int = 0, l2_policy: int = 0, launch_overlap: int = 0,
+                 wait_limit_ms: int = 0, withhold_copies: bool = False,
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         if not torch.cuda.is_available():
@@ -148,7 +152,8 @@ class RPS:
         self._lib.rps_default_options(ctypes.byref(opt))
         opt.dtype, opt.assign, opt.self_delivery = _DTYPE[dtype], assign, int(self_delivery)
         opt.mask_window, opt.sigma = mask_window, sigma
-        opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps = kernel, workers_per_lane, stages, consumer_warps
+        opt.kernel, opt.workers_per_lane, opt.stages = kernel, workers_per_lane, stages
+        opt.consumer_warps = consumer_warps
         opt.row_skew_lines, opt.copy_mode, opt.slice_bytes = row_skew_lines, copy_mode, slice_bytes
         opt.store_mode, opt.wait_limit_ms, opt.withhold_copies = store_mode, wait_limit_ms, int(withhold_copies)
         opt.average = int(average_gradients)

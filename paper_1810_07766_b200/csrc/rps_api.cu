@@ -88,8 +88,20 @@ struct rps_handle {
     int32_t* error_word() const { return reinterpret_cast<int32_t*>(scratch + kErrorOffset); }
     rps::FusedTuning tuning() const
     {
-        return rps::FusedTuning{opt.kernel, opt.workers_per_lane, opt.stages, opt.consumer_warps, opt.copy_mode, opt.slice_bytes, opt.store_mode,
-                                 opt.wait_limit_ms, opt.withhold_copies, opt.traversal, opt.l2_policy, opt.launch_overlap};
+        rps::FusedTuning tune{};
+        tune.kernel = opt.kernel;
+        tune.workers_per_lane = opt.workers_per_lane;
+        tune.stages = opt.stages;
+        tune.consumer_warps = opt.consumer_warps;
+        tune.copy_mode = opt.copy_mode;
+        tune.slice_bytes = opt.slice_bytes;
+        tune.store_mode = opt.store_mode;
+        tune.wait_limit_ms = opt.wait_limit_ms;
+        tune.withhold_copies = opt.withhold_copies;
+        tune.traversal = opt.traversal;
+        tune.l2_policy = opt.l2_policy;
+        tune.launch_overlap = opt.launch_overlap;
+        return tune;
     }
     rps::StepMasks* window() const { return reinterpret_cast<rps::StepMasks*>(scratch + kDiagBytes); }
     rps::StepMasks* probe() const { return window() + opt.mask_window; }
@@ -213,7 +225,9 @@ rps::FusedParams fused_params(rps_handle* h, const rps::StepMasks* masks, int64_
 int launch_fused_window(rps_handle* h, const rps::StepMasks* masks, int64_t begin, int64_t cols)
 {
     const rps::FusedParams prm = fused_params(h, masks, begin, cols);
-    return timed_launch(h, 0, [&] { return rps::launch_fused(prm, h->tuning(), h->opt.dtype == RPS_BF16, h->sm_count, h->stream); });
+    return timed_launch(h, 0, [&] {
+        return rps::launch_fused(prm, h->tuning(), h->opt.dtype == RPS_BF16, h->sm_count, h->stream);
+    });
 }
 
 void advance_step(rps_handle* h)
@@ -410,7 +424,8 @@ int rps_configure(rps_handle* h, const rps_options* opt)
     if (opt->l2_policy < 0 || opt->l2_policy > 2) return fail(h, RPS_EINVAL, "l2_policy must be 0 (auto), 1 or 2");
     if (opt->launch_overlap < 0 || opt->launch_overlap > 2)
         return fail(h, RPS_EINVAL, "launch_overlap must be 0 (auto), 1 or 2");
-    if (opt->shard_cols < 0 || opt->shard_begin < 0) return fail(h, RPS_EINVAL, "shard_begin and shard_cols must not be negative");
+    if (opt->shard_cols < 0 || opt->shard_begin < 0)
+        return fail(h, RPS_EINVAL, "shard_begin and shard_cols must not be negative");
     if (opt->shard_cols == 0 && opt->shard_begin != 0) return fail(h, RPS_EINVAL, "shard_begin without shard_cols");
     if (opt->shard_cols > 0 && (opt->shard_begin % 64 != 0 || opt->shard_begin > h->d - opt->shard_cols))
         return fail(h, RPS_EINVAL, "a shard starts at a multiple of 64 and ends inside the model");
