@@ -1,0 +1,86 @@
+"""Seeded random combinations of every option against the oracle on small models: sizes from one column up,
+any n, both replica types, both server assignments, with and without self-delivery, model and gradient
+averaging, every kernel shape the library accepts, column shards, several steps per pass, odd start steps."""
+import numpy as np
+import pytest
+import torch
+
+from paper_1810_07766_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rps_mod():
+    if not torch.cuda.is_available():
+        pytest.fail("these tests need a CUDA device")
+    from paper_1810_07766_b200 import binding, build
+
+    build.build()
+    binding.load_library()
+    return binding
+
+
+def draw_case(rng):
+    n = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 9, 15, 16, 17, 31, 32, 33, 48, 63, 64]))
+    d = int(rng.choice([1, 2, 5, 63, 64, 65, 257, 1000, 4099, 20_011, 70_003]))
+    dtype = str(rng.choice(["f32", "bf16"]))
+    case = dict(n=n, d=d, dtype=dtype, p=float(rng.choice([0.0, 0.05, 0.3, 0.9, 1.0])),
+                gamma=float(rng.choice([0.02, 0.1, 0.5])), sigma=float(rng.choice([0.0, 0.1])),
+                seed=int(rng.integers(0, 2**63)), steps=int(rng.integers(1, 7)),
+                t0=int(rng.choice([0, 1, 5, 2**32 - 2, 2**40 + 3])),
+                assign=int(rng.integers(0, 2)), self_delivery=bool(rng.integers(0, 2)),
+                average_gradients=bool(rng.integers(0, 4) == 0))
+    opts = dict(kernel=int(rng.choice([0, 1, 2])), traversal=int(rng.integers(0, 2)),
+                mask_window=int(rng.choice([1, 3, 32])), launch_overlap=int(rng.integers(0, 3)))
+    if not case["average_gradients"]:
+        opts["workers_per_lane"] = int(rng.choice([0, 2, 4, 8]))
+        if rng.integers(0, 3) == 0 and opts["mask_window"] > 1:
+            opts["block_steps"] = int(rng.integers(2, opts["mask_window"] + 1))
+    if opts["kernel"] == 2:
+        opts["store_mode"] = int(rng.integers(0, 4))
+        opts["copy_mode"] = int(rng.integers(0, 3))
+        opts["l2_policy"] = int(rng.integers(0, 3))
+        opts["consumer_warps"] = int(rng.choice([0, 1, 3, 8, 16]))
+        opts["stages"] = int(rng.choice([0, 2, 3]))
+        if dtype == "bf16" and rng.integers(0, 3) == 0:
+            opts["slice_bytes"] = 8
+    shard = None
+    if d > 64 and rng.integers(0, 2) == 0:
+        begin = 64 * int(rng.integers(0, d // 64 + 1))
+        begin = min(begin, (d - 1) // 64 * 64)
+        cols = int(rng.integers(1, d - begin + 1))
+        shard = (begin, cols)
+    return case, opts, shard
+
+
+@pytest.mark.parametrize("index", range(160))
+def test_random_options_against_the_oracle(rps_mod, oracle, index):
+    rng = np.random.default_rng(20_240_000 + index)
+    case, opts, shard = draw_case(rng)
+    n, d, dtype = case["n"], case["d"], case["dtype"]
+    w = wl.Workload("fuzz", n=n, d=d, dtype=dtype, p=case["p"], gamma=case["gamma"], sigma=case["sigma"],
+                    seed=case["seed"], steps=case["steps"], hetero=True)
+    b = wl.make_targets(w)
+    x0 = rng.standard_normal((n, d)).astype(np.float32)
+    if dtype == "bf16":
+        x0 = wl.f32_to_bf16_bits(x0)
+    want = x0.copy()
+    oracle.run(want, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=case["t0"], steps=w.steps,
+               self_delivery=case["self_delivery"], assign=case["assign"], average_gradients=case["average_gradients"])
+    begin, cols = shard if shard else (0, d)
+    r = rps_mod.RPS(n, d, w.p, w.gamma, w.seed, dtype=dtype, sigma=w.sigma, assign=case["assign"],
+                    self_delivery=case["self_delivery"], average_gradients=case["average_gradients"],
+                    shard_begin=begin if shard else 0, shard_cols=cols if shard else 0, **opts)
+    r.set_targets(np.ascontiguousarray(b[:, begin:begin + cols]))
+    r.write(np.ascontiguousarray(x0[:, begin:begin + cols]))
+    r.set_step(case["t0"])
+    r.step_n(w.steps)
+    got = r.read()
+    assert r.get_step() == case["t0"] + w.steps
+    r.close()
+    g = wl.as_float64(w, got)
+    o = wl.as_float64(w, np.ascontiguousarray(want[:, begin:begin + cols]))
+    tol = 1e-2 if dtype == "bf16" else 1e-5
+    err = np.abs(g - o) / (1.0 + np.abs(o))
+    assert err.max() <= tol, (case, opts, shard, float(err.max()))
