@@ -64,7 +64,7 @@ def blocked_kernel_digest() -> str:
 
 # rps_options fields that shape the kernels without changing what is computed (command-line flags of the same names)
 SHAPE_OPTIONS = ("kernel", "workers_per_lane", "stages", "consumer_warps", "copy_mode", "slice_bytes", "store_mode",
-                 "traversal", "l2_policy", "launch_overlap", "block_steps")
+                 "traversal", "l2_policy", "launch_overlap", "block_steps", "team_warps")
 
 
 def kernel_digest() -> str:
@@ -82,6 +82,8 @@ def fused_kernel_name(args, w) -> str:
     small = w.n * w.d * w.elem_bytes < 148 * 8192
     if args.kernel == 1 or (args.kernel == 0 and small):
         return "rps_fused_direct_kernel"
+    if args.kernel == 3 and w.dtype == "bf16" and w.n > 4 and not (args.average_gradients or args.track):
+        return "rps_fused_ring_kernel"
     return "rps_fused_staged_kernel"
 
 
@@ -444,7 +446,9 @@ def main(argv=None):
     ap.add_argument("--reference-columns", type=int, default=500_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true", help="tuning sweeps only: leave the host-buffer pass out")
-    ap.add_argument("--kernel", type=int, default=0, help="0 library's choice, 1 direct loads, 2 staged")
+    ap.add_argument("--kernel", type=int, default=0,
+                    help="0 library's choice, 1 direct loads, 2 staged (producer warp), 3 self-refilling ring (bf16)")
+    ap.add_argument("--team-warps", type=int, default=0, help="ring kernel: warps that share a tile")
     ap.add_argument("--workers-per-lane", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--consumer-warps", type=int, default=0)

@@ -88,7 +88,12 @@ typedef struct rps_options {
                                  the row size is a multiple of a large power of two)         */
     int32_t kernel;           /* 1: lanes load their slices directly from global memory;
                                  2: slices are staged through shared memory by bulk
-                                 asynchronous copies (default)                               */
+                                 asynchronous copies issued by a producer warp;
+                                 3: the same staging with no producer warp: all 16 warps of a
+                                 CTA compute, in teams that take the tiles in turn, and the last
+                                 warp to have read a stage refills it (built for bf16 replicas
+                                 with more than 4 workers, plain untracked model averaging;
+                                 any other step runs as kernel 2)                            */
     int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */
     int32_t stages;           /* depth of the shared-memory ring of kernel 2 (2..8)          */
     int32_t consumer_warps;   /* compute warps per CTA of kernel 2 (1..24; shapes that need
@@ -139,6 +144,8 @@ typedef struct rps_options {
      * between two synchronisations), so it is off by default (0 or 1); it applies to rps_step_n only,
      * and only to untracked model averaging.                                                         */
     int32_t block_steps;
+    int32_t team_warps;       /* kernel 3: warps that share a tile: 1, 2, 4, 8 or 16 (0 = the library's
+                                 choice: the largest that leaves room for one more stage than teams) */
 } rps_options;
 
 /*

@@ -101,6 +101,7 @@ struct rps_handle {
         tune.traversal = opt.traversal;
         tune.l2_policy = opt.l2_policy;
         tune.launch_overlap = opt.launch_overlap;
+        tune.team_warps = opt.team_warps;
         return tune;
     }
     rps::StepMasks* window() const { return reinterpret_cast<rps::StepMasks*>(scratch + kDiagBytes); }
@@ -325,6 +326,7 @@ int rps_default_options(rps_options* opt)
     opt->shard_begin = 0;
     opt->shard_cols = 0;
     opt->block_steps = 0;
+    opt->team_warps = 0;
     return RPS_OK;
 }
 
@@ -403,7 +405,7 @@ int rps_configure(rps_handle* h, const rps_options* opt)
     if (!std::isfinite(opt->sigma) || opt->sigma < 0.0) return fail(h, RPS_EINVAL, "sigma must be finite and >= 0");
     if (opt->row_skew_lines < -1 || opt->row_skew_lines > 4096)
         return fail(h, RPS_EINVAL, "row_skew_lines must be -1 (auto) or 0..4096");
-    if (opt->kernel < 0 || opt->kernel > 2) return fail(h, RPS_EINVAL, "kernel must be 0 (auto), 1 or 2");
+    if (opt->kernel < 0 || opt->kernel > 3) return fail(h, RPS_EINVAL, "kernel must be 0 (auto), 1, 2 or 3");
     if (opt->workers_per_lane != 0 && opt->workers_per_lane != 2 && opt->workers_per_lane != 4 &&
         opt->workers_per_lane != 8)
         return fail(h, RPS_EINVAL, "workers_per_lane must be 0 (auto), 2, 4 or 8");
@@ -431,6 +433,9 @@ int rps_configure(rps_handle* h, const rps_options* opt)
         return fail(h, RPS_EINVAL, "a shard starts at a multiple of 64 and ends inside the model");
     if (opt->block_steps < 0 || opt->block_steps > opt->mask_window)
         return fail(h, RPS_EINVAL, "block_steps must be in 0..mask_window");
+    if (opt->team_warps != 0 && opt->team_warps != 1 && opt->team_warps != 2 && opt->team_warps != 4 &&
+        opt->team_warps != 8 && opt->team_warps != 16)
+        return fail(h, RPS_EINVAL, "team_warps must be 0 (auto), 1, 2, 4, 8 or 16");
     h->opt = *opt;
     h->sigma = (float)opt->sigma;
     return RPS_OK;

@@ -221,6 +221,7 @@ cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool b
                          cudaStream_t stream)
 {
     if (tune.kernel == 1) return launch_fused_direct(prm, tune, bf16, sm_count, stream);
+    if (tune.kernel == 3 && ring_kernel_covers(prm, bf16)) return launch_fused_ring(prm, tune, bf16, sm_count, stream);
     if (tune.kernel == 0) {
         // A model this short gives the staged kernel's ring less than a tile per SM: there
         // is nothing to pipeline and its set-up dominates; the step is launch bound and L2 resident.

@@ -22,7 +22,8 @@ struct MaskParams {
 
 // Which fused kernel runs and how it is shaped; 0 everywhere = the library's choice.
 struct FusedTuning {
-    int32_t kernel;            // 1 direct (register loads), 2 staged (bulk-async copies into shared memory)
+    int32_t kernel;            // 1 direct (register loads), 2 staged (a producer warp fills a shared-memory ring),
+                               // 3 self-refilling ring (every warp computes; bf16 replicas)
     int32_t workers_per_lane;  // 2, 4 or 8
     int32_t stages;            // shared-memory ring depth of the staged kernel
     int32_t consumer_warps;    // compute warps per CTA of the staged kernel
@@ -34,6 +35,7 @@ struct FusedTuning {
     int32_t traversal;         // 0 odd steps walk the tiles downwards, 1 always upwards
     int32_t l2_policy;         // staged kernel: 1 plain loads, 2 targets loaded with the L2 evict-first hint
     int32_t launch_overlap;    // staged kernel: 1 plain launch, 2 programmatic stream serialization
+    int32_t team_warps;        // ring kernel: warps that share a tile (1, 2, 4, 8 or 16)
 };
 
 struct FusedParams {
@@ -91,6 +93,10 @@ cudaError_t launch_fused_direct(const FusedParams& prm, const FusedTuning& tune,
                                 cudaStream_t stream);
 cudaError_t launch_fused_staged(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
                                 cudaStream_t stream);
+// The self-refilling ring (rps_ring.cu): whether it is built for this step, and its launch.
+bool ring_kernel_covers(const FusedParams& prm, bool bf16);
+cudaError_t launch_fused_ring(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
+                              cudaStream_t stream);
 // The optional forms of the fused step, built in one family of lane shapes, each group in a
 // translation unit of its own: gradient averaging (prm.average_gradients) and tracked steps
 // (prm.trace != NULL, with either kind of averaging).

@@ -33,6 +33,7 @@
 #include "rps_kernels.h"
 
 #include "rps_device.cuh"
+#include "rps_tma.cuh"
 
 namespace rps {
 
@@ -44,7 +45,6 @@ constexpr int kMaxBoxCols = 256;  // a TMA box is at most 256 elements wide
 constexpr uint32_t kSmemHeaderBytes = 128 + 2 * kMaxWorkers * 8 + kMaxWorkers * 4 + 128;  // barriers, mask copy, flags
 constexpr uint32_t kAbortFlagOffset = kSmemHeaderBytes - 128;
 constexpr int kOutBuffers = 2;
-constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;
 constexpr int kDefaultL2Policy = 1;
 constexpr int kDefaultLaunchOverlap = 2;
 static_assert(kSmemHeaderBytes % 128 == 0, "tile data must start on a 128-byte boundary");
@@ -81,121 +81,6 @@ struct StagedShape {
 
     __device__ __forceinline__ int64_t tile_of_turn(int64_t turn) const { return descending ? tiles - 1 - turn : turn; }
 };
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t arrivals)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(arrivals) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-
-// One try: the hardware may park the thread for up to `kSuspendHintNs` before answering.
-constexpr uint32_t kSuspendHintNs = 1000000u;
-
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
-        : "memory");
-    return done != 0;
-}
-
-__device__ __forceinline__ uint64_t global_timer_ns()
-{
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Waits for the phase with the given parity to complete; gives up after limit_ns.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t start = global_timer_ns();
-#pragma unroll 1
-    for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - start > limit_ns) return false;
-    }
-}
-
-// TMA tensor copy global -> shared of one box whose first element is (column, row) of the
-// tensor described by `map`; completion is signalled on `bar` as the box's bytes.
-__device__ __forceinline__ void tma_load_box(uint32_t dst_smem, const CUtensorMap* map, int32_t column, int32_t row,
-                                             uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-            dst_smem),
-        "l"(map), "r"(column), "r"(row), "r"(bar)
-        : "memory");
-}
-
-// Bulk asynchronous copy global -> shared of one contiguous run of bytes; completion is signalled
-// on `bar`.  Both addresses and the size are multiples of 16.
-__device__ __forceinline__ void bulk_load_row(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     dst_smem),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-
-// The same two copies carrying an L2 cache policy (made by createpolicy).
-__device__ __forceinline__ void tma_load_box(uint32_t dst_smem, const CUtensorMap* map, int32_t column, int32_t row,
-                                             uint32_t bar, uint64_t policy)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, "
-        "%3}], [%4], %5;" ::"r"(dst_smem),
-        "l"(map), "r"(column), "r"(row), "r"(bar), "l"(policy)
-        : "memory");
-}
-
-__device__ __forceinline__ void bulk_load_row(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar,
-                                              uint64_t policy)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
-            dst_smem),
-        "l"(src), "r"(bytes), "r"(bar), "l"(policy)
-        : "memory");
-}
-
-__device__ __forceinline__ uint64_t l2_evict_first_policy()
-{
-    uint64_t policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-    return policy;
-}
-
-// TMA tensor store shared -> global of one box; the unit clips what lies outside the tensor (columns >= d).
-__device__ __forceinline__ void tma_store_box(const CUtensorMap* map, int32_t column, int32_t row, uint32_t src_smem)
-{
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(column),
-                 "r"(row), "r"(src_smem)
-                 : "memory");
-}
-
-__device__ __forceinline__ void report_timeout(const FusedParams& prm, int code)
-{
-    if (prm.error != nullptr) atomicExch(prm.error, code);
-}
 
 // Eight workers per lane need more registers than 17 warps leave: that shape runs with at most 12 consumer
 // warps, or 20 in the narrow bf16 form (8-byte slices: half the raw registers, half the shared memory per warp).
@@ -594,40 +479,6 @@ bool make_plan(const FusedParams& prm, const FusedTuning& tune, int vec, int wpt
     return false;
 }
 
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// cuTensorMapEncodeTiled, fetched from the driver once (the library does not link libcuda).
-EncodeTiledFn encode_tiled_fn()
-{
-    static EncodeTiledFn fn = [] {
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult status;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &status) != cudaSuccess ||
-            status != cudaDriverEntryPointSuccess)
-            ptr = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(ptr);
-    }();
-    return fn;
-}
-
-// Describes one [n][pitch] array to the TMA unit, with boxes of n rows x box_cols columns; `cols` columns
-// of every row belong to the tensor (the pitch for loads, d for stores: what lies beyond is not written).
-bool encode_rows(CUtensorMap* map, const void* base, bool bf16, const FusedParams& prm, int box_cols, int64_t cols)
-{
-    EncodeTiledFn encode = encode_tiled_fn();
-    if (encode == nullptr) return false;
-    const size_t elem = bf16 ? 2 : 4;
-    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)prm.n};
-    const cuuint64_t strides[1] = {(cuuint64_t)prm.pitch * elem};  // bytes between rows
-    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)prm.n};
-    const cuuint32_t elem_strides[2] = {1, 1};
-    return encode(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
-                  const_cast<void*>(base), dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
 
 template <typename T, int VEC, int WPT, int G, bool GRAD = false, bool DIAG = false>
 cudaError_t launch_staged_as(const FusedParams& prm, const FusedTuning& tune, int sm_count, cudaStream_t stream)
