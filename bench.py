@@ -82,7 +82,9 @@ def fused_kernel_name(args, w) -> str:
     small = w.n * w.d * w.elem_bytes < 148 * 8192
     if args.kernel == 1 or (args.kernel == 0 and small):
         return "rps_fused_direct_kernel"
-    if args.kernel == 3 and w.dtype == "bf16" and w.n > 4 and not (args.average_gradients or args.track):
+    ring_built = w.dtype == "bf16" and w.n > 4 and not (args.average_gradients or args.track)
+    staged_only = args.workers_per_lane or args.consumer_warps or args.copy_mode or args.slice_bytes
+    if ring_built and (args.kernel == 3 or (args.kernel == 0 and w.n > 8 and not staged_only)):
         return "rps_fused_ring_kernel"
     return "rps_fused_staged_kernel"
 
@@ -259,6 +261,10 @@ def run_cuda(args):
         w = replace(w, p=args.p)
     if args.d is not None:
         w = w.scaled(d=args.d)
+    if args.sigma is not None:
+        from dataclasses import replace
+
+        w = replace(w, sigma=args.sigma)
     b = wl.make_targets(w)
     # --shard: the ranks cut ONE model by columns (no exchange: columns never interact); default: one whole
     # model per rank.  `cols` is what this rank holds, `jobs` how many models the ranks process together.
@@ -442,6 +448,8 @@ def main(argv=None):
     ap.add_argument("--workload", choices=("cfg1", "cfg2", "cfg3", "cfg4", "cfg5"), default="cfg2")
     ap.add_argument("--p", type=float, default=None, help="override the drop probability (p sweeps)")
     ap.add_argument("--d", type=int, default=None, help="override the model size (small profiler captures)")
+    ap.add_argument("--sigma", type=float, default=None,
+                    help="override the noise level (0 = no gradient noise: the step as pure data movement)")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--reference-columns", type=int, default=500_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")

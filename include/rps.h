@@ -93,18 +93,23 @@ typedef struct rps_options {
                                  CTA compute, in teams that take the tiles in turn, and the last
                                  warp to have read a stage refills it (built for bf16 replicas
                                  with more than 4 workers, plain untracked model averaging;
-                                 any other step runs as kernel 2)                            */
+                                 any other step runs as kernel 2).
+                                 0: kernel 1 for models too short to give every SM a tile, kernel 3
+                                 for bf16 replicas of more than 8 workers (unless an option that
+                                 shapes kernel 2 alone is set), else kernel 2                 */
     int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */
-    int32_t stages;           /* depth of the shared-memory ring of kernel 2 (2..8)          */
+    int32_t stages;           /* depth of the shared-memory ring of kernels 2 and 3 (2..8)   */
     int32_t consumer_warps;   /* compute warps per CTA of kernel 2 (1..24; shapes that need
                                  many registers are clamped lower)                           */
     int32_t copy_mode;        /* kernel 2 fills a stage with 1: one bulk copy per row,
                                  2: two-dimensional TMA boxes covering all n rows            */
     int32_t slice_bytes;      /* kernel 2, bf16 replicas: bytes of a row handled by one lane,
                                  16 or 8 (8 = more, lighter warps per tile)                  */
-    int32_t store_mode;       /* kernel 2 writes results 1: from registers, 16 bytes per lane,
-                                 2: through an output tile in shared memory with TMA tensor
-                                 stores, 3: in place in the stage, stored by a store warp    */
+    int32_t store_mode;       /* kernels 2 and 3 write results 1: from registers, 16 bytes per
+                                 lane, 2: through an output tile in shared memory with TMA tensor
+                                 stores, 3: in place in the stage, with TMA tensor stores from
+                                 there (kernel 2: by a store warp; kernel 3: by the last warp of
+                                 a team to have written)                                      */
     int32_t wait_limit_ms;    /* kernel 2: every wait of a warp on data or on a free stage gives
                                  up after this many milliseconds (0 = 2000); the next
                                  synchronising call then returns RPS_ECUDA                   */

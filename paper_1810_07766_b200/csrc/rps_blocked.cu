@@ -56,11 +56,11 @@ __global__ void __launch_bounds__(kBlockedThreads, sizeof(T) == 4 ? 3 : 2)
             const StepMasks* rec = prm.masks + s;
             const MaskView masks{rec->up, rec->down, rec->inv_cnt};
             const uint64_t t = t0 + (uint64_t)s;
-            // local SGD step, as local_sgd() evaluates it: v = keep * x + gamma * b - (gamma * sigma) * xi
+            // local SGD step, as local_sgd() evaluates it: v = x + gamma * (b - x) - (gamma * sigma) * xi
 #pragma unroll
             for (int w = 0; w < WPT; ++w)
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) v[w][e] = fmaf(prm.gamma, bv[w][e], prm.keep * v[w][e]);
+                for (int e = 0; e < VEC; ++e) v[w][e] = fmaf(prm.gamma, bv[w][e] - v[w][e], v[w][e]);
             if (prm.noisy) add_gradient_noise<VEC, WPT>(v, c, w_first, prm, (uint32_t)t, (uint32_t)(t >> 32));
             live_bits = average_and_select<VEC, WPT, G>(v, c, col_live, w_first, masks, cursor, prm);
             // what a single step would have stored and the next one read back

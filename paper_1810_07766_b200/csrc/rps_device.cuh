@@ -126,7 +126,23 @@ struct RowVec<float, 4> {
         return make_uint4(__float_as_uint(in[0]), __float_as_uint(in[1]), __float_as_uint(in[2]),
                           __float_as_uint(in[3]));
     }
+    // out = b - x, from the raw slice of b and the widened x
+    static __device__ __forceinline__ void deviation(const uint4 raw_b, const float (&x)[4], float (&out)[4])
+    {
+        out[0] = __uint_as_float(raw_b.x) - x[0], out[1] = __uint_as_float(raw_b.y) - x[1];
+        out[2] = __uint_as_float(raw_b.z) - x[2], out[3] = __uint_as_float(raw_b.w) - x[3];
+    }
 };
+
+// (lo, hi) = the two bf16 halves of `pair`, each minus an fp32 value, in fp32: the mixed-precision subtract of
+// sm_100 takes a bf16 operand as it is, so the halves of b are never widened by an instruction of their own.
+// The result is the correctly rounded fp32 difference, the same bits as widening first.
+__device__ __forceinline__ void bf16_pair_minus(uint32_t pair, float x_lo, float x_hi, float& lo, float& hi)
+{
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tsub.rn.f32.bf16 %0, l, %3;\n\tsub.rn.f32.bf16 %1, h, %4;\n\t}"
+        : "=f"(lo), "=f"(hi)
+        : "r"(pair), "f"(x_lo), "f"(x_hi));
+}
 
 template <>
 struct RowVec<__nv_bfloat16, 8> {
@@ -151,6 +167,12 @@ struct RowVec<__nv_bfloat16, 8> {
         }
         return make_uint4(w[0], w[1], w[2], w[3]);
     }
+    static __device__ __forceinline__ void deviation(const uint4 raw_b, const float (&x)[8], float (&out)[8])
+    {
+        const uint32_t w[4] = {raw_b.x, raw_b.y, raw_b.z, raw_b.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) bf16_pair_minus(w[k], x[2 * k], x[2 * k + 1], out[2 * k], out[2 * k + 1]);
+    }
 };
 
 // 8-byte slices of bf16 rows: half the columns per lane, so twice the lanes (and warps) per tile.
@@ -167,6 +189,11 @@ struct RowVec<__nv_bfloat16, 4> {
     {
         const __nv_bfloat162 lo = __floats2bfloat162_rn(in[0], in[1]), hi = __floats2bfloat162_rn(in[2], in[3]);
         return make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+    }
+    static __device__ __forceinline__ void deviation(const uint2 raw_b, const float (&x)[4], float (&out)[4])
+    {
+        bf16_pair_minus(raw_b.x, x[0], x[1], out[0], out[1]);
+        bf16_pair_minus(raw_b.y, x[2], x[3], out[2], out[3]);
     }
 };
 
@@ -204,26 +231,49 @@ __device__ __forceinline__ void add_gradient_noise(float (&v)[WPT][VEC], int64_t
 
 // Local SGD step of one lane: WPT workers (starting at the even worker w_first) x
 // VEC consecutive columns starting at column c, evaluated as
-//   v = x - gamma * ((x - b) + sigma * xi) = keep * x + gamma * b - (gamma * sigma) * xi,  keep = 1 - gamma.
-// One Philox draw serves a worker pair on four columns.  GRAD: leave the update v - x in v instead.
+//   v = x - gamma * ((x - b) + sigma * xi) = x + gamma * (b - x) - (gamma * sigma) * xi :
+// one subtraction, one fused multiply-add, and the noise (one Philox draw serves a worker pair on four
+// columns).  GRAD: leave the update v - x = gamma * (b - x) - (gamma * sigma) * xi in v instead.
+// `dev` holds b - x on entry.
 template <int VEC, int WPT, bool GRAD>
-__device__ __forceinline__ void local_sgd(const float (&xv)[WPT][VEC], const float (&bv)[WPT][VEC],
-                                          float (&v)[WPT][VEC], int64_t c, int w_first, const FusedParams& prm)
+__device__ __forceinline__ void sgd_from_deviation(const float (&xv)[WPT][VEC], const float (&dev)[WPT][VEC],
+                                                   float (&v)[WPT][VEC], int64_t c, int w_first, const FusedParams& prm)
 {
     static_assert(WPT % 2 == 0 && VEC % 4 == 0, "noise draws cover worker pairs and 4 columns");
 #pragma unroll
     for (int w = 0; w < WPT; ++w)
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) v[w][e] = fmaf(prm.gamma, bv[w][e], prm.keep * xv[w][e]);
-    if (GRAD) {
-        // gradient averaging exchanges the update u = v - x = -gamma * g instead of the model (x is
-        // taken off before the noise goes in, so that its registers are free by then)
-#pragma unroll
-        for (int w = 0; w < WPT; ++w)
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) v[w][e] -= xv[w][e];
-    }
+        for (int e = 0; e < VEC; ++e) v[w][e] = GRAD ? prm.gamma * dev[w][e] : fmaf(prm.gamma, dev[w][e], xv[w][e]);
     if (prm.noisy) add_gradient_noise<VEC, WPT>(v, c, w_first, prm, prm.t_lo, prm.t_hi);
+}
+
+// The same from widened x and b.
+template <int VEC, int WPT, bool GRAD>
+__device__ __forceinline__ void local_sgd(const float (&xv)[WPT][VEC], const float (&bv)[WPT][VEC],
+                                          float (&v)[WPT][VEC], int64_t c, int w_first, const FusedParams& prm)
+{
+    float dev[WPT][VEC];
+#pragma unroll
+    for (int w = 0; w < WPT; ++w)
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) dev[w][e] = bv[w][e] - xv[w][e];
+    sgd_from_deviation<VEC, WPT, GRAD>(xv, dev, v, c, w_first, prm);
+}
+
+// The same from the raw slices as they lie in memory: x is widened, b enters the subtraction as it is
+// (bf16 replicas: no instruction is spent on widening b; the bits of the result do not depend on the route).
+template <typename T, int VEC, int WPT, bool GRAD>
+__device__ __forceinline__ void local_sgd_raw(const typename RowVec<T, VEC>::Raw (&raw_x)[WPT],
+                                              const typename RowVec<T, VEC>::Raw (&raw_b)[WPT], float (&v)[WPT][VEC],
+                                              int64_t c, int w_first, const FusedParams& prm)
+{
+    float xv[WPT][VEC], dev[WPT][VEC];
+#pragma unroll
+    for (int w = 0; w < WPT; ++w) {
+        RowVec<T, VEC>::unpack(raw_x[w], xv[w]);
+        RowVec<T, VEC>::deviation(raw_b[w], xv[w], dev[w]);
+    }
+    sgd_from_deviation<VEC, WPT, GRAD>(xv, dev, v, c, w_first, prm);
 }
 
 // s += v where `take` is set, as one predicated add (no branch, no select); a value that is

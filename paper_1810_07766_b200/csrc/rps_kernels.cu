@@ -229,6 +229,11 @@ cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool b
         if (prm.d * bytes_per_column < (int64_t)sm_count * 8192)
             return launch_fused_direct(prm, tune, bf16, sm_count, stream);
     }
+    // bf16 replicas of more than 8 workers: the self-refilling ring (16 compute warps, no producer warp), unless
+    // an option that shapes the staged kernel only was set
+    if (tune.kernel == 0 && bf16 && prm.n > 8 && ring_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 &&
+        tune.consumer_warps == 0 && tune.copy_mode == 0 && tune.slice_bytes == 0)
+        return launch_fused_ring(prm, tune, bf16, sm_count, stream);
     return launch_fused_staged(prm, tune, bf16, sm_count, stream);
 }
 
@@ -245,7 +250,6 @@ void set_philox_key(FusedParams& prm, uint64_t seed)
 void set_sgd_scalars(FusedParams& prm, float gamma, float sigma)
 {
     prm.gamma = gamma;
-    prm.keep = 1.0f - gamma;
     const double gs = (double)gamma * (double)sigma;
     prm.noise_scale = (float)(-2.0 * 0.6931471805599453 * gs * gs);
     prm.noisy = sigma != 0.0f;

@@ -51,8 +51,7 @@ struct FusedParams {
     int64_t block_cols;  // ceil(model size / n): columns per parameter-server block
     int32_t n;
     int32_t narrow;  // model size < 2^31: block index by 32-bit division
-    // v = keep * x + gamma * b - (gamma * sigma) * xi
-    float keep;         // 1 - gamma
+    // v = x + gamma * (b - x) - (gamma * sigma) * xi
     float gamma;
     float noise_scale;  // -2 ln 2 * (gamma * sigma)^2
     int32_t noisy;      // sigma != 0
@@ -67,7 +66,7 @@ struct FusedParams {
 // Fills key0, key1 and round_key from the 64-bit seed.
 void set_philox_key(FusedParams& prm, uint64_t seed);
 
-// Fills keep, gamma, noise_scale and noisy from the float learning rate and noise level.
+// Fills gamma, noise_scale and noisy from the float learning rate and noise level.
 void set_sgd_scalars(FusedParams& prm, float gamma, float sigma);
 
 struct DiagParams {

@@ -288,26 +288,28 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
 
             float v[WPT][VEC];
             {
-                float xv[WPT][VEC], bv[WPT][VEC];
+                using Raw = typename RowVec<T, VEC>::Raw;
+                Raw raw_x[WPT], raw_b[WPT];
 #pragma unroll
                 for (int w = 0; w < WPT; ++w) {
                     // workers past n read the last real row: their values are masked out (their mask bits
                     // are 0) and never stored, so no lane needs a zero-filled stand-in
                     const int row = w_first + w < n ? w_first + w : n - 1;
-                    using Raw = typename RowVec<T, VEC>::Raw;
-                    const Raw raw_x = *reinterpret_cast<const Raw*>(base + (size_t)row * shape.row_bytes);
-                    const Raw raw_b =
-                        *reinterpret_cast<const Raw*>(base + shape.array_bytes + (size_t)row * shape.row_bytes);
-                    RowVec<T, VEC>::unpack(raw_x, xv[w]);
-                    RowVec<T, VEC>::unpack(raw_b, bv[w]);
+                    raw_x[w] = *reinterpret_cast<const Raw*>(base + (size_t)row * shape.row_bytes);
+                    raw_b[w] = *reinterpret_cast<const Raw*>(base + shape.array_bytes + (size_t)row * shape.row_bytes);
                 }
                 if (!hold_stage) {
                     // this warp has read everything it needs from the stage: hand it back to the producer
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_addr(&empty[stage]));
                 }
-                if (DIAG) tracker.targets(bv, present);
-                local_sgd<VEC, WPT, GRAD>(xv, bv, v, c, w_first, prm);
+                if (DIAG) {
+                    float bv[WPT][VEC];
+#pragma unroll
+                    for (int w = 0; w < WPT; ++w) RowVec<T, VEC>::unpack(raw_b[w], bv[w]);
+                    tracker.targets(bv, present);
+                }
+                local_sgd_raw<T, VEC, WPT, GRAD>(raw_x, raw_b, v, c, w_first, prm);
             }
             const uint32_t live_bits = average_and_select<VEC, WPT, G>(v, c, col_live, w_first, masks, cursor, prm);
             if (GRAD) {

@@ -55,9 +55,11 @@ def test_ring_equals_the_staged_kernel_bit_for_bit_and_the_oracle(rps_mod, oracl
     want = x0.copy()
     oracle.run(want, b, dtype="bf16", gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=3, steps=w.steps)
     ref = run(rps_mod, w, b, x0, w.steps, t0=3, kernel=2, workers_per_lane=8, store_mode=1)
-    for team_warps, stages in ((0, 0), (1, 2), (2, 0), (4, 3), (8, 2), (16, 0), (4, 8)):
-        got = run(rps_mod, w, b, x0, w.steps, t0=3, kernel=3, team_warps=team_warps, stages=stages)
-        assert (got == ref).all(), (team_warps, stages, int((got != ref).sum()))
+    for store_mode in (1, 2, 3):  # from registers; TMA tensor stores from an output tile; from the x tile in place
+        for team_warps, stages in ((0, 0), (1, 2), (2, 0), (4, 3), (8, 2), (16, 0), (4, 8)):
+            got = run(rps_mod, w, b, x0, w.steps, t0=3, kernel=3, team_warps=team_warps, stages=stages,
+                      store_mode=store_mode)
+            assert (got == ref).all(), (store_mode, team_warps, stages, int((got != ref).sum()))
     g, o = wl.as_float64(w, ref), wl.as_float64(w, want)
     assert (np.abs(g - o) / (1 + np.abs(o))).max() <= BF16_TOL
 
@@ -69,11 +71,12 @@ def test_ring_options_do_not_change_a_bit(rps_mod):
     b = wl.make_targets(w)
     x0 = wl.f32_to_bf16_bits(np.random.default_rng(5).standard_normal((w.n, w.d)).astype(np.float32))
     ref = run(rps_mod, w, b, x0, w.steps, kernel=3, traversal=1)
-    for opts in (dict(traversal=0), dict(launch_overlap=1), dict(mask_window=1), dict(mask_window=3, team_warps=4)):
-        assert (run(rps_mod, w, b, x0, w.steps, kernel=3, **opts) == ref).all(), opts
-    pieces = [(0, 64_000), (64_000, 100_032), (164_032, w.d - 164_032)]
-    parts = [run(rps_mod, w, b, x0, w.steps, shard=piece, kernel=3) for piece in pieces]
-    assert (np.concatenate(parts, axis=1) == ref).all()
+    for store_mode in (1, 2, 3):
+        for opts in (dict(traversal=0), dict(launch_overlap=1), dict(mask_window=1), dict(mask_window=3, team_warps=4)):
+            assert (run(rps_mod, w, b, x0, w.steps, kernel=3, store_mode=store_mode, **opts) == ref).all(), opts
+        pieces = [(0, 64_000), (64_000, 100_032), (164_032, w.d - 164_032)]
+        parts = [run(rps_mod, w, b, x0, w.steps, shard=piece, kernel=3, store_mode=store_mode) for piece in pieces]
+        assert (np.concatenate(parts, axis=1) == ref).all()
 
 
 def test_steps_the_ring_is_not_built_for_run_as_the_staged_kernel(rps_mod, oracle):
@@ -102,14 +105,15 @@ def test_steps_the_ring_is_not_built_for_run_as_the_staged_kernel(rps_mod, oracl
     assert (np.abs(g - o) / (1 + np.abs(o))).max() <= BF16_TOL and np.isfinite(trace).all()
 
 
-def test_a_ring_wait_that_runs_out_is_reported_and_harmless(rps_mod):
+@pytest.mark.parametrize("store_mode", [1, 2, 3])
+def test_a_ring_wait_that_runs_out_is_reported_and_harmless(rps_mod, store_mode):
     """Nothing is copied, so every warp's wait for its first tile runs out after the shortened limit: the kernel
     ends by itself, x is untouched, the next read reports it, and the device is as usable as before."""
     w = wl.Workload("ring", n=64, d=40_002, dtype="bf16", p=0.1, gamma=0.1, sigma=0.1, seed=9, steps=1)
     b = wl.make_targets(w)
     x0 = wl.f32_to_bf16_bits(np.random.default_rng(1).standard_normal((w.n, w.d)).astype(np.float32))
     r = rps_mod.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype="bf16", sigma=w.sigma, kernel=3, wait_limit_ms=20,
-                    withhold_copies=True)
+                    store_mode=store_mode, withhold_copies=True)
     r.set_targets(b)
     r.write(x0)
     r.step()
@@ -119,5 +123,5 @@ def test_a_ring_wait_that_runs_out_is_reported_and_harmless(rps_mod):
     torch.cuda.synchronize()
     assert (r.x_dev[:, :w.d].view(torch.int16).cpu().numpy().view(np.uint16) == x0.view(np.uint16)).all()
     r.close()
-    got = run(rps_mod, w, b, x0, 1, kernel=3, wait_limit_ms=20)
+    got = run(rps_mod, w, b, x0, 1, kernel=3, wait_limit_ms=20, store_mode=store_mode)
     assert (got == run(rps_mod, w, b, x0, 1, kernel=2, workers_per_lane=8, store_mode=1)).all()
