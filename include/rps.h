@@ -95,7 +95,7 @@ typedef struct rps_options {
                                  with more than 4 workers, plain untracked model averaging;
                                  any other step runs as kernel 2).
                                  0: kernel 1 for models too short to give every SM a tile, kernel 3
-                                 for bf16 replicas of more than 8 workers (unless an option that
+                                 for bf16 replicas of 9 to 56 workers (unless an option that
                                  shapes kernel 2 alone is set), else kernel 2                 */
     int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */
     int32_t stages;           /* depth of the shared-memory ring of kernels 2 and 3 (2..8)   */

@@ -5,11 +5,13 @@
 // handed out by warp scheduler: 16 warps of 128 registers fill it, a 17th warp (a producer) would cut every
 // warp to 96.  So here every warp computes and nobody only produces:
 //
-//   * The 16 warps of a CTA form teams of team_warps warps.  A tile (team_warps x WARP_COLS columns of
-//     all n rows of x and b) belongs to one team; the CTA's tiles go to the teams in turn, and tile L
-//     of the CTA lives in stage L mod stages of a shared-memory ring filled by TMA box copies
-//     (cp.async.bulk.tensor.2d, completion on the stage's mbarrier).  Tiles of 8 warps (64 KB at n = 64)
-//     instead of 16 are what lets a ring of three stages fit beside 16 compute warps.
+//   * A tile is team_warps x WARP_COLS columns of all n rows of x and b, one warp per slice of WARP_COLS
+//     columns; the 16 warps of a CTA are 16 / team_warps warps for every slice position, so that many tiles
+//     are worked on at a time.  Tile L of the CTA lives in stage L mod stages of a shared-memory ring filled
+//     by TMA box copies (cp.async.bulk.tensor.2d, completion on the stage's mbarrier).  Tiles of 8 warps
+//     (64 KB at n = 64) instead of 16 are what lets a ring of three stages fit beside 16 compute warps.
+//     A warp that is free takes the next tile of its slice position from a counter: no warp is tied to
+//     particular tiles, so a warp that fell behind is not waited for by the warps of other tiles.
 //   * A warp copies its slices of the stage to registers and counts itself off on the stage's counter
 //     (a shared-memory atomic).  The warp that counts last knows the stage is free: it resets the
 //     counter and issues the copies of the tile that comes `stages` tiles later, then goes on computing.
@@ -18,7 +20,7 @@
 //
 //   * Results leave either straight from registers with 16-byte streaming stores, or in place: x and b then
 //     have rings of their own; a b tile is handed back as soon as it has been read, the results are written
-//     over the x tile they came from, and the last warp of the team to have written sends the tile out with
+//     over the x tile they came from, and the last warp to have written its part of a tile sends the tile out with
 //     TMA tensor stores of whole boxes (whole 512-byte pieces of rows instead of the 64 bytes a lane group
 //     covers at n = 64), sees the unit finish reading it and refills the stage.
 //
@@ -34,7 +36,7 @@ constexpr int kRingMaxStages = 8;
 constexpr int kRingDefaultStoreMode = 1;  // 1 stores from registers, 3 in place + TMA tensor stores
 constexpr int kRingWarps = 16;  // 16 warps x 32 lanes x 128 registers = the whole register file
 // two sets (x ring, b ring) of: landed-data barriers, counters of warps done with a stage, counts of fills issued
-constexpr uint32_t kRingSyncBytes = 2 * kRingMaxStages * (8 + 4 + 4) + 2 * kRingWarps * 4;  // + the output tiles' counters
+constexpr uint32_t kRingSyncBytes = 2 * kRingMaxStages * (8 + 4 + 4) + 4 * kRingWarps * 4;  // + the output tiles' counters, the tile counters
 constexpr uint32_t kRingHeaderBytes = kRingSyncBytes + 2 * kMaxWorkers * 8 + kMaxWorkers * 4 + 128;  // + masks, flags
 constexpr uint32_t kRingFlagOffset = kRingHeaderBytes - 128;
 static_assert(kRingSyncBytes % 128 == 0 && kRingHeaderBytes % 128 == 0, "tile data must start on a 128-byte boundary");
@@ -54,7 +56,7 @@ struct RingShape {
     uint32_t array_bytes;   // one tile of one array: all its boxes
     uint32_t b_ring_offset; // of the b ring from the start of the x ring
     uint32_t out_offset;    // of the teams' output tiles from the start of the x ring (store_mode 2)
-    // 1: results leave from registers with 16-byte stores.  2: through an output tile per team in shared
+    // 1: results leave from registers with 16-byte stores.  2: through one of `teams` output tiles in shared
     // memory and TMA tensor stores of whole boxes.  In both a tile's x and b share one barrier and one
     // counter and are handed back as soon as they have been read.  3: results are written back over the x
     // tile and leave as TMA tensor stores from there; the b tile is handed back as soon as it has been read,
@@ -70,7 +72,7 @@ struct RingShape {
 // One ring's bookkeeping in shared memory.
 struct RingSync {
     uint64_t* full;       // [stages] mbarrier: the tile's copies have landed
-    int* done;            // [stages] warps of the team that are done with the stage
+    int* done;            // [stages] warps that are done with the stage (team_warps of them free it)
     volatile int* fills;  // [stages] fills issued so far
 };
 
@@ -99,21 +101,12 @@ struct RingCursor {
     int stage;
     uint32_t phase;
     int fill_no;
-    __device__ __forceinline__ RingCursor(int64_t local, int stages)
-        : stage((int)(local % stages)), phase((uint32_t)(local / stages) & 1u), fill_no((int)(local / stages) + 1)
+    __device__ __forceinline__ RingCursor(uint32_t local, uint32_t stages)
+        : stage((int)(local % stages)), phase((local / stages) & 1u), fill_no((int)(local / stages) + 1)
     {
-    }
-    __device__ __forceinline__ void advance(int by, int stages)
-    {
-        stage += by;
-        while (stage >= stages) {
-            stage -= stages;
-            phase ^= 1u;
-            ++fill_no;
-        }
     }
     // A parity wait can only tell a phase from the one before it, and the tile that had this stage last may
-    // belong to a slower team: first see that this tile's fill has been issued (which happens only after the
+    // still be with a slower warp: first see that this tile's fill has been issued (which happens only after the
     // earlier tile was done with), then wait for it to land.
     __device__ __forceinline__ bool wait(const RingSync& ring, uint64_t limit_ns) const
     {
@@ -144,12 +137,12 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
     unsigned char* b_ring = x_ring + shape.b_ring_offset;
     int* out_done = reinterpret_cast<int*>(smem + 256);                    // [teams] warps that have written their results
     volatile int* out_free = reinterpret_cast<volatile int*>(smem + 320);  // [teams] stores that have left the output tile
+    int* next_tile = reinterpret_cast<int*>(smem + 384);                   // [team_warps] next tile of each slice position
 
     const int n = prm.n;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const int team = warp / shape.team_warps;
-    const int warp_in_team = warp - team * shape.team_warps;
+    const int slot = warp % shape.team_warps;  // which slice of WARP_COLS columns of a tile this warp works on
     const bool in_place = shape.store_mode == 3, out_tiles = shape.store_mode == 2;
     // tiles of this CTA: turns blockIdx.x, blockIdx.x + gridDim.x, ...
     const int64_t my_tiles =
@@ -162,7 +155,7 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
             xs.done[s] = bs.done[s] = 0;
             xs.fills[s] = bs.fills[s] = 0;
         }
-        for (int k = 0; k < kRingWarps; ++k) out_done[k] = out_free[k] = 0;
+        for (int k = 0; k < kRingWarps; ++k) out_done[k] = out_free[k] = next_tile[k] = 0;
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
@@ -222,13 +215,11 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
     const MaskView masks{s_up, s_down, s_inv};
     const int sub = lane % LPG;
     const int w_first = (lane / LPG) * WPT;
-    const int col_in_tile = warp_in_team * WARP_COLS + sub * VEC;
+    const int col_in_tile = slot * WARP_COLS + sub * VEC;
     const uint32_t lane_off =
         (uint32_t)(col_in_tile / shape.box_cols) * shape.box_bytes + (uint32_t)(col_in_tile % shape.box_cols) * elem;
-    RingCursor at_x(team, shape.x_stages), at_b(team, shape.b_stages);
     BlockCursor cursor;
     bool stores_pending = false;
-    int tiles_done = 0;  // of this warp's team
     // What a warp does when something it waited for never came: say so, stop the refilling, and see the
     // copies that were issued land and its own stores leave (bounded) before its part of the CTA's shared
     // memory is given up.  Warps that still wait for something this warp will not count itself off on run
@@ -246,7 +237,13 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
         }
         if (stores_pending) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     };
-    for (int64_t local = team; local < my_tiles; local += shape.teams) {
+    for (;;) {
+        // the next tile of the CTA that no warp has taken at this slice position
+        int taken = 0;
+        if (lane == 0) taken = atomicAdd(&next_tile[slot], 1);
+        const int64_t local = __shfl_sync(0xFFFFFFFFu, taken, 0);
+        if (local >= my_tiles) break;
+        const RingCursor at_x((uint32_t)local, (uint32_t)shape.x_stages), at_b((uint32_t)local, (uint32_t)shape.b_stages);
         if (!__all_sync(0xFFFFFFFFu, (!in_place || at_x.wait(xs, shape.wait_limit_ns)) && at_b.wait(bs, shape.wait_limit_ns))) {
             give_up(2);
             return;
@@ -268,7 +265,7 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
                 raw_b[w] = *reinterpret_cast<const Raw*>(b_base + (size_t)row * shape.row_bytes);
             }
             // This warp has everything it needs from the tile (from its b half, if results go back in place).
-            // The last warp of the team to say so refills the stage with the tile that comes b_stages later.
+            // The last warp to say so refills the stage with the tile that comes b_stages later.
             __syncwarp();
             if (lane == 0 && count_off(&bs.done[at_b.stage]) == (uint32_t)shape.team_warps - 1u) {
                 bs.done[at_b.stage] = 0;  // seen by the stage's next readers through the barrier the refill completes
@@ -283,13 +280,16 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
         const uint32_t live_bits = average_and_select<VEC, WPT, G>(v, c, col_live, w_first, masks, cursor, prm);
         if (in_place || out_tiles) {
             unsigned char* out_base = x_base;
+            const int out_slot = (int)((uint32_t)local % (uint32_t)shape.teams);
+            const int out_turn = (int)((uint32_t)local / (uint32_t)shape.teams);
             if (out_tiles) {
-                // the team's output tile is free again once the store of the team's previous tile has read it
-                if (!__all_sync(0xFFFFFFFFu, wait_for_count(&out_free[team], tiles_done, shape.wait_limit_ns))) {
+                // tile L goes out through output tile L mod teams, which is free once the store of the tile
+                // that had it before has read it
+                if (!__all_sync(0xFFFFFFFFu, wait_for_count(&out_free[out_slot], out_turn, shape.wait_limit_ns))) {
                     give_up(3);
                     return;
                 }
-                out_base = x_ring + shape.out_offset + (size_t)team * shape.array_bytes + lane_off;
+                out_base = x_ring + shape.out_offset + (size_t)out_slot * shape.array_bytes + lane_off;
             }
             // in place every lane overwrites exactly the slices of x it read; columns past d are clipped by the store
 #pragma unroll
@@ -298,15 +298,15 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
                     *reinterpret_cast<Raw*>(out_base + (size_t)(w_first + w) * shape.row_bytes) = RowVec<T, VEC>::pack(v[w]);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // visible to the TMA unit
             __syncwarp();
-            // The last warp of the team to have written sends the tile to global memory and sees the unit finish
-            // reading it; then the output tile is free for the team's next tile, or (in place) the stage is
+            // The last warp to have written its part sends the tile to global memory and sees the unit finish
+            // reading it; then the output tile is free for the next tile that uses it, or (in place) the stage is
             // refilled with the x tile that comes x_stages later.
-            int* done = in_place ? &xs.done[at_x.stage] : &out_done[team];
+            int* done = in_place ? &xs.done[at_x.stage] : &out_done[out_slot];
             if (lane == 0 && count_off(done) == (uint32_t)shape.team_warps - 1u) {
                 *done = 0;
                 const int32_t c0 = (int32_t)(tile * shape.tile_cols);
                 const uint32_t src = in_place ? smem_addr(x_ring) + (uint32_t)at_x.stage * shape.array_bytes
-                                              : smem_addr(x_ring) + shape.out_offset + (uint32_t)team * shape.array_bytes;
+                                              : smem_addr(x_ring) + shape.out_offset + (uint32_t)out_slot * shape.array_bytes;
                 for (int k = 0; k < shape.boxes_per_tile; ++k) {
                     const int32_t col = c0 + k * shape.box_cols;
                     if (col < prm.d) tma_store_box(&map_out, col, 0, src + (uint32_t)k * shape.box_bytes);
@@ -316,13 +316,12 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
                 stores_pending = true;
                 if (out_tiles) {
                     __threadfence_block();
-                    out_free[team] = tiles_done + 1;
+                    out_free[out_slot] = out_turn + 1;
                 } else {
                     const int64_t next = local + shape.x_stages;
                     if (next < my_tiles && !*abort_flag) fill(next, true, false);
                 }
             }
-            ++tiles_done;
         } else {
             T* dst = xg + (int64_t)w_first * prm.pitch + c;  // this lane's slice of its first worker's row
             if (live_bits == (1u << VEC) - 1u) {
@@ -335,8 +334,6 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
                     if (w_first + w < n) store_ragged<T, VEC>(dst, v[w], live_bits);
             }
         }
-        at_x.advance(shape.teams, shape.x_stages);
-        at_b.advance(shape.teams, shape.b_stages);
     }
     // tensor stores issued by this thread still read this CTA's shared memory: see them through
     if (stores_pending) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
@@ -369,7 +366,7 @@ bool plan_ring(const FusedParams& prm, const FusedTuning& tune, int vec, int g, 
         sh->array_bytes = (uint32_t)sh->boxes_per_tile * sh->box_bytes;
         // shared memory holds `units` tiles of one array; an x tile is held through the arithmetic when
         // results go back in place, a b tile only until it has been read: the odd unit goes to x
-        const int out_units = sh->store_mode == 2 ? sh->teams : 0;  // one output tile per team
+        const int out_units = sh->store_mode == 2 ? sh->teams : 0;  // one output tile per tile in work
         const int units = (int)((smem_limit - kRingHeaderBytes) / sh->array_bytes) - out_units;
         int b_stages = units / 2, x_stages = sh->store_mode == 3 ? units - b_stages : b_stages;
         if (tune.stages > 0 && b_stages > tune.stages) b_stages = tune.stages;
