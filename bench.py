@@ -39,17 +39,17 @@ FALLBACK_HBM_GBS = 6650.0
 # algorithmic bytes.  "cold_bytes_per_launch": one launch alone with the caches flushed first
 # (cfg3 and cfg5 from captures at d/4 and d/8, scaled by 4 and 8).
 NCU_TRAFFIC = {
-    "kernel_digest": "f53f1dba271480c3",
-    "bytes_per_launch": {"cfg2": 959924941, "cfg3": 4802226586, "cfg4": 1429876250, "cfg5": 6407438387},
-    "cold_bytes_per_launch": {"cfg2": 1022663936, "cfg3": 4713299968, "cfg4": 1490523304, "cfg5": 6076841984},
+    "kernel_digest": "227d43ac0d269397",
+    "bytes_per_launch": {"cfg2": 961970022, "cfg3": 4803649894, "cfg4": 1430062464, "cfg5": 6381472333},
+    "cold_bytes_per_launch": {"cfg2": 1021500928, "cfg3": 4713249792, "cfg4": 1486095952, "cfg5": 6073051136},
 }
 
 
 # Lane instructions (warp instructions x 32) per replica-param and step of the temporally blocked kernel, from
 # ncu's smsp__inst_executed.sum of one launch of `bench.py --block-steps 16` (profiles/), keyed by workload.
 BLOCKED_LANE_INSTRUCTIONS = {
-    "kernel_digest": "89b9831650423752",
-    "per_replica_param_step": {"cfg2": 19.33, "cfg3": 20.47, "cfg4": 20.98, "cfg5": 20.56},
+    "kernel_digest": "2894f7e15240b1f2",
+    "per_replica_param_step": {"cfg2": 19.32, "cfg3": 20.46, "cfg4": 20.97, "cfg5": 20.56},
 }
 
 
@@ -71,7 +71,7 @@ def kernel_digest() -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_1810_07766_b200", "csrc")
     # the fused kernels, their arithmetic and the choice of the default shape
-    for name in ("rps_device.cuh", "rps_direct.cuh", "rps_staged.cuh", "rps_staged.cu"):
+    for name in ("rps_device.cuh", "rps_tma.cuh", "rps_direct.cuh", "rps_staged.cuh", "rps_staged.cu", "rps_kernels.cu"):
         with open(os.path.join(csrc, name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -265,6 +265,10 @@ def run_cuda(args):
         from dataclasses import replace
 
         w = replace(w, sigma=args.sigma)
+    if args.n is not None:
+        from dataclasses import replace
+
+        w = replace(w, n=args.n, name=f"{w.name}@n={args.n}")
     b = wl.make_targets(w)
     # --shard: the ranks cut ONE model by columns (no exchange: columns never interact); default: one whole
     # model per rank.  `cols` is what this rank holds, `jobs` how many models the ranks process together.
@@ -448,6 +452,7 @@ def main(argv=None):
     ap.add_argument("--workload", choices=("cfg1", "cfg2", "cfg3", "cfg4", "cfg5"), default="cfg2")
     ap.add_argument("--p", type=float, default=None, help="override the drop probability (p sweeps)")
     ap.add_argument("--d", type=int, default=None, help="override the model size (small profiler captures)")
+    ap.add_argument("--n", type=int, default=None, help="override the number of workers (shape sweeps)")
     ap.add_argument("--sigma", type=float, default=None,
                     help="override the noise level (0 = no gradient noise: the step as pure data movement)")
     ap.add_argument("--e2e-steps", type=int, default=20)
