@@ -21,6 +21,7 @@ import statistics
 import sys
 import threading
 import time
+from dataclasses import replace
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
@@ -256,18 +257,12 @@ def run_cuda(args):
 
     w = wl.WORKLOADS[args.workload]
     if args.p is not None:
-        from dataclasses import replace
-
         w = replace(w, p=args.p)
     if args.d is not None:
         w = w.scaled(d=args.d)
     if args.sigma is not None:
-        from dataclasses import replace
-
         w = replace(w, sigma=args.sigma)
     if args.n is not None:
-        from dataclasses import replace
-
         w = replace(w, n=args.n, name=f"{w.name}@n={args.n}")
     b = wl.make_targets(w)
     # --shard: the ranks cut ONE model by columns (no exchange: columns never interact); default: one whole
@@ -409,8 +404,6 @@ def run_reference(args):
 
     w = wl.WORKLOADS[args.workload]
     if args.p is not None:
-        from dataclasses import replace
-
         w = replace(w, p=args.p)
     cols_n = min(w.d, args.reference_columns)
     sample = wl.Workload(w.name, n=w.n, d=cols_n, dtype=w.dtype, p=w.p, gamma=w.gamma, sigma=w.sigma, seed=w.seed,
