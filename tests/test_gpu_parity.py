@@ -451,6 +451,40 @@ def test_full_size_sampled_columns(rps_mod, oracle, name):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
+def test_full_size_whole_run_sampled_columns(rps_mod, oracle, name):
+    """The workload at its full size for its whole run (50, 200, 50 and 100 steps), every drop probability of
+    its sweep, library defaults, free-running from x = 0: the sampled columns against the oracle's own run of
+    those columns, within the T-step bar.  cfg3 runs tracked, as its description asks (distance to the optimum
+    at every step): the trace must be what rps_diag measures on the final state, and must have come down."""
+    w0 = wl.WORKLOADS[name]
+    b = wl.make_targets(w0)
+    cols = sampled_columns(w0, np.random.default_rng(w0.seed + 1000), count=2048)
+    b_cols = np.ascontiguousarray(b[:, cols])
+    tracked = name == "cfg3"
+    for p in (w0.p_sweep or (w0.p,)):
+        want = np.ascontiguousarray(wl.make_initial(w0)[:, cols])
+        for t in range(w0.steps):
+            oracle.step_columns(w0.d, cols, want, b_cols, dtype=w0.dtype, gamma=w0.gamma, sigma=w0.sigma, p=p,
+                                seed=w0.seed, t=t)
+        r = make(rps_mod, w0, p=p)
+        r.set_targets(b)
+        if tracked:
+            r.track(w0.steps)
+        r.step_n(w0.steps)
+        got = r.read()[:, cols]
+        assert r.get_step() == w0.steps
+        assert_close(w0, got, want, BF16_TOL if w0.dtype == "bf16" else RUN_TOL)
+        if tracked:
+            trace = r.read_trace()
+            dist2, cons = r.diag()
+            assert np.allclose(trace[-1], (dist2, cons), rtol=1e-4)
+            assert trace[-1][0] < 0.01 * trace[0][0] and np.isfinite(trace).all()
+        r.close()
+    del b
+    torch.cuda.empty_cache()
+
+
 # ------------------------------------------------------------------ bounded waits
 
 @pytest.mark.parametrize("store_mode", [1, 2, 3])
