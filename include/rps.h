@@ -125,7 +125,7 @@ typedef struct rps_options {
                                  L2 evict-first hint, which leaves the cache to the lines of x
                                  (a retained line of x saves a read and a write-back, one of b
                                  only a read); 0 = the library's choice                        */
-    int32_t launch_overlap;   /* kernel 2: 2 = the fused kernel is launched with programmatic stream
+    int32_t launch_overlap;   /* all kernels: 2 = the fused kernel is launched with programmatic stream
                                  serialization: its CTAs may be placed and set up while the kernel
                                  before it in the stream drains, and wait (griddepcontrol.wait) for
                                  that kernel to complete before they read anything it may have

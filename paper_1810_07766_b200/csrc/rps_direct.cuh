@@ -32,6 +32,13 @@ __global__ void __launch_bounds__(THREADS) rps_fused_direct_kernel(const FusedPa
     T* __restrict__ x = static_cast<T*>(prm.x);
     const T* __restrict__ b = static_cast<const T*>(prm.b);
     const MaskView masks{prm.masks->up, prm.masks->down, prm.masks->inv_cnt};
+    // Launched with programmatic stream serialization this CTA may have been placed while the kernel before
+    // it in the stream was still running: let the kernel after this one do the same, then wait for the one
+    // before to complete (its writes visible) before reading anything from global memory.  At the sizes this
+    // kernel serves a step is as long as a launch, so hiding the launch is most of what there is to gain.
+    // Both are no-ops in a plain launch.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const int64_t warps_total = (int64_t)gridDim.x * (THREADS / 32);
     const int64_t tiles = (prm.d + WARP_COLS - 1) / WARP_COLS;
@@ -115,7 +122,7 @@ __global__ void __launch_bounds__(THREADS) rps_fused_direct_kernel(const FusedPa
 constexpr int kThreads = 256;
 
 template <typename T, int VEC, int WPT, int G, bool GRAD = false, bool DIAG = false>
-cudaError_t launch_direct_as(const FusedParams& prm, int sm_count, cudaStream_t stream)
+cudaError_t launch_direct_as(const FusedParams& prm, int sm_count, cudaStream_t stream, bool overlap = true)
 {
     constexpr int warp_cols = (32 / G) * VEC;
     const int64_t tiles = (prm.d + warp_cols - 1) / warp_cols;
@@ -132,6 +139,19 @@ cudaError_t launch_direct_as(const FusedParams& prm, int sm_count, cudaStream_t 
     int64_t grid = (int64_t)sm_count * per_sm;
     if (grid > ctas_needed) grid = ctas_needed;
     if (grid < 1) grid = 1;
+    if (overlap) {
+        cudaLaunchConfig_t config = {};
+        config.gridDim = dim3((unsigned)grid);
+        config.blockDim = dim3(kThreads);
+        config.dynamicSmemBytes = 0;
+        config.stream = stream;
+        cudaLaunchAttribute attribute[1];
+        attribute[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attribute[0].val.programmaticStreamSerializationAllowed = 1;
+        config.attrs = attribute;
+        config.numAttrs = 1;
+        return cudaLaunchKernelEx(&config, rps_fused_direct_kernel<T, VEC, WPT, G, kThreads, GRAD, DIAG>, prm);
+    }
     rps_fused_direct_kernel<T, VEC, WPT, G, kThreads, GRAD, DIAG><<<(unsigned)grid, kThreads, 0, stream>>>(prm);
     return cudaGetLastError();
 }
@@ -139,15 +159,15 @@ cudaError_t launch_direct_as(const FusedParams& prm, int sm_count, cudaStream_t 
 // The one family of lane shapes (4 workers per lane, 2 for n <= 2) in which the optional forms of the
 // step (gradient averaging, tracking) are built.
 template <typename T, int VEC, bool GRAD, bool DIAG>
-cudaError_t launch_direct_light(const FusedParams& prm, int sm_count, cudaStream_t stream)
+cudaError_t launch_direct_light(const FusedParams& prm, int sm_count, cudaStream_t stream, bool overlap = true)
 {
     const int n = prm.n;
-    if (n <= 2) return launch_direct_as<T, VEC, 2, 1, GRAD, DIAG>(prm, sm_count, stream);
-    if (n <= 4) return launch_direct_as<T, VEC, 4, 1, GRAD, DIAG>(prm, sm_count, stream);
-    if (n <= 8) return launch_direct_as<T, VEC, 4, 2, GRAD, DIAG>(prm, sm_count, stream);
-    if (n <= 16) return launch_direct_as<T, VEC, 4, 4, GRAD, DIAG>(prm, sm_count, stream);
-    if (n <= 32) return launch_direct_as<T, VEC, 4, 8, GRAD, DIAG>(prm, sm_count, stream);
-    return launch_direct_as<T, VEC, 4, 16, GRAD, DIAG>(prm, sm_count, stream);
+    if (n <= 2) return launch_direct_as<T, VEC, 2, 1, GRAD, DIAG>(prm, sm_count, stream, overlap);
+    if (n <= 4) return launch_direct_as<T, VEC, 4, 1, GRAD, DIAG>(prm, sm_count, stream, overlap);
+    if (n <= 8) return launch_direct_as<T, VEC, 4, 2, GRAD, DIAG>(prm, sm_count, stream, overlap);
+    if (n <= 16) return launch_direct_as<T, VEC, 4, 4, GRAD, DIAG>(prm, sm_count, stream, overlap);
+    if (n <= 32) return launch_direct_as<T, VEC, 4, 8, GRAD, DIAG>(prm, sm_count, stream, overlap);
+    return launch_direct_as<T, VEC, 4, 16, GRAD, DIAG>(prm, sm_count, stream, overlap);
 }
 
 }  // namespace

@@ -187,24 +187,24 @@ cudaError_t launch_masks(const MaskParams& prm, int steps, cudaStream_t stream)
 namespace {
 
 template <typename T, int VEC>
-cudaError_t launch_direct_for_n(const FusedParams& prm, int wpt, int sm_count, cudaStream_t stream)
+cudaError_t launch_direct_for_n(const FusedParams& prm, int wpt, int sm_count, cudaStream_t stream, bool overlap)
 {
     const int n = prm.n;
     // the gradient-averaging comparison is built in one family of lane shapes only
-    if (prm.average_gradients) return launch_direct_light<T, VEC, true, false>(prm, sm_count, stream);
+    if (prm.average_gradients) return launch_direct_light<T, VEC, true, false>(prm, sm_count, stream, overlap);
     if (wpt == 4) {
-        if (n <= 4) return launch_direct_as<T, VEC, 4, 1>(prm, sm_count, stream);
-        if (n <= 8) return launch_direct_as<T, VEC, 4, 2>(prm, sm_count, stream);
-        if (n <= 16) return launch_direct_as<T, VEC, 4, 4>(prm, sm_count, stream);
-        if (n <= 32) return launch_direct_as<T, VEC, 4, 8>(prm, sm_count, stream);
-        return launch_direct_as<T, VEC, 4, 16>(prm, sm_count, stream);
+        if (n <= 4) return launch_direct_as<T, VEC, 4, 1>(prm, sm_count, stream, overlap);
+        if (n <= 8) return launch_direct_as<T, VEC, 4, 2>(prm, sm_count, stream, overlap);
+        if (n <= 16) return launch_direct_as<T, VEC, 4, 4>(prm, sm_count, stream, overlap);
+        if (n <= 32) return launch_direct_as<T, VEC, 4, 8>(prm, sm_count, stream, overlap);
+        return launch_direct_as<T, VEC, 4, 16>(prm, sm_count, stream, overlap);
     }
-    if (n <= 2) return launch_direct_as<T, VEC, 2, 1>(prm, sm_count, stream);
-    if (n <= 4) return launch_direct_as<T, VEC, 4, 1>(prm, sm_count, stream);
-    if (n <= 8) return launch_direct_as<T, VEC, 8, 1>(prm, sm_count, stream);
-    if (n <= 16) return launch_direct_as<T, VEC, 8, 2>(prm, sm_count, stream);
-    if (n <= 32) return launch_direct_as<T, VEC, 8, 4>(prm, sm_count, stream);
-    return launch_direct_as<T, VEC, 8, 8>(prm, sm_count, stream);
+    if (n <= 2) return launch_direct_as<T, VEC, 2, 1>(prm, sm_count, stream, overlap);
+    if (n <= 4) return launch_direct_as<T, VEC, 4, 1>(prm, sm_count, stream, overlap);
+    if (n <= 8) return launch_direct_as<T, VEC, 8, 1>(prm, sm_count, stream, overlap);
+    if (n <= 16) return launch_direct_as<T, VEC, 8, 2>(prm, sm_count, stream, overlap);
+    if (n <= 32) return launch_direct_as<T, VEC, 8, 4>(prm, sm_count, stream, overlap);
+    return launch_direct_as<T, VEC, 8, 8>(prm, sm_count, stream, overlap);
 }
 
 }  // namespace
@@ -213,8 +213,9 @@ cudaError_t launch_fused_direct(const FusedParams& prm, const FusedTuning& tune,
                                 cudaStream_t stream)
 {
     if (prm.trace != nullptr) return launch_direct_tracked(prm, bf16, sm_count, stream);
-    if (bf16) return launch_direct_for_n<__nv_bfloat16, 8>(prm, tune.workers_per_lane, sm_count, stream);
-    return launch_direct_for_n<float, 4>(prm, tune.workers_per_lane, sm_count, stream);
+    const bool overlap = tune.launch_overlap != 1;  // programmatic stream serialization unless plain launches are asked for
+    if (bf16) return launch_direct_for_n<__nv_bfloat16, 8>(prm, tune.workers_per_lane, sm_count, stream, overlap);
+    return launch_direct_for_n<float, 4>(prm, tune.workers_per_lane, sm_count, stream, overlap);
 }
 
 cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
