@@ -85,7 +85,7 @@ def fused_kernel_name(args, w) -> str:
         return "rps_fused_direct_kernel"
     ring_built = w.dtype == "bf16" and w.n > 4 and not (args.average_gradients or args.track)
     staged_only = args.workers_per_lane or args.consumer_warps or args.copy_mode or args.slice_bytes
-    if ring_built and (args.kernel == 3 or (args.kernel == 0 and 8 < w.n <= 56 and not staged_only)):
+    if ring_built and (args.kernel == 3 or (args.kernel == 0 and not staged_only)):
         return "rps_fused_ring_kernel"
     return "rps_fused_staged_kernel"
 

@@ -90,12 +90,12 @@ typedef struct rps_options {
                                  2: slices are staged through shared memory by bulk
                                  asynchronous copies issued by a producer warp;
                                  3: the same staging with no producer warp: all 16 warps of a
-                                 CTA compute, in teams that take the tiles in turn, and the last
-                                 warp to have read a stage refills it (built for bf16 replicas
+                                 CTA compute, each taking the next slice of the next tile from a
+                                 counter, and the last warp to have read a stage refills it (built for bf16 replicas
                                  with more than 4 workers, plain untracked model averaging;
                                  any other step runs as kernel 2).
                                  0: kernel 1 for models too short to give every SM a tile, kernel 3
-                                 for bf16 replicas of 9 to 56 workers (unless an option that
+                                 for bf16 replicas of more than 4 workers (unless an option that
                                  shapes kernel 2 alone is set), else kernel 2                 */
     int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */
     int32_t stages;           /* depth of the shared-memory ring of kernels 2 and 3 (2..8)   */
@@ -149,8 +149,8 @@ typedef struct rps_options {
      * between two synchronisations), so it is off by default (0 or 1); it applies to rps_step_n only,
      * and only to untracked model averaging.                                                         */
     int32_t block_steps;
-    int32_t team_warps;       /* kernel 3: warps that share a tile: 1, 2, 4, 8 or 16 (0 = the library's
-                                 choice: the largest that leaves room for one more stage than teams) */
+    int32_t team_warps;       /* kernel 3: warp slices per tile, 1..16 (0 = the library's choice: 8, or
+                                 fewer where the ring would otherwise be too shallow)             */
 } rps_options;
 
 /*

@@ -433,9 +433,8 @@ int rps_configure(rps_handle* h, const rps_options* opt)
         return fail(h, RPS_EINVAL, "a shard starts at a multiple of 64 and ends inside the model");
     if (opt->block_steps < 0 || opt->block_steps > opt->mask_window)
         return fail(h, RPS_EINVAL, "block_steps must be in 0..mask_window");
-    if (opt->team_warps != 0 && opt->team_warps != 1 && opt->team_warps != 2 && opt->team_warps != 4 &&
-        opt->team_warps != 8 && opt->team_warps != 16)
-        return fail(h, RPS_EINVAL, "team_warps must be 0 (auto), 1, 2, 4, 8 or 16");
+    if (opt->team_warps < 0 || opt->team_warps > 16)
+        return fail(h, RPS_EINVAL, "team_warps must be 0 (auto) or 1..16");
     h->opt = *opt;
     h->sigma = (float)opt->sigma;
     return RPS_OK;

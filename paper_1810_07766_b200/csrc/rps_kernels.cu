@@ -230,11 +230,9 @@ cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool b
         if (prm.d * bytes_per_column < (int64_t)sm_count * 8192)
             return launch_fused_direct(prm, tune, bf16, sm_count, stream);
     }
-    // bf16 replicas of 9 to 56 workers: the self-refilling ring (16 compute warps, no producer warp), unless an
-    // option that shapes the staged kernel only was set.  Measured side by side it is 2-5 % ahead where its
-    // ring holds four or more tiles of 8 warps (n <= 56) and level or behind with three (n = 64) or with the
-    // long rows of n <= 8.
-    if (tune.kernel == 0 && bf16 && prm.n > 8 && prm.n <= 56 && ring_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 &&
+    // bf16 replicas of more than 4 workers: the self-refilling ring (16 compute warps, no producer warp), unless an
+    // option that shapes the staged kernel only was set.  Measured side by side it is 3-8 % ahead at every n.
+    if (tune.kernel == 0 && bf16 && ring_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 &&
         tune.consumer_warps == 0 && tune.copy_mode == 0 && tune.slice_bytes == 0)
         return launch_fused_ring(prm, tune, bf16, sm_count, stream);
     return launch_fused_staged(prm, tune, bf16, sm_count, stream);

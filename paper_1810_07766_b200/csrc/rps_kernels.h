@@ -35,7 +35,7 @@ struct FusedTuning {
     int32_t traversal;         // 0 odd steps walk the tiles downwards, 1 always upwards
     int32_t l2_policy;         // staged kernel: 1 plain loads, 2 targets loaded with the L2 evict-first hint
     int32_t launch_overlap;    // staged kernel: 1 plain launch, 2 programmatic stream serialization
-    int32_t team_warps;        // ring kernel: warps that share a tile (1, 2, 4, 8 or 16)
+    int32_t team_warps;        // ring kernel: warp slices per tile (1..16)
 };
 
 struct FusedParams {

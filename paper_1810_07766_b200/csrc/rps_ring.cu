@@ -5,13 +5,14 @@
 // handed out by warp scheduler: 16 warps of 128 registers fill it, a 17th warp (a producer) would cut every
 // warp to 96.  So here every warp computes and nobody only produces:
 //
-//   * A tile is team_warps x WARP_COLS columns of all n rows of x and b, one warp per slice of WARP_COLS
-//     columns; the 16 warps of a CTA are 16 / team_warps warps for every slice position, so that many tiles
-//     are worked on at a time.  Tile L of the CTA lives in stage L mod stages of a shared-memory ring filled
-//     by TMA box copies (cp.async.bulk.tensor.2d, completion on the stage's mbarrier).  Tiles of 8 warps
-//     (64 KB at n = 64) instead of 16 are what lets a ring of three stages fit beside 16 compute warps.
-//     A warp that is free takes the next tile of its slice position from a counter: no warp is tied to
-//     particular tiles, so a warp that fell behind is not waited for by the warps of other tiles.
+//   * A tile is team_warps x WARP_COLS columns of all n rows of x and b, cut into team_warps slices of
+//     WARP_COLS columns, one warp's work each.  Tile L of the CTA lives in stage L mod stages of a
+//     shared-memory ring filled by TMA box copies (cp.async.bulk.tensor.2d, completion on the stage's
+//     mbarrier).  Tiles of 8 slices (64 KB at n = 64) instead of 16 are what lets a ring of three stages fit
+//     beside 16 compute warps.
+//   * A warp that is free takes the next slice of the next tile from one counter: no warp is tied to a tile
+//     or to a position in it, so 16 warps share tiles of any number of slices evenly, about 16 / team_warps
+//     tiles are in work at a time, and a warp that fell behind holds nobody up.
 //   * A warp copies its slices of the stage to registers and counts itself off on the stage's counter
 //     (a shared-memory atomic).  The warp that counts last knows the stage is free: it resets the
 //     counter and issues the copies of the tile that comes `stages` tiles later, then goes on computing.
@@ -45,8 +46,8 @@ struct RingShape {
     int64_t tiles;
     int32_t x_stages;       // depth of the ring of x tiles
     int32_t b_stages;       // depth of the ring of b tiles (the same, and filled together, unless results go back in place)
-    int32_t team_warps;     // warps that share a tile
-    int32_t teams;          // warps of the CTA / team_warps
+    int32_t team_warps;     // warp slices per tile
+    int32_t teams;          // tiles in work at a time: warps of the CTA / team_warps, rounded up
     int32_t tile_cols;      // team_warps x WARP_COLS
     int32_t box_cols;       // columns per TMA box (<= 256); a tile is boxes_per_tile boxes side by side
     int32_t boxes_per_tile;
@@ -137,12 +138,11 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
     unsigned char* b_ring = x_ring + shape.b_ring_offset;
     int* out_done = reinterpret_cast<int*>(smem + 256);                    // [teams] warps that have written their results
     volatile int* out_free = reinterpret_cast<volatile int*>(smem + 320);  // [teams] stores that have left the output tile
-    int* next_tile = reinterpret_cast<int*>(smem + 384);                   // [team_warps] next tile of each slice position
+    int* next_item = reinterpret_cast<int*>(smem + 384);                   // next (tile, slice) of the CTA that no warp has taken
 
     const int n = prm.n;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const int slot = warp % shape.team_warps;  // which slice of WARP_COLS columns of a tile this warp works on
     const bool in_place = shape.store_mode == 3, out_tiles = shape.store_mode == 2;
     // tiles of this CTA: turns blockIdx.x, blockIdx.x + gridDim.x, ...
     const int64_t my_tiles =
@@ -155,7 +155,8 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
             xs.done[s] = bs.done[s] = 0;
             xs.fills[s] = bs.fills[s] = 0;
         }
-        for (int k = 0; k < kRingWarps; ++k) out_done[k] = out_free[k] = next_tile[k] = 0;
+        for (int k = 0; k < kRingWarps; ++k) out_done[k] = out_free[k] = 0;
+        *next_item = 0;
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
@@ -215,9 +216,6 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
     const MaskView masks{s_up, s_down, s_inv};
     const int sub = lane % LPG;
     const int w_first = (lane / LPG) * WPT;
-    const int col_in_tile = slot * WARP_COLS + sub * VEC;
-    const uint32_t lane_off =
-        (uint32_t)(col_in_tile / shape.box_cols) * shape.box_bytes + (uint32_t)(col_in_tile % shape.box_cols) * elem;
     BlockCursor cursor;
     bool stores_pending = false;
     // What a warp does when something it waited for never came: say so, stop the refilling, and see the
@@ -238,11 +236,16 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
         if (stores_pending) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     };
     for (;;) {
-        // the next tile of the CTA that no warp has taken at this slice position
-        int taken = 0;
-        if (lane == 0) taken = atomicAdd(&next_tile[slot], 1);
-        const int64_t local = __shfl_sync(0xFFFFFFFFu, taken, 0);
+        // the next slice of WARP_COLS columns, of the next tile of the CTA, that no warp has taken
+        uint32_t taken = 0;
+        if (lane == 0) taken = (uint32_t)atomicAdd(next_item, 1);
+        taken = __shfl_sync(0xFFFFFFFFu, taken, 0);
+        const int64_t local = taken / (uint32_t)shape.team_warps;
         if (local >= my_tiles) break;
+        const int slot = (int)(taken % (uint32_t)shape.team_warps);
+        const int col_in_tile = slot * WARP_COLS + sub * VEC;
+        const uint32_t lane_off =
+            (uint32_t)(col_in_tile / shape.box_cols) * shape.box_bytes + (uint32_t)(col_in_tile % shape.box_cols) * elem;
         const RingCursor at_x((uint32_t)local, (uint32_t)shape.x_stages), at_b((uint32_t)local, (uint32_t)shape.b_stages);
         if (!__all_sync(0xFFFFFFFFu, (!in_place || at_x.wait(xs, shape.wait_limit_ns)) && at_b.wait(bs, shape.wait_limit_ns))) {
             give_up(2);
@@ -339,20 +342,19 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
     if (stores_pending) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
-// Teams, tiles and ring depths for one instantiation: the team size asked for if rings of two stages fit,
-// else the largest team (from 8 warps down) whose tiles leave room for one more stage than teams.
+// Tiles and ring depths for one instantiation: the number of slices per tile asked for if rings of two
+// stages fit, else the largest (from 8 down) whose tiles leave room for as many stages as tiles are in work.
 bool plan_ring(const FusedParams& prm, const FusedTuning& tune, int vec, int g, size_t elem, size_t smem_limit,
                RingShape* sh, uint32_t* smem_bytes)
 {
     const int warp_cols = (32 / g) * vec;
     int team_warps = tune.team_warps > 0 ? tune.team_warps : 8;
     if (team_warps > kRingWarps) team_warps = kRingWarps;
-    while (kRingWarps % team_warps != 0) --team_warps;
     const int team_asked = team_warps;
     sh->store_mode = tune.store_mode != 0 ? tune.store_mode : kRingDefaultStoreMode;
-    for (; team_warps >= 1; team_warps /= 2) {
+    for (; team_warps >= 1; team_warps = team_warps > 8 ? 8 : team_warps / 2) {
         sh->team_warps = team_warps;
-        sh->teams = kRingWarps / team_warps;
+        sh->teams = (kRingWarps + team_warps - 1) / team_warps;  // tiles in work at a time, rounded up
         sh->tile_cols = team_warps * warp_cols;
         // the widest box (<= 256 elements) that tiles the tile exactly; warp_cols always does
         int box_cols = warp_cols;

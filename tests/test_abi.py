@@ -70,7 +70,7 @@ def test_options_pitch_and_state_errors(lib):
                              ("stages", 9), ("consumer_warps", 25), ("slice_bytes", 4), ("store_mode", 4), ("wait_limit_ms", -1), ("withhold_copies", 2), ("average", 2), ("row_skew_lines", -2), ("copy_mode", 3),
                              ("traversal", 2), ("l2_policy", 3), ("launch_overlap", 3),
                              ("shard_cols", -1), ("shard_begin", 64), ("shard_cols", 11_173_963),
-                             ("block_steps", -1), ("block_steps", 33), ("team_warps", 3), ("team_warps", 32)):
+                             ("block_steps", -1), ("block_steps", 33), ("team_warps", -1), ("team_warps", 17)):
             bad = rps_options()
             lib.rps_default_options(ctypes.byref(bad))
             setattr(bad, field, value)

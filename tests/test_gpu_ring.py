@@ -56,7 +56,7 @@ def test_ring_equals_the_staged_kernel_bit_for_bit_and_the_oracle(rps_mod, oracl
     oracle.run(want, b, dtype="bf16", gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=3, steps=w.steps)
     ref = run(rps_mod, w, b, x0, w.steps, t0=3, kernel=2, workers_per_lane=8, store_mode=1)
     for store_mode in (1, 2, 3):  # from registers; TMA tensor stores from an output tile; from the x tile in place
-        for team_warps, stages in ((0, 0), (1, 2), (2, 0), (4, 3), (8, 2), (16, 0), (4, 8)):
+        for team_warps, stages in ((0, 0), (1, 2), (2, 0), (4, 3), (8, 2), (16, 0), (4, 8), (12, 0), (3, 5), (7, 2)):
             got = run(rps_mod, w, b, x0, w.steps, t0=3, kernel=3, team_warps=team_warps, stages=stages,
                       store_mode=store_mode)
             assert (got == ref).all(), (store_mode, team_warps, stages, int((got != ref).sum()))
