@@ -22,6 +22,8 @@
  *                        paper fixes only zero mean and bounded variance
  *                        (Assumption 1), so its exact values are a convention of
  *                        this implementation: parity unpinned by the paper for that part
+ *   run, run_gradavg     equal to repeated single steps with step indices t0, t0+1, ... bit for
+ *                        bit (a late, repeated or skipped index fails), cut points, closed form
  *   bf16 rounding        library conversion on random inputs
  *   alpha_mc             exact alpha_1, alpha_2 from all drop patterns on tiny n (within the
  *                        sampling error), 0 and 1 at p = 0 and p = 1, a second route to the
@@ -113,7 +115,7 @@ static void assign_servers(int n, uint64_t seed, uint64_t t, int assign, int32_t
 {
     for (int j = 0; j < n; ++j) server[j] = j;
     if (assign != RPS_ORACLE_ASSIGN_PERM) return;
-    /* Fisher-Yates shuffle: a uniform draw "without replacement". */
+    /* Fisher-Yates shuffle: every assignment of servers to blocks equally likely, no worker twice. */
     for (int k = n - 1; k >= 1; --k) {
         uint32_t r[4];
         philox_draw(seed, t, (uint32_t)k, STREAM_PERM, r);
@@ -128,8 +130,9 @@ static void assign_servers(int n, uint64_t seed, uint64_t t, int assign, int32_t
  * Drop masks of step t.  Bit i of up[j]   = worker i's block j reached its server.
  *                        Bit i of down[j] = worker i received the averaged block j.
  * With self_delivery the server's own copy never crosses the network, so its
- * two bits are always 1 (proof of Lemma 7: the server "must receive its own
- * block"; Case 2: "node n's block is always received by itself").  Without it
+ * two bits are always 1 (proof of Lemma 7: a server always holds its own copy of
+ * the block; proof of Lemma 8, Case 2: a node's own block needs no message to
+ * reach it).  Without it
  * all 2n messages of a block can be lost; if nothing arrives there is no
  * average to send, so nobody receives one (down = 0) and every worker keeps v.
  * cnt[j] = |N_t^(j)|.
