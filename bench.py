@@ -1,12 +1,15 @@
 #!/usr/bin/env python
 """Benchmark of the RPS synchronisation step.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--p 0.1]
-    python bench.py --impl reference ...        # the CPU oracle on the host cores
+    python bench.py [--gpus N] [--steps K] [--warmup W]            # every workload, cfg3 as the headline
+    python bench.py --workload cfg5 [--p 0.1] [--kernel 3 ...]     # one workload (sweeps, profiler captures)
+    python bench.py --impl reference ...                           # the CPU oracle on the host cores
 
 A step is one pass of the whole hot path (drop masks, local SGD step, masked
 average, masked write-back) over all n replicas.  The metric is replica-params
-synchronised per second, n*d per step.  With N > 1 (torchrun, one rank per GPU)
+synchronised per second, n*d per step.  Without --workload the line's top-level
+fields describe the headline workload (the largest fp32 model) and `workloads`
+holds every configuration, the swept ones with each drop probability.  With N > 1 (torchrun, one rank per GPU)
 every rank runs an independent replica of the job: the path needs no exchange
 between GPUs, so there is no collective on the data path; only the timing is
 reduced (max over ranks).  Prints ONE JSON line on rank 0.
@@ -72,7 +75,8 @@ def kernel_digest() -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_1810_07766_b200", "csrc")
     # the fused kernels, their arithmetic and the choice of the default shape
-    for name in ("rps_device.cuh", "rps_tma.cuh", "rps_staged.cuh", "rps_staged.cu", "rps_ring.cu", "rps_kernels.cu"):
+    for name in ("rps_device.cuh", "rps_tma.cuh", "rps_staged.cuh", "rps_staged.cu", "rps_ring.cu", "rps_stream.cu",
+                 "rps_kernels.cu"):
         with open(os.path.join(csrc, name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -83,6 +87,10 @@ def fused_kernel_name(args, w) -> str:
     small = w.n * w.d * w.elem_bytes < 148 * 8192
     if args.kernel == 1 or (args.kernel == 0 and small):
         return "rps_fused_direct_kernel"
+    stream_built = w.n >= 2 and not (args.average_gradients or args.track)
+    staged_only = args.workers_per_lane or args.copy_mode or args.slice_bytes
+    if stream_built and (args.kernel == 4 or (args.kernel == 0 and w.dtype == "bf16" and w.n > 32 and not staged_only)):
+        return "rps_fused_stream_kernel"
     ring_built = w.dtype == "bf16" and w.n > 4 and not (args.average_gradients or args.track)
     staged_only = args.workers_per_lane or args.consumer_warps or args.copy_mode or args.slice_bytes
     if ring_built and (args.kernel == 3 or (args.kernel == 0 and not staged_only)):
@@ -236,10 +244,184 @@ def oracle_baseline(w, b, min_seconds=10.0, max_steps=8):
             "sample": f"{steps} full-size step(s) (n={w.n}, d={w.d}) of the fp64 C oracle, {dt:.2f} s, single thread"}
 
 
+# The workloads of a default run, the headline first: the largest fp32 model (d >= 11M; its L2 carry-over
+# between steps is the smallest of the fp32 workloads), then the other configurations, the swept ones once per
+# drop probability of their sweep.
+HEADLINE = "cfg3"
+DEFAULT_SUITE = ("cfg3", "cfg2", "cfg4", "cfg5")
+
+
+def resolve_workload(args, name, p=None):
+    from paper_1810_07766_b200 import workloads as wl
+
+    w = wl.WORKLOADS[name]
+    if p is not None:
+        w = replace(w, p=p)
+    if args.d is not None:
+        w = w.scaled(d=args.d)
+    if args.sigma is not None:
+        w = replace(w, sigma=args.sigma)
+    if args.n is not None:
+        w = replace(w, n=args.n, name=f"{w.name}@n={args.n}")
+    return w
+
+
+def measure(args, ctx, w, b, *, with_e2e, with_upwards, p_sweep=()):
+    """Times one workload on this rank's GPU.  Returns its entry of the JSON line.
+
+    Pass 1 brackets every launch with events (per-kernel durations; this serialises what the programmatic launch
+    overlap hides, so the mean launch can be longer than the step it is part of), pass 2 is W warm-up steps and
+    exactly K timed steps, pass 3 (optional) the same steps through the host-buffer call.  `p_sweep`: further drop
+    probabilities timed on the same arrays (pass 2 only).
+    """
+    import numpy as np
+
+    from paper_1810_07766_b200 import binding
+
+    torch, device, rank, local_rank, world = ctx["torch"], ctx["device"], ctx["rank"], ctx["local_rank"], ctx["world"]
+    begin, cols, jobs = 0, w.d, world
+    if args.shard and world > 1:
+        begin, cols = binding.shard_columns(w.d, world, rank)
+        if cols == 0:
+            raise SystemExit("--shard: the model is too short for this many ranks")
+        b = np.ascontiguousarray(b[:, begin:begin + cols])
+        jobs = 1
+    sharded = jobs != world
+    shape = {name: getattr(args, name) for name in SHAPE_OPTIONS}  # all 0 = the library's choice
+    bytes_per_step = w.bytes_per_step * cols // w.d
+
+    def make(p, **more):
+        r = binding.RPS(w.n, w.d, p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma,
+                        average_gradients=args.average_gradients, shard_begin=begin if sharded else 0,
+                        shard_cols=cols if sharded else 0, row_skew_lines=args.row_skew_lines, **{**shape, **more})
+        r.set_targets(b)
+        if args.track:  # every step of the run also records the distance to the optimum and the consensus error
+            r.track(2 * max(args.warmup, 3) + 2 * args.steps + args.warmup + 64)
+        return r
+
+    def timed_run(r):
+        r.step_n(args.warmup)
+        before = r.launch_count()
+        ms = timed_steps(torch, r.stream, lambda: r.step_n(args.steps), device)
+        return ms, r.launch_count() - before
+
+    r = make(w.p)
+    # the clocks are sampled from here to the end of the timed steps: an NVML query takes milliseconds, so
+    # the timed region alone (tens of milliseconds) would yield a single sample
+    with ClockSampler(local_rank) as clocks:
+        r.step_n(max(args.warmup, 3))
+        r.profile(True)
+        r.step_n(args.steps)
+        fused_ms, fused_n, mask_ms, mask_n = r.profile_read()
+        r.profile(False)
+        total_ms, gpu_launches = timed_run(r)
+
+    e2e = None
+    if with_e2e:
+        tdtype = torch.float32 if w.dtype == "f32" else torch.int16  # bf16 bit patterns travel as 16-bit words
+        x_host = torch.zeros((w.n, cols), dtype=tdtype).pin_memory()
+        b_host = torch.from_numpy(b if w.dtype == "f32" else b.view(np.int16)).pin_memory()
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        for _ in range(2):
+            r.step_host(x_host, b_host)
+        e2e_ms = timed_steps(torch, r.stream, lambda: [r.step_host(x_host, b_host) for _ in range(e2e_steps)], device)
+        e2e = {"value": jobs * w.n * w.d * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
+               "h2d_bytes_per_step": 2 * w.n * cols * w.elem_bytes, "d2h_bytes_per_step": w.n * cols * w.elem_bytes,
+               "call": "rps_step_host (pinned host x and b)"}
+        del x_host, b_host
+    r.close()
+
+    ms_per_step = total_ms / args.steps
+    peak, peak_kind = measured_peak_gbs()
+    fused_avg_ms = fused_ms / max(fused_n, 1)
+    achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
+    whole_step = bytes_per_step / (ms_per_step * 1e-3) / 1e9
+    traffic = traffic_cold = None
+    default_shape = not (any(shape.values()) or args.average_gradients or args.track or sharded or
+                         args.row_skew_lines != -1)
+    if default_shape and NCU_TRAFFIC["kernel_digest"] == kernel_digest():
+        traffic = NCU_TRAFFIC["bytes_per_launch"].get(w.name)
+        traffic_cold = NCU_TRAFFIC["cold_bytes_per_launch"].get(w.name)
+    mask_window = 32  # steps whose masks one launch of the mask kernel generates (rps_options.mask_window)
+    roofline = {
+        "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+        "traffic": traffic, "traffic_cold_cache": traffic_cold, "peak_kind": f"of {peak_kind}",
+        "kernel": fused_kernel_name(args, w), "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n,
+        # the same bytes over the time of a whole step inside a train of steps (launch overlap kept, mask kernel in)
+        "whole_step_achieved": whole_step, "whole_step_frac": whole_step / peak,
+        "whole_step_frac_of_8TBs_nominal": whole_step / 8000.0,
+        # what crossed the HBM interface (ncu, when recorded for these sources) over the same times
+        "dram_achieved": traffic / (fused_avg_ms * 1e-3) / 1e9 if traffic else None,
+        "dram_frac": traffic / (fused_avg_ms * 1e-3) / 1e9 / peak if traffic else None,
+        "dram_whole_step_achieved": traffic / (ms_per_step * 1e-3) / 1e9 if traffic else None,
+        "dram_whole_step_frac_of_8TBs_nominal": traffic / (ms_per_step * 1e-3) / 8e12 if traffic else None,
+        "note": "avg_launch_ms brackets every launch with events, which serialises the launches and loses the "
+                "programmatic launch overlap a train of steps has: it can exceed ms_per_step",
+        "mask_kernel_ms_per_launch": mask_ms / max(mask_n, 1) if mask_n else None,
+        "mask_kernel_ms_per_step_amortised": mask_ms / mask_n / mask_window if mask_n else None,
+        "mask_launches_timed": mask_n,
+    }
+    entry = {
+        "workload": f"{w.name}: n={w.n} workers, d={w.d} {w.dtype}, p={w.p}, gamma={w.gamma}, sigma={w.sigma}, "
+                    f"seed={w.seed}; quadratic objective, b_i ~ N({'mu_i' if w.hetero else '0'},1)",
+        "n": w.n, "d": w.d, "p": w.p, "dtype": w.dtype, "cols_on_this_gpu": cols,
+        "value": jobs * w.n * w.d * args.steps / (total_ms * 1e-3), "unit": UNIT, "ms_per_step": ms_per_step,
+        "algorithmic_bytes_per_step": bytes_per_step, "hbm_gbs_whole_step": whole_step,
+        "frac_of_8TBs_nominal": whole_step / 8000.0,
+        "l2": "inputs larger than L2 (x and b are %.0f MB each)" % (w.n * cols * w.elem_bytes / 1e6),
+        "clocks": clocks.summary(), "gpu_launches": gpu_launches, "roofline": roofline, "e2e": e2e,
+        "sharded": sharded, "kernel_shape": shape,
+    }
+    if p_sweep:
+        entry["p_sweep"] = {}
+        for p in p_sweep:
+            rp = make(p)
+            ms, _ = timed_run(rp)
+            rp.close()
+            entry["p_sweep"][str(p)] = {"ms_per_step": ms / args.steps,
+                                        "value": jobs * w.n * w.d * args.steps / (ms * 1e-3),
+                                        "hbm_gbs_whole_step": bytes_per_step / (ms / args.steps * 1e-3) / 1e9}
+    if with_upwards:
+        # every step walks the columns upwards: no step starts on what the step before it left in L2
+        ru = make(w.p, traversal=1)
+        ms, _ = timed_run(ru)
+        ru.close()
+        entry["traversal_always_upwards"] = {"ms_per_step": ms / args.steps,
+                                             "hbm_gbs_whole_step": bytes_per_step / (ms / args.steps * 1e-3) / 1e9,
+                                             "frac_of_8TBs_nominal": bytes_per_step / (ms / args.steps * 1e-3) / 8e12}
+    torch.cuda.empty_cache()
+    return entry
+
+
+def blocked_roofline(args, ctx, w, cols, entry):
+    """Several steps per pass over x and b: the pass is bound by the arithmetic of a step, not by HBM.
+    achieved = lane instructions executed per second (ncu's count per replica-param and step, recorded above
+    with the digest of the kernel sources, x replica-params x steps per second); peak = one warp instruction of
+    32 lanes per scheduler and clock."""
+    torch, device = ctx["torch"], ctx["device"]
+    old = entry["roofline"]
+    fused_avg_ms, fused_n = old["avg_launch_ms"], old["launches_timed"]
+    steps_per_launch = args.steps / max(fused_n, 1)
+    rp_steps_per_s = w.n * cols * steps_per_launch / (fused_avg_ms * 1e-3)
+    sm_count = torch.cuda.get_device_properties(device).multi_processor_count
+    mhz = entry["clocks"].get("sm_max_mhz") or 1965
+    peak_alu = sm_count * 4 * 32 * mhz * 1e6 / 1e12
+    instr = None
+    if BLOCKED_LANE_INSTRUCTIONS["kernel_digest"] == blocked_kernel_digest():
+        instr = BLOCKED_LANE_INSTRUCTIONS["per_replica_param_step"].get(w.name)
+    alu = instr * rp_steps_per_s / 1e12 if instr else None
+    return {"bound": "alu", "achieved": alu, "peak": peak_alu, "unit": "T lane-instructions/s",
+            "frac": alu / peak_alu if alu else None, "traffic": None,
+            "peak_kind": "derived: SMs x 4 schedulers x 32 lanes x max SM clock",
+            "kernel": "rps_fused_blocked_kernel", "lane_instructions_per_replica_param_step": instr,
+            "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n, "steps_per_launch": steps_per_launch,
+            "hbm_gbs_moved_per_launch": 3 * w.elem_bytes * w.n * cols / (fused_avg_ms * 1e-3) / 1e9}
+
+
 def run_cuda(args):
     import torch
 
-    from paper_1810_07766_b200 import binding, build
+    from paper_1810_07766_b200 import build
     from paper_1810_07766_b200 import workloads as wl
 
     rank, local_rank, world = dist_env()
@@ -256,134 +438,59 @@ def run_cuda(args):
 
         dist.init_process_group("nccl", device_id=device)
     build.build()
-    import numpy as np
+    ctx = {"torch": torch, "device": device, "rank": rank, "local_rank": local_rank, "world": world}
 
-    w = wl.WORKLOADS[args.workload]
-    if args.p is not None:
-        w = replace(w, p=args.p)
-    if args.d is not None:
-        w = w.scaled(d=args.d)
-    if args.sigma is not None:
-        w = replace(w, sigma=args.sigma)
-    if args.n is not None:
-        w = replace(w, n=args.n, name=f"{w.name}@n={args.n}")
-    b = wl.make_targets(w)
-    # --shard: the ranks cut ONE model by columns (no exchange: columns never interact); default: one whole
-    # model per rank.  `cols` is what this rank holds, `jobs` how many models the ranks process together.
-    begin, cols, jobs = 0, w.d, world
-    if args.shard and world > 1:
-        begin, cols = binding.shard_columns(w.d, world, rank)
-        if cols == 0:
-            raise SystemExit("--shard: the model is too short for this many ranks")
-        b = np.ascontiguousarray(b[:, begin:begin + cols])
-        jobs = 1
-    sharded = jobs != world
-    # the kernel-shape options, all 0 = the library's choice
-    shape = {name: getattr(args, name) for name in SHAPE_OPTIONS}
-    r = binding.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma,
-                    average_gradients=args.average_gradients, shard_begin=begin if sharded else 0,
-                    shard_cols=cols if sharded else 0, **shape)
-    r.set_targets(b)
-    if args.track:
-        # every step of the run also records the distance to the optimum and the consensus error
-        r.track(2 * max(args.warmup, 3) + 2 * args.steps + args.warmup + 64)
-    stream = r.stream
-    bytes_per_step = w.bytes_per_step * cols // w.d
-
-    # the clocks are sampled from here to the end of the timed steps: an NVML query takes milliseconds, so
-    # the timed region alone (tens of milliseconds) would yield a single sample
-    with ClockSampler(local_rank) as clocks:
-        # pass 1 (untimed for `value`): every launch bracketed by events -> per-kernel durations
-        r.step_n(max(args.warmup, 3))
-        r.profile(True)
-        r.step_n(args.steps)
-        fused_ms, fused_n, mask_ms, mask_n = r.profile_read()
-        r.profile(False)
-
-        # pass 2: W warm-up steps, then exactly K timed steps
-        r.step_n(args.warmup)
-        launches_before = r.launch_count()
-        total_ms = timed_steps(torch, stream, lambda: r.step_n(args.steps), device)
-        gpu_launches = r.launch_count() - launches_before
-
-    # pass 3: end to end through the host-buffer call: H2D of x and b, the step, D2H of x, every step
-    e2e = None
-    if not args.skip_e2e:
-        tdtype = torch.float32 if w.dtype == "f32" else torch.int16  # bf16 bit patterns travel as 16-bit words
-        x_host = torch.zeros((w.n, cols), dtype=tdtype).pin_memory()
-        b_host = torch.from_numpy(b if w.dtype == "f32" else b.view(np.int16)).pin_memory()
-        e2e_steps = max(1, min(args.steps, args.e2e_steps))
-        for _ in range(2):
-            r.step_host(x_host, b_host)
-        e2e_ms = timed_steps(torch, stream, lambda: [r.step_host(x_host, b_host) for _ in range(e2e_steps)], device)
-        e2e = {"value": jobs * w.n * w.d * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
-               "h2d_bytes_per_step": 2 * w.n * cols * w.elem_bytes, "d2h_bytes_per_step": w.n * cols * w.elem_bytes,
-               "call": "rps_step_host (pinned host x and b)"}
-    row_bytes = w.n * cols * w.elem_bytes
-
+    # one workload when one is named (tuning sweeps, profiler captures), else the whole suite with the headline first
+    names = (args.workload,) if args.workload else DEFAULT_SUITE
+    headline = names[0]
+    entries, cpu = {}, None
+    for name in names:
+        sweep = wl.WORKLOADS[name].p_sweep if (args.workload is None and args.p is None) else ()
+        w = resolve_workload(args, name, args.p)
+        b = wl.make_targets(w)
+        first = name == headline
+        entry = measure(args, ctx, w, b, with_e2e=first and not args.skip_e2e,
+                        with_upwards=first and args.workload is None and args.traversal == 0,
+                        p_sweep=tuple(p for p in sweep if p != w.p))
+        if args.block_steps > 1:
+            entry["roofline"] = blocked_roofline(args, ctx, w, entry["cols_on_this_gpu"], entry)
+        if first and rank == 0 and world == 1 and not args.no_cpu_baseline:
+            cpu = oracle_baseline(w, b)
+        entries[name] = entry
+        del b
     copy_gbs = in_situ_copy_gbs(torch, device)
-    peak, peak_kind = measured_peak_gbs()
-    fused_avg_ms = fused_ms / max(fused_n, 1)
-    achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
-    traffic = traffic_cold = None
-    default_shape = not (any(shape.values()) or args.average_gradients or args.track or sharded)
-    if default_shape and NCU_TRAFFIC["kernel_digest"] == kernel_digest():
-        traffic = NCU_TRAFFIC["bytes_per_launch"].get(w.name)
-        traffic_cold = NCU_TRAFFIC["cold_bytes_per_launch"].get(w.name)
 
+    top = entries[headline]
     line = {
-        "metric": METRIC, "value": jobs * w.n * w.d * args.steps / (total_ms * 1e-3), "unit": UNIT,
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
-        "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
-        "dtype": w.dtype, "data": "synthetic",
+        "metric": METRIC, "value": top["value"], "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": top["ms_per_step"],
+        "higher_is_better": True, "scaling": "strong" if top["sharded"] else "weak", "vs_baseline": None,
+        "dtype": top["dtype"], "data": "synthetic",
         "config": {
-            "workload": f"{w.name}: n={w.n} workers, d={w.d} {w.dtype}, p={w.p}, gamma={w.gamma}, sigma={w.sigma}, "
-                        f"seed={w.seed}; quadratic objective, b_i ~ N({'mu_i' if w.hetero else '0'},1)",
-            "n": w.n, "d": w.d, "p": w.p,
-            "replicas": ("one model cut by columns over the GPUs, no collective" if sharded
+            "workload": top["workload"], "n": top["n"], "d": top["d"], "p": top["p"],
+            "replicas": ("one model cut by columns over the GPUs, no collective" if top["sharded"]
                          else "one independent job per GPU, no collective"),
-            "kernel_shape": shape,
+            "kernel_shape": top["kernel_shape"],
             "average": "gradients" if args.average_gradients else "models",
             "tracked": bool(args.track),
-            "l2": "inputs larger than L2 (x and b are %.0f MB each)" % (row_bytes / 1e6),
-            "algorithmic_bytes_per_step": bytes_per_step,
-            "hbm_gbs_whole_step": bytes_per_step / (total_ms / args.steps * 1e-3) / 1e9,
-            "frac_of_8TBs_nominal": bytes_per_step / (total_ms / args.steps * 1e-3) / 8e12,
+            "l2": top["l2"],
+            "algorithmic_bytes_per_step": top["algorithmic_bytes_per_step"],
+            "hbm_gbs_whole_step": top["hbm_gbs_whole_step"],
+            "frac_of_8TBs_nominal": top["frac_of_8TBs_nominal"],
         },
-        "clocks": clocks.summary(),
-        "e2e": e2e,
-        "gpu_launches": gpu_launches,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "traffic_cold_cache": traffic_cold, "peak_kind": f"of {peak_kind}",
-                     "kernel": fused_kernel_name(args, w),
-                     "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n,
-                     "mask_kernel_ms_per_launch": mask_ms / max(mask_n, 1), "mask_launches_timed": mask_n,
-                     "in_situ_copy_gbs": copy_gbs, "frac_of_in_situ_copy": achieved / copy_gbs},
+        "clocks": top["clocks"],
+        "e2e": top["e2e"],
+        "gpu_launches": top["gpu_launches"],
+        "roofline": dict(top["roofline"], in_situ_copy_gbs=copy_gbs,
+                         frac_of_in_situ_copy=(top["roofline"]["achieved"] / copy_gbs
+                                               if top["roofline"]["bound"] == "hbm" else None)),
     }
-    if args.block_steps > 1:
-        # several steps per pass over x and b: the pass is bound by the arithmetic of a step, not by HBM.
-        # achieved = lane instructions executed per second (ncu's count per replica-param and step, recorded
-        # above with the digest of the kernel sources, x replica-params x steps per second); peak = one warp
-        # instruction of 32 lanes per scheduler and clock.
-        steps_per_launch = args.steps / max(fused_n, 1)
-        rp_steps_per_s = w.n * cols * steps_per_launch / (fused_avg_ms * 1e-3)
-        sm_count = torch.cuda.get_device_properties(device).multi_processor_count
-        mhz = line["clocks"].get("sm_max_mhz") or 1965
-        peak_alu = sm_count * 4 * 32 * mhz * 1e6 / 1e12
-        instr = None
-        if BLOCKED_LANE_INSTRUCTIONS["kernel_digest"] == blocked_kernel_digest():
-            instr = BLOCKED_LANE_INSTRUCTIONS["per_replica_param_step"].get(w.name)
-        alu = instr * rp_steps_per_s / 1e12 if instr else None
-        line["roofline"] = {"bound": "alu", "achieved": alu, "peak": peak_alu, "unit": "T lane-instructions/s",
-                            "frac": alu / peak_alu if alu else None, "traffic": None,
-                            "peak_kind": "derived: SMs x 4 schedulers x 32 lanes x max SM clock",
-                            "kernel": "rps_fused_blocked_kernel", "lane_instructions_per_replica_param_step": instr,
-                            "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n,
-                            "steps_per_launch": steps_per_launch,
-                            "hbm_gbs_moved_per_launch": 3 * w.elem_bytes * w.n * cols / (fused_avg_ms * 1e-3) / 1e9}
-    r.close()
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = oracle_baseline(w, b)
+    if len(entries) > 1:
+        # every workload of the run, the headline included, each with its own clocks and roofline
+        line["workloads"] = {name: {k: v for k, v in e.items() if k not in ("kernel_shape", "sharded")}
+                             for name, e in entries.items()}
+    if cpu is not None:
+        line["cpu_baseline"] = cpu
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -405,7 +512,7 @@ def run_reference(args):
     import oracle
     from paper_1810_07766_b200 import workloads as wl
 
-    w = wl.WORKLOADS[args.workload]
+    w = wl.WORKLOADS[args.workload or HEADLINE]
     if args.p is not None:
         w = replace(w, p=args.p)
     cols_n = min(w.d, args.reference_columns)
@@ -442,10 +549,12 @@ def run_reference(args):
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=("cuda", "reference"), default="cuda")
-    ap.add_argument("--workload", choices=("cfg1", "cfg2", "cfg3", "cfg4", "cfg5"), default="cfg2")
+    ap.add_argument("--workload", choices=("cfg1", "cfg2", "cfg3", "cfg4", "cfg5"), default=None,
+                    help="time this workload only (default: cfg3 as the headline, then cfg2 and cfg4 with every drop "
+                         "probability of their sweeps, and cfg5, all in one JSON line)")
     ap.add_argument("--p", type=float, default=None, help="override the drop probability (p sweeps)")
     ap.add_argument("--d", type=int, default=None, help="override the model size (small profiler captures)")
     ap.add_argument("--n", type=int, default=None, help="override the number of workers (shape sweeps)")
@@ -456,8 +565,11 @@ def main(argv=None):
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true", help="tuning sweeps only: leave the host-buffer pass out")
     ap.add_argument("--kernel", type=int, default=0,
-                    help="0 library's choice, 1 direct loads, 2 staged (producer warp), 3 self-refilling ring (bf16)")
+                    help="0 library's choice, 1 direct loads, 2 staged (producer warp), 3 self-refilling ring (bf16), "
+                         "4 workers streamed through a ring per warp")
     ap.add_argument("--team-warps", type=int, default=0, help="ring kernel: warps that share a tile")
+    ap.add_argument("--row-skew-lines", type=int, default=-1,
+                    help="extra 128-byte lines of padding per device row (-1 = the library's choice)")
     ap.add_argument("--workers-per-lane", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--consumer-warps", type=int, default=0)

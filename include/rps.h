@@ -18,11 +18,15 @@
  *     scratch buffer with rps_bind() and keeps ownership.
  *   - Work is enqueued on the CUDA stream given to rps_bind(); calls that return
  *     data to the host synchronise that stream first.
- *   - A handle is not thread-safe; distinct handles are independent.
+ *   - A handle is not thread-safe; distinct handles are independent: they may be
+ *     used from different host threads at the same time and bound on different
+ *     devices of one process.  A handle belongs to the device that was current at
+ *     rps_bind(); every later call that touches the device must be made with that
+ *     device current (RPS_ESTATE otherwise).
  *   - Dense host arrays are row-major [n][d] in the replica type (float, or
  *     bfloat16 bit patterns in uint16_t).  On the device a row occupies
- *     rps_pitch() elements (d rounded up so that every row starts on a 128-byte
- *     boundary, plus row_skew_lines lines); columns d..pitch-1 are padding that
+ *     rps_pitch() elements (d rounded up so that every row starts on a 1 KB
+ *     boundary, or as row_skew_lines says); columns d..pitch-1 are padding that
  *     belongs to the library: it reads it, may zero the few padding columns that
  *     share a 16-byte unit with column d-1, and leaves the rest as it found it.
  */
@@ -83,9 +87,10 @@ typedef struct rps_options {
     double sigma;          /* std-dev of the Gaussian gradient noise, default 0           */
     /* Shape of the fused kernel; 0 = the library's choice.  None of these changes what is
      * computed beyond the order of the fp32 additions inside the masked average.           */
-    int32_t row_skew_lines;   /* extra 128-byte lines of padding per device row, -1 = automatic
-                                 (keeps the n rows from all mapping to one DRAM channel when
-                                 the row size is a multiple of a large power of two)         */
+    int32_t row_skew_lines;   /* extra 128-byte lines of padding per device row after d has been
+                                 rounded up to a whole line; -1 = automatic: as many as make the
+                                 row a whole number of kilobytes (the kernels' row pieces are then
+                                 whole DRAM pages in every row)                               */
     int32_t kernel;           /* 1: lanes load their slices directly from global memory;
                                  2: slices are staged through shared memory by bulk
                                  asynchronous copies issued by a producer warp;
@@ -93,14 +98,22 @@ typedef struct rps_options {
                                  CTA compute, each taking the next slice of the next tile from a
                                  counter, and the last warp to have read a stage refills it (built for bf16 replicas
                                  with more than 4 workers, plain untracked model averaging;
-                                 any other step runs as kernel 2).
+                                 any other step runs as kernel 2);
+                                 4: workers streamed: a lane owns one 16-byte slice of columns and
+                                 walks all n workers in order, two at a time, adding each v to the
+                                 running sum and storing it at once where the return message is
+                                 lost; the average is rounded once and stored to every receiver.
+                                 Every warp has a shared-memory ring of its own that it refills
+                                 itself; a warp reads and writes whole 512-byte pieces of rows
+                                 (plain untracked model averaging, n >= 2; any other step runs as
+                                 kernel 2).
                                  0: kernel 1 for models too short to give every SM a tile, kernel 3
                                  for bf16 replicas of more than 4 workers (unless an option that
                                  shapes kernel 2 alone is set), else kernel 2                 */
     int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */
-    int32_t stages;           /* depth of the shared-memory ring of kernels 2 and 3 (2..8)   */
+    int32_t stages;           /* depth of the shared-memory ring(s) of kernels 2, 3 and 4 (2..8) */
     int32_t consumer_warps;   /* compute warps per CTA of kernel 2 (1..24; shapes that need
-                                 many registers are clamped lower)                           */
+                                 many registers are clamped lower) and of kernel 4 (1..32)   */
     int32_t copy_mode;        /* kernel 2 fills a stage with 1: one bulk copy per row,
                                  2: two-dimensional TMA boxes covering all n rows            */
     int32_t slice_bytes;      /* kernel 2, bf16 replicas: bytes of a row handled by one lane,

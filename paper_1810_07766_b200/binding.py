@@ -7,6 +7,7 @@ There is no CPU fallback: a missing library or a failing call raises.
 from __future__ import annotations
 
 import ctypes
+import functools
 import os
 from typing import Optional, Tuple
 
@@ -57,6 +58,18 @@ def shard_columns(d: int, world: int, rank: int, align: int = 64) -> Tuple[int, 
     last = (units * (rank + 1)) // world
     begin, end = min(first * align, d), min(last * align, d)
     return begin, end - begin
+
+
+def _device_current(method):
+    """Runs a method of RPS with the handle's device current: the library launches on the current device and
+    refuses a call made with another one current (RPS_ESTATE)."""
+    @functools.wraps(method)
+    def wrapper(self, *args, **kwargs):
+        if torch.cuda.current_device() == self.device.index:
+            return method(self, *args, **kwargs)
+        with torch.cuda.device(self.device):
+            return method(self, *args, **kwargs)
+    return wrapper
 
 
 class RPSError(RuntimeError):
@@ -206,10 +219,12 @@ class RPS:
             raise ValueError(f"{name} has the wrong element size for {self.dtype} replicas")
 
     # ------------------------------------------------------------------ C ABI, one method per call
+    @_device_current
     def set_targets(self, b_host) -> None:
         self._expect(b_host, "b_host")
         self._check(self._lib.rps_set_targets(self._h, _host_ptr(b_host)), "rps_set_targets")
 
+    @_device_current
     def write(self, x_host) -> None:
         self._expect(x_host, "x_host")
         self._check(self._lib.rps_write(self._h, _host_ptr(x_host)), "rps_write")
@@ -222,12 +237,15 @@ class RPS:
         self._check(self._lib.rps_get_step(self._h, ctypes.byref(t)), "rps_get_step")
         return t.value
 
+    @_device_current
     def step(self) -> None:
         self._check(self._lib.rps_step(self._h), "rps_step")
 
+    @_device_current
     def step_n(self, steps: int) -> None:
         self._check(self._lib.rps_step_n(self._h, steps), "rps_step_n")
 
+    @_device_current
     def step_forced(self, up, down) -> None:
         up = np.ascontiguousarray(up, dtype=np.uint64)
         down = np.ascontiguousarray(down, dtype=np.uint64)
@@ -237,6 +255,7 @@ class RPS:
         self._check(self._lib.rps_step_forced(self._h, up.ctypes.data_as(u64p), down.ctypes.data_as(u64p)),
                     "rps_step_forced")
 
+    @_device_current
     def step_host(self, x_host, b_host=None) -> None:
         self._expect(x_host, "x_host")
         if b_host is not None:
@@ -244,12 +263,14 @@ class RPS:
         self._check(self._lib.rps_step_host(self._h, _host_ptr(x_host), None if b_host is None else _host_ptr(b_host)),
                     "rps_step_host")
 
+    @_device_current
     def read(self, out=None):
         out = self._host_array() if out is None else out
         self._expect(out, "out")
         self._check(self._lib.rps_read(self._h, _host_ptr(out)), "rps_read")
         return out
 
+    @_device_current
     def read_masks(self, t: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
         up = np.zeros(self.n, dtype=np.uint64)
         down = np.zeros(self.n, dtype=np.uint64)
@@ -260,11 +281,13 @@ class RPS:
                                              cnt.ctypes.data_as(i32p), server.ctypes.data_as(i32p)), "rps_read_masks")
         return up, down, cnt, server
 
+    @_device_current
     def diag(self) -> Tuple[float, float]:
         a, c = ctypes.c_double(), ctypes.c_double()
         self._check(self._lib.rps_diag(self._h, ctypes.byref(a), ctypes.byref(c)), "rps_diag")
         return a.value, c.value
 
+    @_device_current
     def estimate_alpha(self, t0: int, steps: int) -> Tuple[float, float]:
         """Monte-Carlo (alpha_1, alpha_2) of Eqs. (4), (5) from the drop masks of ``steps`` steps from ``t0``."""
         a1, a2 = ctypes.c_double(), ctypes.c_double()
@@ -272,6 +295,7 @@ class RPS:
                     "rps_estimate_alpha")
         return a1.value, a2.value
 
+    @_device_current
     def track(self, capacity: int) -> None:
         """Records {dist2_to_opt, consensus} of the state each of the next `capacity` steps leaves behind, as a
         by-product of the fused pass (rps_track); 0 switches tracking off."""
@@ -280,6 +304,7 @@ class RPS:
         with torch.cuda.device(self.device):
             self._check(self._lib.rps_track(self._h, ptr, capacity), "rps_track")
 
+    @_device_current
     def read_trace(self) -> np.ndarray:
         """The recorded pairs so far as a float64 array [steps][2] (synchronises)."""
         held = getattr(self, "trace_dev", None)
@@ -290,9 +315,11 @@ class RPS:
                         "rps_read_trace")
         return out[:count.value]
 
+    @_device_current
     def profile(self, enable: bool) -> None:
         self._check(self._lib.rps_profile(self._h, int(enable)), "rps_profile")
 
+    @_device_current
     def profile_read(self):
         """(fused_ms, fused_launches, mask_ms, mask_launches) since profiling was enabled; resets them."""
         fm, mm = ctypes.c_double(), ctypes.c_double()

@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(CSRC, "librps.so")
 SOURCES = ["rps_api.cu", "rps_kernels.cu", "rps_direct_track.cu", "rps_blocked.cu", "rps_staged.cu",
-           "rps_staged_grad.cu", "rps_staged_track.cu", "rps_ring.cu", "rps_static.cu"]
+           "rps_staged_grad.cu", "rps_staged_track.cu", "rps_ring.cu", "rps_stream.cu", "rps_static.cu"]
 HEADERS = ["rps_device.cuh", "rps_kernels.h", "rps_direct.cuh", "rps_staged.cuh", "rps_tma.cuh"]
 
 

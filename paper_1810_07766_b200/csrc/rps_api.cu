@@ -15,13 +15,15 @@
 
 static_assert(sizeof(rps::StepMasks) == rps::kStepMasksBytes, "mask record layout");
 
-// Extra 128-byte lines appended to every row so that the rows of x and b do not all start at
-// the same offset modulo a large power of two (which would send the n row streams of a tile
-// to the same DRAM channel and bank).  `asked` < 0 = automatic.
+// Extra 128-byte lines appended to every row.  `asked` < 0 = automatic: as many as make the row a whole
+// number of kilobytes, so that every row starts on a 1 KB boundary and the row pieces the kernels move (1 to
+// 4 KB wide, cut at multiples of their width from the start of the row) are whole DRAM pages in every row
+// instead of straddling page boundaries in most of them (measured: up to 3 % of the step).  Rows that all
+// start at the same offset modulo a large power of two are no problem on this memory system.
 static int64_t rps_row_skew_lines(int64_t lines, int32_t asked)
 {
     if (asked >= 0) return asked;
-    return (lines % 2 == 0) ? 1 : 0;
+    return (8 - lines % 8) % 8;
 }
 
 namespace {
@@ -53,6 +55,7 @@ struct rps_handle {
     void* b = nullptr;
     unsigned char* scratch = nullptr;
     cudaStream_t stream = nullptr;
+    int device = -1;  // the device that was current at rps_bind: x, b, scratch and the stream belong to it
     int sm_count = 0;
     // run state
     uint64_t t = 0;
@@ -133,6 +136,10 @@ int need_bound(rps_handle* h)
 {
     if (!h) return RPS_EINVAL;
     if (!h->bound) return fail(h, RPS_ESTATE, "rps_bind has not been called");
+    // kernels are launched on, and attributes set for, the CURRENT device: it has to be the handle's
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != h->device)
+        return fail(h, RPS_ESTATE, "the device the handle was bound on is not the current device");
     return RPS_OK;
 }
 
@@ -405,13 +412,13 @@ int rps_configure(rps_handle* h, const rps_options* opt)
     if (!std::isfinite(opt->sigma) || opt->sigma < 0.0) return fail(h, RPS_EINVAL, "sigma must be finite and >= 0");
     if (opt->row_skew_lines < -1 || opt->row_skew_lines > 4096)
         return fail(h, RPS_EINVAL, "row_skew_lines must be -1 (auto) or 0..4096");
-    if (opt->kernel < 0 || opt->kernel > 3) return fail(h, RPS_EINVAL, "kernel must be 0 (auto), 1, 2 or 3");
+    if (opt->kernel < 0 || opt->kernel > 4) return fail(h, RPS_EINVAL, "kernel must be 0 (auto) or 1..4");
     if (opt->workers_per_lane != 0 && opt->workers_per_lane != 2 && opt->workers_per_lane != 4 &&
         opt->workers_per_lane != 8)
         return fail(h, RPS_EINVAL, "workers_per_lane must be 0 (auto), 2, 4 or 8");
     if (opt->stages != 0 && (opt->stages < 2 || opt->stages > 8)) return fail(h, RPS_EINVAL, "stages must be 0 or 2..8");
-    if (opt->consumer_warps < 0 || opt->consumer_warps > 24)
-        return fail(h, RPS_EINVAL, "consumer_warps must be 0 (auto) or 1..24");
+    if (opt->consumer_warps < 0 || opt->consumer_warps > 32)
+        return fail(h, RPS_EINVAL, "consumer_warps must be 0 (auto) or 1..32");
     if (opt->slice_bytes != 0 && opt->slice_bytes != 8 && opt->slice_bytes != 16)
         return fail(h, RPS_EINVAL, "slice_bytes must be 0 (auto), 8 or 16");
     if (opt->average != RPS_AVERAGE_MODELS && opt->average != RPS_AVERAGE_GRADIENTS)
@@ -456,6 +463,7 @@ int rps_bind(rps_handle* h, void* x_dev, void* b_dev, int64_t pitch, void* scrat
     int dev = 0;
     RPS_CUDA(h, cudaGetDevice(&dev));
     RPS_CUDA(h, cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, dev));
+    h->device = dev;
     h->x = x_dev;
     h->b = b_dev;
     h->scratch = static_cast<unsigned char*>(scratch_dev);

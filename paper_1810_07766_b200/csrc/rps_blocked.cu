@@ -87,14 +87,10 @@ cudaError_t launch_blocked_as(const FusedParams& prm, int steps, int sm_count, c
     constexpr int warp_cols = (32 / G) * VEC;
     const int64_t tiles = (prm.d + warp_cols - 1) / warp_cols;
     const int64_t ctas_needed = (tiles + kBlockedThreads / 32 - 1) / (kBlockedThreads / 32);
-    static int per_sm = 0;  // resident CTAs per SM of this instantiation, asked once
-    if (per_sm == 0) {
-        int occ = 0;
-        cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, rps_fused_blocked_kernel<T, VEC, WPT, G>,
-                                                                        kBlockedThreads, 0);
-        if (err != cudaSuccess) return err;
-        per_sm = occ < 1 ? 1 : occ;
-    }
+    static LaunchState state;  // of this instantiation, per device
+    int per_sm = 1;                // resident CTAs per SM, asked once per device
+    cudaError_t err = resident_ctas_per_sm(state, rps_fused_blocked_kernel<T, VEC, WPT, G>, kBlockedThreads, 0, &per_sm);
+    if (err != cudaSuccess) return err;
     int64_t grid = (int64_t)sm_count * per_sm;
     if (grid > ctas_needed) grid = ctas_needed;
     if (grid < 1) grid = 1;

@@ -79,33 +79,50 @@ __device__ __forceinline__ Philox4 philox4x32_keyed(uint32_t c0, uint32_t c1, ui
     return Philox4{c0, c1, c2, c3};
 }
 
-// One Box-Muller pair from one 32-bit word, already scaled by gamma*sigma.  The low
-// 16 bits pick the radius uniform and the high 16 bits the angle uniform, both at
-// bin centres (k + 1/2) / 2^16.  2^23 + k is built in the mantissa, so one fma
-// gives the uniform exactly.  Returns radius, and (cos, sin) of the angle.
+// One Box-Muller pair from one 32-bit word, already scaled by -(gamma*sigma): the sign of the update
+// v = ... - (gamma sigma) xi is carried by the angle, which is taken half a turn on
+// (cos(a + pi) = -cos a, sin(a + pi) = -sin a), so callers ADD radius * (c, s).  The low 16 bits pick the
+// radius uniform and the high 16 bits the angle uniform, both at bin centres (k + 1/2) / 2^16.  2^23 + k is
+// built in the mantissa, so one fma gives the uniform exactly.  Returns radius, and (c, s) = -(cos, sin) of
+// the angle.
 struct ScaledPair {
     float radius, c, s;
 };
+
+// u = (k + 1/2) / 2^16 = (2^23 + k) * 2^-16 - (128 - 2^-17), exact in fp32
+constexpr float kUniformScale = 1.52587890625e-05f, kUniformShift = -127.99999237060546875f;
+// the angle in turns plus half a turn, in (1/2, 3/2): (2^23 + k) * 2^-16 - (127.5 - 2^-17), exact for the same
+// reason (127.5 - 2^-17 has 24 significant bits; 128.5 - 2^-17, for half a turn less, would have 25); it is
+// scaled by 2 pi only after that, so that the rounding of the constant is not multiplied by 2^23
+constexpr float kAngleShift = -127.49999237060546875f;
+constexpr float kTwoPi = 6.283185307179586f;
+
+__device__ __forceinline__ float approx_log2(float u)
+{
+    float r;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(u));
+    return r;
+}
+
+// radius = gamma*sigma * sqrt(-2 ln u), with ln u = ln 2 * log2 u folded into noise_scale (scaled_log2 =
+// noise_scale * log2 u).  The special-function unit's approximations are used in their flush-to-zero forms:
+// no operand here is subnormal (u >= 2^-17), so the slower subnormal handling buys nothing.
+__device__ __forceinline__ ScaledPair radius_and_direction(float scaled_log2, float angle_rad)
+{
+    ScaledPair out;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(out.radius) : "f"(scaled_log2));
+    asm("sin.approx.ftz.f32 %0, %1;" : "=f"(out.s) : "f"(angle_rad));
+    asm("cos.approx.ftz.f32 %0, %1;" : "=f"(out.c) : "f"(angle_rad));
+    return out;
+}
 
 __device__ __forceinline__ ScaledPair gaussian_pair(uint32_t word, float noise_scale)
 {
     const float k_radius = __uint_as_float(__byte_perm(word, 0x4B000000u, 0x7410));  // 2^23 + low half
     const float k_angle = __uint_as_float(__byte_perm(word, 0x4B000000u, 0x7432));   // 2^23 + high half
-    // u = (k + 1/2) / 2^16 = (2^23 + k) * 2^-16 - (128 - 2^-17), exact in fp32
-    const float u = fmaf(k_radius, 1.52587890625e-05f, -127.99999237060546875f);
-    // the angle in turns, exact for the same reason; it is scaled by 2 pi only after that, so that
-    // the rounding of the constant is not multiplied by 2^23
-    const float angle_turns = fmaf(k_angle, 1.52587890625e-05f, -127.99999237060546875f);
-    ScaledPair out;
-    // radius = gamma*sigma * sqrt(-2 ln u), with ln u = ln 2 * log2 u folded into noise_scale.
-    // The special-function unit's approximations are used in their flush-to-zero forms: no
-    // operand here is subnormal (u >= 2^-17), so the slower subnormal handling buys nothing.
-    float log2_u, turns_to_rad = 6.283185307179586f * angle_turns;
-    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(log2_u) : "f"(u));
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(out.radius) : "f"(noise_scale * log2_u));
-    asm("sin.approx.ftz.f32 %0, %1;" : "=f"(out.s) : "f"(turns_to_rad));
-    asm("cos.approx.ftz.f32 %0, %1;" : "=f"(out.c) : "f"(turns_to_rad));
-    return out;
+    const float u = fmaf(k_radius, kUniformScale, kUniformShift);
+    const float angle_turns = fmaf(k_angle, kUniformScale, kAngleShift);
+    return radius_and_direction(noise_scale * approx_log2(u), kTwoPi * angle_turns);
 }
 
 // Row slices of one lane: VEC replica-typed elements (16 bytes, or 8 for the narrow bf16 form) <-> fp32 registers.
@@ -222,10 +239,126 @@ __device__ __forceinline__ void add_gradient_noise(float (&v)[WPT][VEC], int64_t
                 const ScaledPair z = gaussian_pair(words[m], prm.noise_scale);
                 float(&row)[VEC] = v[w + (m >> 1)];  // words 0,1 -> worker w, words 2,3 -> worker w+1
                 const int k = 4 * q + 2 * (m & 1);
-                row[k] = fmaf(-z.radius, z.c, row[k]);
-                row[k + 1] = fmaf(-z.radius, z.s, row[k + 1]);
+                row[k] = fmaf(z.radius, z.c, row[k]);
+                row[k + 1] = fmaf(z.radius, z.s, row[k + 1]);
             }
         }
+    }
+}
+
+// ---- The same arithmetic two columns at a time, in the packed fp32 forms of sm_100 (fma / mul / add / sub
+// .f32x2: one instruction, two IEEE operations, the same bits as the scalar forms).  A Float2 is two floats
+// in one 64-bit register (an aligned register pair: packing and unpacking cost nothing where the halves
+// already lie side by side, as the halves of a 16-byte load do).
+using Float2 = unsigned long long;
+
+__device__ __forceinline__ Float2 pack2(float lo, float hi)
+{
+    Float2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ Float2 pack2(uint32_t lo, uint32_t hi)
+{
+    Float2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(Float2 v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ Float2 fma2(Float2 a, Float2 b, Float2 c)
+{
+    Float2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ Float2 mul2(Float2 a, Float2 b)
+{
+    Float2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ Float2 sub2(Float2 a, Float2 b)
+{
+    Float2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// s += v (both halves) where `take` is set, as one predicated instruction
+__device__ __forceinline__ void add2_if(Float2& s, Float2 v, uint32_t take)
+{
+    asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p add.rn.f32x2 %0, %0, %1;\n\t}" : "+l"(s) : "l"(v), "r"(take));
+}
+
+// Loop-invariant operands of the packed step.
+struct PackedScalars {
+    Float2 gamma;          // (gamma, gamma)
+    Float2 uniform_scale;  // (2^-16, 2^-16)
+    Float2 uniform_shift;  // (shift of the radius uniform, shift of the angle)
+    Float2 noise_and_turn; // (noise_scale, 2 pi)
+    __device__ __forceinline__ explicit PackedScalars(const FusedParams& prm)
+        : gamma(pack2(prm.gamma, prm.gamma)),
+          uniform_scale(pack2(kUniformScale, kUniformScale)),
+          uniform_shift(pack2(kUniformShift, kAngleShift)),
+          noise_and_turn(pack2(prm.noise_scale, kTwoPi))
+    {
+    }
+};
+
+// v (two adjacent columns of one worker) += the Box-Muller pair of `word`; bit for bit what gaussian_pair and two
+// scalar multiply-adds give.
+__device__ __forceinline__ Float2 add_noise_pair(Float2 v, uint32_t word, const PackedScalars& k)
+{
+    const uint32_t k_radius = __byte_perm(word, 0x4B000000u, 0x7410);  // 2^23 + low half
+    const uint32_t k_angle = __byte_perm(word, 0x4B000000u, 0x7432);   // 2^23 + high half
+    float u, angle_turns;
+    unpack2(fma2(pack2(k_radius, k_angle), k.uniform_scale, k.uniform_shift), u, angle_turns);
+    float scaled_log2, angle_rad;
+    unpack2(mul2(pack2(approx_log2(u), angle_turns), k.noise_and_turn), scaled_log2, angle_rad);
+    const ScaledPair z = radius_and_direction(scaled_log2, angle_rad);
+    return fma2(pack2(z.radius, z.radius), pack2(z.c, z.s), v);
+}
+
+// Local SGD step of one lane on a worker pair (k even) x VEC columns from column c, from the raw slices, two
+// columns at a time: v = x + gamma (b - x) - (gamma sigma) xi.  Same bits as local_sgd_raw<T, VEC, 2, false>.
+template <typename T, int VEC>
+__device__ __forceinline__ void local_sgd_pair_packed(const uint4 (&raw_x)[2], const uint4 (&raw_b)[2],
+                                                      Float2 (&v)[2][VEC / 2], int64_t c, int k,
+                                                      const FusedParams& prm, const PackedScalars& scalars)
+{
+    static_assert(VEC * sizeof(T) == 16, "a slice is 16 bytes");
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t wx[4] = {raw_x[h].x, raw_x[h].y, raw_x[h].z, raw_x[h].w};
+        const uint32_t wb[4] = {raw_b[h].x, raw_b[h].y, raw_b[h].z, raw_b[h].w};
+        if (sizeof(T) == 4) {
+#pragma unroll
+            for (int m = 0; m < 2; ++m) {
+                const Float2 x2 = pack2(wx[2 * m], wx[2 * m + 1]);
+                v[h][m % (VEC / 2)] = fma2(scalars.gamma, sub2(pack2(wb[2 * m], wb[2 * m + 1]), x2), x2);
+            }
+        } else {
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+                const float x_lo = __uint_as_float(wx[m] << 16), x_hi = __uint_as_float(wx[m] & 0xFFFF0000u);
+                float d_lo, d_hi;
+                bf16_pair_minus(wb[m], x_lo, x_hi, d_lo, d_hi);
+                v[h][m % (VEC / 2)] = fma2(scalars.gamma, pack2(d_lo, d_hi), pack2(x_lo, x_hi));
+            }
+        }
+    }
+    if (!prm.noisy) return;
+#pragma unroll
+    for (int q = 0; q < VEC / 4; ++q) {
+        const Philox4 r = philox4x32_keyed<kNoiseRounds>(prm.t_lo, prm.t_hi, (uint32_t)((c + prm.col_offset) >> 2) + q,
+                                                         kStreamNoise | ((uint32_t)(k >> 1) << 8), prm.round_key);
+        // words 0,1 -> the pair's first worker (columns 0,1 and 2,3 of the four), words 2,3 -> its second
+        v[0][2 * q] = add_noise_pair(v[0][2 * q], r.x, scalars);
+        v[0][2 * q + 1] = add_noise_pair(v[0][2 * q + 1], r.y, scalars);
+        v[1][2 * q] = add_noise_pair(v[1][2 * q], r.z, scalars);
+        v[1][2 * q + 1] = add_noise_pair(v[1][2 * q + 1], r.w, scalars);
     }
 }
 

@@ -223,6 +223,7 @@ cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool b
 {
     if (tune.kernel == 1) return launch_fused_direct(prm, tune, bf16, sm_count, stream);
     if (tune.kernel == 3 && ring_kernel_covers(prm, bf16)) return launch_fused_ring(prm, tune, bf16, sm_count, stream);
+    if (tune.kernel == 4 && stream_kernel_covers(prm, bf16)) return launch_fused_stream(prm, tune, bf16, sm_count, stream);
     if (tune.kernel == 0) {
         // A model this short gives the staged kernel's ring less than a tile per SM: there
         // is nothing to pipeline and its set-up dominates; the step is launch bound and L2 resident.
@@ -230,6 +231,12 @@ cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool b
         if (prm.d * bytes_per_column < (int64_t)sm_count * 8192)
             return launch_fused_direct(prm, tune, bf16, sm_count, stream);
     }
+    // bf16 replicas of more than 32 workers: workers streamed through the teams' rings (what is staged does not
+    // grow with n, every row piece is 2 KB); measured side by side 5 % ahead of the ring kernel at n = 64 and
+    // a third at n = 48, level with it or behind at n <= 32.
+    if (tune.kernel == 0 && bf16 && prm.n > 32 && stream_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 &&
+        tune.copy_mode == 0 && tune.slice_bytes == 0)
+        return launch_fused_stream(prm, tune, bf16, sm_count, stream);
     // bf16 replicas of more than 4 workers: the self-refilling ring (16 compute warps, no producer warp), unless an
     // option that shapes the staged kernel only was set.  Measured side by side it is 3-8 % ahead at every n.
     if (tune.kernel == 0 && bf16 && ring_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 &&

@@ -4,7 +4,84 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 namespace rps {
+
+// What a launch wrapper remembers about one kernel instantiation, PER DEVICE and under a lock: the dynamic
+// shared memory the kernel has been granted (cudaFuncSetAttribute acts on the current device's copy of the
+// function) and its resident CTAs per SM.  Handles bound on several devices, and host threads stepping
+// distinct handles, may launch the same instantiation at the same time.
+constexpr int kMaxDevices = 64;
+
+struct LaunchState {
+    std::mutex lock;
+    size_t smem_limit[kMaxDevices] = {};     // opt-in shared memory per CTA of the device (0 = not asked yet)
+    uint32_t smem_granted[kMaxDevices] = {};
+    int occ_threads[kMaxDevices] = {};       // the launch shape the occupancy below was asked for
+    uint32_t occ_smem[kMaxDevices] = {};
+    int occ_per_sm[kMaxDevices] = {};        // 0 = not asked yet
+};
+
+inline cudaError_t current_device(int* dev)
+{
+    cudaError_t err = cudaGetDevice(dev);
+    if (err != cudaSuccess) return err;
+    return *dev >= 0 && *dev < kMaxDevices ? cudaSuccess : cudaErrorInvalidDevice;
+}
+
+// Opt-in shared memory per CTA of the current device.
+inline cudaError_t smem_limit_of_device(LaunchState& st, size_t* out)
+{
+    int dev = 0;
+    cudaError_t err = current_device(&dev);
+    if (err != cudaSuccess) return err;
+    std::lock_guard<std::mutex> hold(st.lock);
+    if (st.smem_limit[dev] == 0) {
+        int optin = 0;
+        if ((err = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
+            return err;
+        st.smem_limit[dev] = (size_t)optin;
+    }
+    *out = st.smem_limit[dev];
+    return cudaSuccess;
+}
+
+// Makes sure `kernel` may be launched with `bytes` of dynamic shared memory on the current device.
+template <typename Kernel>
+cudaError_t grant_smem(LaunchState& st, Kernel kernel, uint32_t bytes)
+{
+    int dev = 0;
+    cudaError_t err = current_device(&dev);
+    if (err != cudaSuccess) return err;
+    std::lock_guard<std::mutex> hold(st.lock);
+    if (bytes > st.smem_granted[dev]) {
+        if ((err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes)) != cudaSuccess)
+            return err;
+        st.smem_granted[dev] = bytes;
+    }
+    return cudaSuccess;
+}
+
+// Resident CTAs per SM of `kernel` in this launch shape on the current device (at least 1).
+template <typename Kernel>
+cudaError_t resident_ctas_per_sm(LaunchState& st, Kernel kernel, int threads, uint32_t smem_bytes, int* out)
+{
+    int dev = 0;
+    cudaError_t err = current_device(&dev);
+    if (err != cudaSuccess) return err;
+    std::lock_guard<std::mutex> hold(st.lock);
+    if (st.occ_per_sm[dev] == 0 || st.occ_threads[dev] != threads || st.occ_smem[dev] != smem_bytes) {
+        int occ = 0;
+        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, threads, smem_bytes)) != cudaSuccess)
+            return err;
+        st.occ_per_sm[dev] = occ < 1 ? 1 : occ;
+        st.occ_threads[dev] = threads;
+        st.occ_smem[dev] = smem_bytes;
+    }
+    *out = st.occ_per_sm[dev];
+    return cudaSuccess;
+}
 
 struct StepMasks;  // defined in rps_device.cuh
 
@@ -23,7 +100,8 @@ struct MaskParams {
 // Which fused kernel runs and how it is shaped; 0 everywhere = the library's choice.
 struct FusedTuning {
     int32_t kernel;            // 1 direct (register loads), 2 staged (a producer warp fills a shared-memory ring),
-                               // 3 self-refilling ring (every warp computes; bf16 replicas)
+                               // 3 self-refilling ring (every warp computes; bf16 replicas), 4 workers streamed
+                               // through a ring per warp
     int32_t workers_per_lane;  // 2, 4 or 8
     int32_t stages;            // shared-memory ring depth of the staged kernel
     int32_t consumer_warps;    // compute warps per CTA of the staged kernel
@@ -96,6 +174,10 @@ cudaError_t launch_fused_staged(const FusedParams& prm, const FusedTuning& tune,
 bool ring_kernel_covers(const FusedParams& prm, bool bf16);
 cudaError_t launch_fused_ring(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
                               cudaStream_t stream);
+// Workers streamed through per-warp rings (rps_stream.cu): whether it is built for this step, and its launch.
+bool stream_kernel_covers(const FusedParams& prm, bool bf16);
+cudaError_t launch_fused_stream(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
+                                cudaStream_t stream);
 // The optional forms of the fused step, built in one family of lane shapes, each group in a
 // translation unit of its own: gradient averaging (prm.average_gradients) and tracked steps
 // (prm.trace != NULL, with either kind of averaging).

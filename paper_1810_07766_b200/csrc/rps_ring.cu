@@ -398,16 +398,10 @@ template <typename T, int VEC, int WPT, int G>
 cudaError_t launch_ring_as(const FusedParams& prm, const FusedTuning& tune, int sm_count, cudaStream_t stream)
 {
     auto kernel = rps_fused_ring_kernel<T, VEC, WPT, G>;
-    static size_t smem_limit = 0;  // opt-in shared memory per CTA of this device
-    static uint32_t smem_granted = 0;
-    cudaError_t err;
-    if (smem_limit == 0) {
-        int dev = 0, optin = 0;
-        if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
-        if ((err = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
-            return err;
-        smem_limit = (size_t)optin;
-    }
+    static LaunchState state;  // of this instantiation, per device
+    size_t smem_limit = 0;
+    cudaError_t err = smem_limit_of_device(state, &smem_limit);
+    if (err != cudaSuccess) return err;
     RingShape shape;
     uint32_t smem_bytes = 0;
     if (!plan_ring(prm, tune, VEC, G, sizeof(T), smem_limit, &shape, &smem_bytes)) return cudaErrorInvalidConfiguration;
@@ -418,12 +412,7 @@ cudaError_t launch_ring_as(const FusedParams& prm, const FusedTuning& tune, int 
         !encode_rows(&map_b, prm.b, bf16, prm, shape.box_cols, prm.cols_in_row) ||
         !encode_rows(&map_out, prm.x, bf16, prm, shape.box_cols, prm.d))
         return cudaErrorInvalidValue;
-    if (smem_bytes > smem_granted) {
-        if ((err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes)) !=
-            cudaSuccess)
-            return err;
-        smem_granted = smem_bytes;
-    }
+    if ((err = grant_smem(state, kernel, smem_bytes)) != cudaSuccess) return err;
     // persistent CTAs, one per SM (a CTA is the whole register file), each striding over the tiles
     int64_t grid = sm_count;
     if (grid > shape.tiles) grid = shape.tiles;

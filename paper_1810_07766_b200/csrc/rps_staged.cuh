@@ -486,18 +486,10 @@ template <typename T, int VEC, int WPT, int G, bool GRAD = false, bool DIAG = fa
 cudaError_t launch_staged_as(const FusedParams& prm, const FusedTuning& tune, int sm_count, cudaStream_t stream)
 {
     auto kernel = rps_fused_staged_kernel<T, VEC, WPT, G, GRAD, DIAG>;
-    static size_t smem_limit = 0;   // opt-in shared memory per CTA of this device
-    static uint32_t smem_granted = 0;
-    static int occ_threads = 0, occ_per_sm = 0;
-    static uint32_t occ_smem = 0;
-    cudaError_t err;
-    if (smem_limit == 0) {
-        int dev = 0, optin = 0;
-        if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
-        if ((err = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
-            return err;
-        smem_limit = (size_t)optin;
-    }
+    static LaunchState state;  // of this instantiation, per device
+    size_t smem_limit = 0;
+    cudaError_t err = smem_limit_of_device(state, &smem_limit);
+    if (err != cudaSuccess) return err;
     Plan plan;
     if (!make_plan(prm, tune, VEC, WPT, G, sizeof(T), smem_limit, &plan)) return cudaErrorInvalidConfiguration;
     constexpr bool bf16 = sizeof(T) == 2;
@@ -507,21 +499,9 @@ cudaError_t launch_staged_as(const FusedParams& prm, const FusedTuning& tune, in
         !encode_rows(&map_b, prm.b, bf16, prm, map_box_cols, prm.cols_in_row) ||
         !encode_rows(&map_out, prm.x, bf16, prm, plan.shape.out_box_cols, prm.d))
         return cudaErrorInvalidValue;
-    if (plan.smem_bytes > smem_granted) {
-        if ((err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes)) !=
-            cudaSuccess)
-            return err;
-        smem_granted = plan.smem_bytes;
-    }
-    if (occ_threads != plan.threads || occ_smem != plan.smem_bytes) {
-        int occ = 0;
-        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, plan.threads, plan.smem_bytes)) !=
-            cudaSuccess)
-            return err;
-        occ_per_sm = occ < 1 ? 1 : occ;
-        occ_threads = plan.threads;
-        occ_smem = plan.smem_bytes;
-    }
+    if ((err = grant_smem(state, kernel, plan.smem_bytes)) != cudaSuccess) return err;
+    int occ_per_sm = 1;
+    if ((err = resident_ctas_per_sm(state, kernel, plan.threads, plan.smem_bytes, &occ_per_sm)) != cudaSuccess) return err;
     // persistent CTAs: a whole number of resident CTAs per SM, each striding over the tiles
     int64_t grid = (int64_t)sm_count * occ_per_sm;
     if (grid > plan.shape.tiles) grid = plan.shape.tiles;

@@ -1,0 +1,500 @@
+// Fused RPS step, streamed workers (sm_100a).
+//
+// The AG step gives every worker that receives block j the SAME value (Section 4.1: x <- the average if
+// the return message arrived, else the worker's own v), so a worker's v has to outlive the running sum only
+// if its return message is lost (a fraction p of the workers).  This form is built on that:
+//
+//   * A lane owns one 16-byte slice of columns (4 floats / 8 bf16) and walks ALL n workers in index order,
+//     two at a time (one noise draw serves a worker pair).  For each worker it forms v, adds it to the
+//     running sum of its columns where the up bit is set, and stores v AT ONCE where the down bit is clear.
+//     After the last worker the average is formed, rounded and packed ONCE, and stored to every receiver's
+//     row.  Nothing like v[workers][columns] stays live: no select, no shuffle, summation in worker order
+//     (the order of the plain definition), about half the registers of the lane-group forms.
+//   * A warp therefore covers 32 slices = 512 contiguous bytes of every row it touches, in loads and in
+//     stores alike (the lane-group forms store 64-byte pieces at n = 64), and the shared memory a warp needs
+//     does not grow with n: what is staged is a worker pair, not a tile of all workers.
+//   * Warps work in teams of team_warps neighbours.  A team owns a ring in shared memory whose stage holds
+//     one worker pair of the team's tile: 2 rows x (team_warps x 512 bytes) of x and of b, fetched by two TMA box
+//     copies (the arrays are described to the unit in 8-byte units, so one box spans up to 2 KB of a row).  A
+//     warp copies its part of a stage to registers and counts itself off; the warp that counts last refills
+//     the stage with the pair that comes `stages` pairs later (of the same tile or of the team's next one).
+//     Nobody waits for a free stage; the only wait is the bounded one for a stage's copies to land.  Teams
+//     take the tiles in fixed turns, so every warp knows the whole sequence of pairs in advance.
+//
+// A lane whose slice straddles two blocks or the end of the row (at most n such lanes per step) takes a
+// per-column branch with the same arithmetic, so a column's result does not depend on where it lies.
+//
+// Every mbarrier wait is bounded; a warp that gives up records a code in *prm.error, sees the copies that may
+// still be in flight land (bounded again) and leaves; its team mates run into their own limits.
+#include "rps_device.cuh"
+#include "rps_tma.cuh"
+
+namespace rps {
+
+namespace {
+
+constexpr int kStreamMaxWarps = 32;
+constexpr int kStreamMaxStages = 8;
+constexpr int kStreamDefaultStages = 3;
+constexpr int kStreamDefaultStoreMode = 1;            // 1: 16-byte stores from registers; 2: bulk copies from shared memory
+constexpr int kStreamMaxTeamWarps = 4;                // a team's row piece is one TMA box: at most 256 8-byte units
+constexpr uint32_t kPieceBytes = 512;                 // of one row per warp: 32 lanes x 16 bytes
+// shared-memory header: a line per team (barriers, counters), the step's masks
+constexpr uint32_t kTeamLineBytes = 128;              // [8] mbarriers, then [8] int counters of warps done with a stage
+constexpr uint32_t kMaskOffset = kStreamMaxWarps * kTeamLineBytes;  // up[64], down[64] u64, inv[64] f32
+constexpr uint32_t kStreamHeaderBytes = kMaskOffset + 2 * kMaxWorkers * 8 + kMaxWorkers * 4 + 256;
+static_assert(kStreamHeaderBytes % 128 == 0, "stages start on 128-byte boundaries");
+static_assert(kStreamMaxStages * (8 + 4) <= kTeamLineBytes, "a team's barriers and counters fit its line");
+static_assert(kStreamMaxTeamWarps * kPieceBytes / 8 <= 256, "a team's row piece is one box");
+
+struct StreamShape {
+    int32_t tiles;            // team tiles in the row
+    int32_t stages;           // depth of every team's ring
+    int32_t team_warps;       // warps per team: a tile is team_warps x 32 slices wide
+    int32_t teams;            // teams per CTA
+    int32_t withhold_copies;  // test aid: nothing is ever copied, so that the waits run out
+    int32_t descending;       // 1: the tiles are taken from the last to the first (odd steps)
+    int32_t bulk_stores;      // 1: the average leaves through shared memory and bulk copies (see the kernel)
+    uint32_t out_offset;      // of the warps' output slots from the start of the rings
+    uint64_t wait_limit_ns;
+
+    __device__ __forceinline__ int tile_of_turn(int64_t turn) const
+    {
+        return descending ? tiles - 1 - (int)turn : (int)turn;
+    }
+};
+
+// The two steps of a lane whose slice is cut by a block boundary or by the end of the row, per column:
+// columns [0, cut) of the slice belong to block j, columns [cut, VEC) to block j + 1, columns from live_n on
+// do not exist.  Same arithmetic as the regular path (predicated add in worker order, one multiplication).
+// Out of line and on copies of the caller's registers: this is rare.
+template <typename T, int VEC>
+__device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[2][VEC], int k, int j, int j_next,
+                                            int cut, int live_n, uint64_t valid, const uint64_t* s_up,
+                                            const uint64_t* s_down, T* dst, int64_t pitch)
+{
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int w = k + h;
+        const uint32_t up_lo = (uint32_t)(s_up[j] >> w) & 1u, up_hi = (uint32_t)(s_up[j_next] >> w) & 1u;
+        const uint32_t keep_lo = (uint32_t)((~s_down[j] & valid) >> w) & 1u;
+        const uint32_t keep_hi = (uint32_t)((~s_down[j_next] & valid) >> w) & 1u;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            const bool live = e < live_n, hi = e >= cut;
+            add_if(sum[e], v[h][e], live ? (hi ? up_hi : up_lo) : 0u);
+            if (live && (hi ? keep_hi : keep_lo)) dst[(int64_t)w * pitch + e] = RowVec<T, VEC>::narrow(v[h][e]);
+        }
+    }
+}
+
+template <typename T, int VEC>
+__device__ __noinline__ void irregular_receivers(const float (&sum)[VEC], int n, int j, int j_next, int cut,
+                                                 int live_n, const uint64_t* s_down, const float* s_inv, T* dst,
+                                                 int64_t pitch)
+{
+    T avg[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) avg[e] = RowVec<T, VEC>::narrow(sum[e] * (e >= cut ? s_inv[j_next] : s_inv[j]));
+    const uint64_t down_lo = s_down[j], down_hi = s_down[j_next];
+#pragma unroll 1
+    for (int i = 0; i < n; ++i) {
+        const bool lo = (down_lo >> i) & 1u, hi = (down_hi >> i) & 1u;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e)
+            if (e < live_n && (e >= cut ? hi : lo)) dst[(int64_t)i * pitch + e] = avg[e];
+    }
+}
+
+// 16 bytes of a row from VEC / 2 column pairs, rounded to T (nearest even).
+template <typename T, int VEC>
+__device__ __forceinline__ uint4 pack_pairs(const Float2 (&v)[VEC / 2])
+{
+    uint32_t w[4];
+    if (sizeof(T) == 4) {
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+            float lo, hi;
+            unpack2(v[m % (VEC / 2)], lo, hi);
+            w[2 * m] = __float_as_uint(lo), w[2 * m + 1] = __float_as_uint(hi);
+        }
+    } else {
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            float lo, hi;
+            unpack2(v[m % (VEC / 2)], lo, hi);
+            const __nv_bfloat162 pair = __floats2bfloat162_rn(lo, hi);
+            w[m] = *reinterpret_cast<const uint32_t*>(&pair);
+        }
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Waits for the phase with the given parity: one cheap test first (the data has usually landed long ago), then
+// the bounded wait.
+__device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;
+    return mbar_wait(bar, parity, limit_ns);
+}
+
+template <typename T, int VEC, int MAXW, int ROWS>
+__global__ void __launch_bounds__(MAXW * 32, 1)
+    rps_fused_stream_kernel(const __grid_constant__ FusedParams prm, const StreamShape shape,
+                            const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_b)
+{
+    constexpr int WARP_COLS = 32 * VEC;
+    static_assert(ROWS == 2 || ROWS == 4, "a stage holds one or two worker pairs");
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int n = prm.n;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int team = warp / shape.team_warps, member = warp - team * shape.team_warps;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + team * kTeamLineBytes);         // [stages] the rows have landed
+    int* done = reinterpret_cast<int*>(smem + team * kTeamLineBytes + kStreamMaxStages * 8);  // [stages] warps done with them
+    uint64_t* s_up = reinterpret_cast<uint64_t*>(smem + kMaskOffset);
+    uint64_t* s_down = s_up + kMaxWorkers;
+    float* s_inv = reinterpret_cast<float*>(s_down + kMaxWorkers);
+    // a stage: ROWS rows of x, then ROWS rows of b, each row the team's piece (team_warps x 512 bytes)
+    const uint32_t row_bytes = (uint32_t)shape.team_warps * kPieceBytes;
+    const uint32_t array_bytes = ROWS * row_bytes;
+    const uint32_t stage_bytes = 2 * array_bytes;
+    unsigned char* ring = smem + kStreamHeaderBytes + (size_t)team * shape.stages * stage_bytes;
+    const uint32_t ring_addr = smem_addr(ring);
+    const int team_cols = shape.team_warps * WARP_COLS;
+    const int32_t units_per_tile = (int32_t)(row_bytes / 8);  // 8-byte units of one row of a tile
+
+    // tiles of this team: turns g, g + teams_total, ...
+    const int teams_total = (int)gridDim.x * shape.teams;
+    const int g = (int)blockIdx.x * shape.teams + team;
+    const int my_tiles = g < shape.tiles ? (shape.tiles - g + teams_total - 1) / teams_total : 0;
+    const int chunks_per_tile = (n + ROWS - 1) / ROWS;
+    const uint32_t total = (uint32_t)my_tiles * (uint32_t)chunks_per_tile;  // stages' worth of rows this team goes through
+
+    if (member == 0 && lane == 0) {
+        for (int s = 0; s < shape.stages; ++s) {
+            mbar_init(smem_addr(&full[s]), 1);
+            done[s] = 0;
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (threadIdx.x == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    }
+    // With programmatic stream serialization this CTA may have been placed while the kernel before it in
+    // the stream was still draining: let the next kernel do the same, then wait for the one before to
+    // complete before reading anything from global memory.  Both are no-ops in a plain launch.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (int j = threadIdx.x; j < kMaxWorkers; j += blockDim.x) {
+        const bool used = j < n;
+        s_up[j] = used ? prm.masks->up[j] : 0;
+        s_down[j] = used ? prm.masks->down[j] : 0;
+        s_inv[j] = used ? prm.masks->inv_cnt[j] : 0.0f;
+    }
+    __syncthreads();  // the only CTA-wide barrier
+
+    // Copies rows [ROWS * chunk, ROWS * chunk + ROWS) of the team's tile number `local` into `stage` (which must be
+    // free): one thread, one box per array.  Boxes arrive whole (rows past n and columns past the pitch as
+    // zeros), so the byte count is fixed.  The maps count columns in 8-byte units.
+    auto issue = [&](int stage, int local, int chunk) {
+        if (shape.withhold_copies) return;
+        const int tile = shape.tile_of_turn((int64_t)g + (int64_t)local * teams_total);
+        const uint32_t bar = smem_addr(&full[stage]);
+        const uint32_t dst = ring_addr + (uint32_t)stage * stage_bytes;
+        mbar_arrive_expect_tx(bar, stage_bytes);
+        tma_load_box(dst, &map_x, tile * units_per_tile, ROWS * chunk, bar);
+        tma_load_box(dst + array_bytes, &map_b, tile * units_per_tile, ROWS * chunk, bar);
+    };
+    // where the filling stands: every warp keeps the count (the warp that frees a stage refills it)
+    int fill_local = 0, fill_chunk = 0;
+    for (int s = 0; s < shape.stages; ++s) {
+        if ((uint32_t)s < total && member == 0 && lane == 0) issue(s, fill_local, fill_chunk);
+        if (++fill_chunk == chunks_per_tile) fill_chunk = 0, ++fill_local;
+    }
+
+    T* __restrict__ xg = static_cast<T*>(prm.x);
+    const uint64_t valid = n >= 64 ? ~(uint64_t)0 : (((uint64_t)1 << n) - 1);
+    const PackedScalars scalars(prm);
+    // bulk stores: two 512-byte slots per warp, used in turn by the warp's tiles
+    unsigned char* out_slots = smem + kStreamHeaderBytes + shape.out_offset + (size_t)warp * 2 * kPieceBytes;
+    const unsigned char* my_ring = ring + member * kPieceBytes + lane * 16;
+    int stage = 0;
+    uint32_t phase = 0, q = 0;
+    for (int local = 0; local < my_tiles; ++local) {
+        // ---- a new tile: this lane's columns, the masks of their block, an empty sum
+        const int tile = shape.tile_of_turn((int64_t)g + (int64_t)local * teams_total);
+        const int64_t c = (int64_t)tile * team_cols + member * WARP_COLS + lane * VEC;
+        T* dst = xg + c;
+        const int64_t left = prm.d - c;
+        const int live_n = left >= VEC ? VEC : (left > 0 ? (int)left : 0);
+        uint64_t up = 0, down = 0, keep = 0;  // a lane past the end of the row adds nothing and stores nothing
+        float inv = 0.0f;
+        int j = 0, j_next = 0, cut = VEC;
+        if (live_n > 0) {
+            j = block_of(c, prm);
+            j_next = j + 1 < n ? j + 1 : j;
+            const int64_t in_block = (int64_t)(j + 1) * prm.block_cols - prm.col_offset - c;
+            cut = in_block >= VEC ? VEC : (int)in_block;
+            up = s_up[j], down = s_down[j], inv = s_inv[j];
+            keep = ~down & valid;
+        }
+        const bool regular = live_n == 0 || (live_n == VEC && cut == VEC);
+        // the whole warp inside one block and inside the row: every lane's masks are the same words
+        const bool warp_whole = __all_sync(0xFFFFFFFFu, live_n == VEC && cut == VEC) &&
+                                __all_sync(0xFFFFFFFFu, j == __shfl_sync(0xFFFFFFFFu, j, 0));
+        Float2 sum[VEC / 2];
+#pragma unroll
+        for (int m = 0; m < VEC / 2; ++m) sum[m] = 0ull;  // (+0, +0)
+
+        for (int chunk = 0; chunk < chunks_per_tile; ++chunk, ++q) {
+            if (!__all_sync(0xFFFFFFFFu, stream_wait(smem_addr(&full[stage]), phase, shape.wait_limit_ns))) {
+                // Something this warp waited for never came: say so, and see the copies that may have been issued
+                // into the team's ring land (bounded) before this warp's part of the shared memory is given up.
+                report_timeout(prm, 2);
+                if (!shape.withhold_copies && lane == 0) {
+                    for (int s = 1; s < shape.stages && q + (uint32_t)s < total; ++s) {
+                        if (++stage == shape.stages) stage = 0, phase ^= 1u;
+                        if (!mbar_wait(smem_addr(&full[stage]), phase, shape.wait_limit_ns)) break;
+                    }
+                }
+                if (shape.bulk_stores && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+                return;
+            }
+            const unsigned char* src = my_ring + (size_t)stage * stage_bytes;
+#pragma unroll
+            for (int half = 0; half < ROWS / 2; ++half) {
+                const int k = ROWS * chunk + 2 * half;  // the pair's first worker
+                if (ROWS == 4 && k >= n) break;         // the last stage of a tile may hold one pair only
+                uint4 raw_x[2], raw_b[2];
+                raw_x[0] = *reinterpret_cast<const uint4*>(src + (2 * half) * row_bytes);
+                raw_x[1] = *reinterpret_cast<const uint4*>(src + (2 * half + 1) * row_bytes);
+                raw_b[0] = *reinterpret_cast<const uint4*>(src + array_bytes + (2 * half) * row_bytes);
+                raw_b[1] = *reinterpret_cast<const uint4*>(src + array_bytes + (2 * half + 1) * row_bytes);
+                Float2 v[2][VEC / 2];
+                local_sgd_pair_packed<T, VEC>(raw_x, raw_b, v, c, k, prm, scalars);
+                if (regular) {
+                    const uint32_t arrived = (uint32_t)(up >> k), kept = (uint32_t)(keep >> k) & 3u;
+                    // RS: the running sum over the workers whose copy arrived, in worker order
+#pragma unroll
+                    for (int m = 0; m < VEC / 2; ++m) add2_if(sum[m], v[0][m], arrived & 1u);
+#pragma unroll
+                    for (int m = 0; m < VEC / 2; ++m) add2_if(sum[m], v[1][m], arrived & 2u);
+                    // AG, the workers whose return message is lost: they keep v, which can go out now
+                    if (kept) {
+                        if (kept & 1u) __stcs(reinterpret_cast<uint4*>(dst + (int64_t)k * prm.pitch), pack_pairs<T, VEC>(v[0]));
+                        if (kept & 2u)
+                            __stcs(reinterpret_cast<uint4*>(dst + (int64_t)(k + 1) * prm.pitch), pack_pairs<T, VEC>(v[1]));
+                    }
+                } else {
+                    float sum_copy[VEC], v_copy[2][VEC];
+#pragma unroll
+                    for (int m = 0; m < VEC / 2; ++m) {
+                        unpack2(sum[m], sum_copy[2 * m], sum_copy[2 * m + 1]);
+                        unpack2(v[0][m], v_copy[0][2 * m], v_copy[0][2 * m + 1]);
+                        unpack2(v[1][m], v_copy[1][2 * m], v_copy[1][2 * m + 1]);
+                    }
+                    irregular_pair<T, VEC>(sum_copy, v_copy, k, j, j_next, cut, live_n, valid, s_up, s_down, dst, prm.pitch);
+#pragma unroll
+                    for (int m = 0; m < VEC / 2; ++m) sum[m] = pack2(sum_copy[2 * m], sum_copy[2 * m + 1]);
+                }
+            }
+            // This warp is done with the stage (its values have been used, so its reads have completed).  The
+            // last warp of the team to say so refills the stage with the rows that come `stages` stages later.
+            __syncwarp();
+            if (lane == 0) {
+                bool last = true;
+                if (shape.team_warps > 1) {
+                    uint32_t before;
+                    asm volatile("atom.relaxed.cta.shared::cta.add.u32 %0, [%1], 1;"
+                                 : "=r"(before) : "r"(smem_addr(&done[stage])) : "memory");
+                    last = before == (uint32_t)shape.team_warps - 1u;
+                    if (last) done[stage] = 0;  // seen by the stage's next readers through the barrier the refill completes
+                }
+                if (last && q + (uint32_t)shape.stages < total) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // reads before the unit's writes
+                    issue(stage, fill_local, fill_chunk);
+                }
+            }
+            if (++fill_chunk == chunks_per_tile) fill_chunk = 0, ++fill_local;
+            if (++stage == shape.stages) stage = 0, phase ^= 1u;
+        }
+
+        // ---- AG, the receivers: one average, rounded and packed once, to every row whose down bit is set
+        if (regular) {
+            const Float2 inv2 = pack2(inv, inv);
+            Float2 avg[VEC / 2];
+#pragma unroll
+            for (int m = 0; m < VEC / 2; ++m) avg[m] = mul2(sum[m], inv2);
+            const uint4 packed = pack_pairs<T, VEC>(avg);
+            if (warp_whole && shape.bulk_stores) {
+                // The warp's 512 bytes of averages go to one of its two slots in shared memory, and one thread
+                // sends the slot to every receiver's row with an asynchronous bulk copy: the rows are written by
+                // the copy unit, 512 bytes at a time, while the warp is already at its next tile.  A slot is
+                // reused two tiles later, once the copies that read it have done so.
+                unsigned char* slot = out_slots + (local & 1) * kPieceBytes;
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                __syncwarp();
+                *reinterpret_cast<uint4*>(slot + lane * 16) = packed;
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // visible to the copy unit
+                __syncwarp();
+                if (lane == 0) {
+                    const uint32_t src = smem_addr(slot);
+                    uint64_t rest = down;
+                    const T* row = dst;  // lane 0 holds the warp's first column
+#pragma unroll 4
+                    for (int i = 0; i < n; ++i, row += prm.pitch, rest >>= 1)
+                        if (rest & 1u)
+                            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(row), "r"(src),
+                                         "n"(kPieceBytes)
+                                         : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+            } else {
+                uint64_t rest = down;
+                T* row = dst;
+#pragma unroll 4
+                for (int i = 0; i < n; ++i, row += prm.pitch, rest >>= 1)
+                    if (rest & 1u) __stcs(reinterpret_cast<uint4*>(row), packed);
+            }
+        } else {
+            float sum_copy[VEC];
+#pragma unroll
+            for (int m = 0; m < VEC / 2; ++m) unpack2(sum[m], sum_copy[2 * m], sum_copy[2 * m + 1]);
+            irregular_receivers<T, VEC>(sum_copy, n, j, j_next, cut, live_n, s_down, s_inv, dst, prm.pitch);
+        }
+    }
+    // the bulk copies issued by this thread still read this CTA's shared memory: see them through
+    if (shape.bulk_stores && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+// Describes one [n][pitch] array to the TMA unit in 8-byte units (so that a box may span 2 KB of a row whatever
+// the replica type), with boxes of `rows` rows x team_warps x 512 bytes.  Row starts, the pitch and the part of a
+// row that may be read are multiples of 128 bytes.
+bool encode_row_boxes(CUtensorMap* map, const void* base, size_t elem, const FusedParams& prm, int team_warps, int rows)
+{
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (encode == nullptr) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)prm.cols_in_row * elem / 8, (cuuint64_t)prm.n};
+    const cuuint64_t strides[1] = {(cuuint64_t)prm.pitch * elem};  // bytes between rows
+    const cuuint32_t box[2] = {(cuuint32_t)team_warps * (kPieceBytes / 8), (cuuint32_t)rows};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(base), dims, strides, box, elem_strides,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <typename T, int VEC, int MAXW, int ROWS>
+cudaError_t launch_stream_as(const FusedParams& prm, const FusedTuning& tune, int warps, int team_warps, int sm_count,
+                             cudaStream_t stream)
+{
+    auto kernel = rps_fused_stream_kernel<T, VEC, MAXW, ROWS>;
+    static LaunchState state;
+    size_t smem_limit = 0;
+    cudaError_t err = smem_limit_of_device(state, &smem_limit);
+    if (err != cudaSuccess) return err;
+    constexpr int warp_cols = 32 * VEC;
+    StreamShape shape{};
+    shape.team_warps = team_warps;
+    shape.teams = warps / team_warps;
+    shape.stages = tune.stages > 0 ? tune.stages : kStreamDefaultStages;
+    if (shape.stages > kStreamMaxStages) shape.stages = kStreamMaxStages;
+    shape.bulk_stores = (tune.store_mode != 0 ? tune.store_mode : kStreamDefaultStoreMode) == 2;
+    // the rings, then (bulk stores) two 512-byte output slots per warp
+    auto ring_bytes = [&] {
+        return (size_t)shape.teams * team_warps * (shape.stages * (2 * ROWS * kPieceBytes) + (shape.bulk_stores ? 2 * kPieceBytes : 0));
+    };
+    while (shape.stages > 2 && kStreamHeaderBytes + ring_bytes() > smem_limit) --shape.stages;
+    while (shape.teams > 1 && kStreamHeaderBytes + ring_bytes() > smem_limit) --shape.teams;
+    if (kStreamHeaderBytes + ring_bytes() > smem_limit) return cudaErrorInvalidConfiguration;
+    shape.out_offset = (uint32_t)((size_t)shape.teams * team_warps * shape.stages * (2 * ROWS * kPieceBytes));
+    const int64_t team_cols = (int64_t)team_warps * warp_cols;
+    shape.tiles = (int32_t)((prm.d + team_cols - 1) / team_cols);
+    shape.wait_limit_ns = tune.wait_limit_ms > 0 ? (uint64_t)tune.wait_limit_ms * 1000000ull : kDefaultWaitLimitNs;
+    shape.withhold_copies = tune.withhold_copies;
+    shape.descending = prm.descending;
+    const uint32_t smem_bytes = kStreamHeaderBytes + (uint32_t)ring_bytes();
+    if ((err = grant_smem(state, kernel, smem_bytes)) != cudaSuccess) return err;
+    alignas(64) CUtensorMap map_x, map_b;
+    // boxes of ROWS workers x one team's row piece; loads may read up to the pitch (padding arrives and is ignored)
+    if (!encode_row_boxes(&map_x, prm.x, sizeof(T), prm, team_warps, ROWS) ||
+        !encode_row_boxes(&map_b, prm.b, sizeof(T), prm, team_warps, ROWS))
+        return cudaErrorInvalidValue;
+    // Persistent CTAs, one per SM; the teams take the tiles in fixed turns, so the step lasts as long as
+    // the team with the most tiles.  A few SMs fewer can even that out: take the grid, from the SM count
+    // down to 7/8 of it, that loses the least to the last, partly filled round of turns.
+    int64_t grid = sm_count;
+    if (grid * shape.teams > shape.tiles) grid = (shape.tiles + shape.teams - 1) / shape.teams;
+    if (grid < 1) grid = 1;
+    if (grid == sm_count) {
+        double best = 0.0;
+        for (int64_t cand = sm_count; cand >= sm_count - sm_count / 8 && cand >= 1; --cand) {
+            const int64_t teams_total = cand * shape.teams;
+            const int64_t rounds = (shape.tiles + teams_total - 1) / teams_total;
+            const double busy = (double)shape.tiles / (double)(rounds * shape.teams * sm_count);  // of all SMs' time
+            if (busy > best + 1e-9) best = busy, grid = cand;
+        }
+    }
+    cudaLaunchConfig_t config = {};
+    config.gridDim = dim3((unsigned)grid);
+    config.blockDim = dim3((unsigned)(shape.teams * team_warps) * 32);
+    config.dynamicSmemBytes = smem_bytes;
+    config.stream = stream;
+    cudaLaunchAttribute attribute[1];
+    attribute[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attribute[0].val.programmaticStreamSerializationAllowed = 1;
+    config.attrs = attribute;
+    config.numAttrs = tune.launch_overlap == 1 ? 0 : 1;
+    return cudaLaunchKernelEx(&config, kernel, prm, shape, map_x, map_b);
+}
+
+template <typename T, int VEC, int ROWS>
+cudaError_t launch_stream_for_warps(const FusedParams& prm, const FusedTuning& tune, int sm_count, cudaStream_t stream)
+{
+    // the register file is shared out by launch bound: 32 warps of 64 registers, 24 of 80, 20 of 96, 16 of 128
+    // defaults from sweeps on B200 (n = 64, bf16): 5 teams of 4 warps; 16 warps leave issue slots idle, 24 and
+    // more lose more to the memory system than they gain
+    int warps = tune.consumer_warps > 0 ? tune.consumer_warps : 20;
+    if (warps > kStreamMaxWarps) warps = kStreamMaxWarps;
+    int team_warps = tune.team_warps == 0 || tune.team_warps >= 4 ? 4 : (tune.team_warps >= 2 ? 2 : 1);
+    while (team_warps > warps) team_warps /= 2;
+    warps -= warps % team_warps;  // whole teams
+    if (warps <= 16) return launch_stream_as<T, VEC, 16, ROWS>(prm, tune, warps, team_warps, sm_count, stream);
+    if (warps <= 20) return launch_stream_as<T, VEC, 20, ROWS>(prm, tune, warps, team_warps, sm_count, stream);
+    if (warps <= 24) return launch_stream_as<T, VEC, 24, ROWS>(prm, tune, warps, team_warps, sm_count, stream);
+    return launch_stream_as<T, VEC, 32, ROWS>(prm, tune, warps, team_warps, sm_count, stream);
+}
+
+}  // namespace
+
+bool stream_kernel_covers(const FusedParams& prm, bool bf16)
+{
+    // plain model averaging, untracked, at least one worker pair, blocks at least as wide as a lane's slice
+    // (a slice then meets at most two blocks); TMA coordinates are 32-bit
+    return prm.n >= 2 && prm.trace == nullptr && !prm.average_gradients && prm.block_cols >= (bf16 ? 8 : 4) &&
+           prm.pitch < ((int64_t)1 << 31);
+}
+
+cudaError_t launch_fused_stream(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
+                                cudaStream_t stream)
+{
+    if (!stream_kernel_covers(prm, bf16)) return cudaErrorInvalidConfiguration;
+    // rows per stage: two worker pairs, unless one pair is asked for (workers_per_lane = 2)
+    const bool one_pair = tune.workers_per_lane == 2 || prm.n <= 2;
+    if (bf16)
+        return one_pair ? launch_stream_for_warps<__nv_bfloat16, 8, 2>(prm, tune, sm_count, stream)
+                        : launch_stream_for_warps<__nv_bfloat16, 8, 4>(prm, tune, sm_count, stream);
+    return one_pair ? launch_stream_for_warps<float, 4, 2>(prm, tune, sm_count, stream)
+                    : launch_stream_for_warps<float, 4, 4>(prm, tune, sm_count, stream);
+}
+
+}  // namespace rps

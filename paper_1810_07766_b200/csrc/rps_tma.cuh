@@ -147,21 +147,28 @@ EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-// Describes one [n][pitch] array to the TMA unit, with boxes of n rows x box_cols columns; `cols` columns
+// Describes one [n][pitch] array to the TMA unit, with boxes of box_rows rows x box_cols columns; `cols` columns
 // of every row belong to the tensor (the pitch for loads, d for stores: what lies beyond is not written).
-bool encode_rows(CUtensorMap* map, const void* base, bool bf16, const FusedParams& prm, int box_cols, int64_t cols)
+bool encode_boxes(CUtensorMap* map, const void* base, bool bf16, const FusedParams& prm, int box_cols, int box_rows,
+                  int64_t cols)
 {
     EncodeTiledFn encode = encode_tiled_fn();
     if (encode == nullptr) return false;
     const size_t elem = bf16 ? 2 : 4;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)prm.n};
     const cuuint64_t strides[1] = {(cuuint64_t)prm.pitch * elem};  // bytes between rows
-    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)prm.n};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const cuuint32_t elem_strides[2] = {1, 1};
     return encode(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
                   const_cast<void*>(base), dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The same with boxes that span all n rows.
+bool encode_rows(CUtensorMap* map, const void* base, bool bf16, const FusedParams& prm, int box_cols, int64_t cols)
+{
+    return encode_boxes(map, base, bf16, prm, box_cols, prm.n, cols);
 }
 
 }  // namespace

@@ -52,7 +52,7 @@ def test_options_pitch_and_state_errors(lib):
     h = ctypes.c_void_p()
     assert lib.rps_create(8, 11_173_962, 0.1, 0.05, 1, ctypes.byref(h)) == 0
     try:
-        assert lib.rps_pitch(h) == 11_173_984                      # rounded up to 32 floats
+        assert lib.rps_pitch(h) == 11_174_144                      # rounded up to a whole number of kilobytes
         opt = rps_options()
         assert lib.rps_default_options(ctypes.byref(opt)) == 0
         assert (opt.dtype, opt.assign, opt.self_delivery, opt.mask_window, opt.sigma) == (0, 0, 1, 32, 0.0)
@@ -64,10 +64,10 @@ def test_options_pitch_and_state_errors(lib):
         assert lib.rps_scratch_bytes(h) == 256 + 34 * 1792
         opt.dtype = 1
         assert lib.rps_configure(h, ctypes.byref(opt)) == 0
-        assert lib.rps_pitch(h) == 11_174_080                      # rounded up to 64 bf16, plus one skew line
+        assert lib.rps_pitch(h) == 11_174_400                      # the same in bf16
         for field, value in (("dtype", 7), ("assign", 2), ("self_delivery", 3), ("mask_window", 0),
-                             ("mask_window", 257), ("sigma", -1.0), ("kernel", 4), ("workers_per_lane", 3), ("stages", 1),
-                             ("stages", 9), ("consumer_warps", 25), ("slice_bytes", 4), ("store_mode", 4), ("wait_limit_ms", -1), ("withhold_copies", 2), ("average", 2), ("row_skew_lines", -2), ("copy_mode", 3),
+                             ("mask_window", 257), ("sigma", -1.0), ("kernel", 5), ("workers_per_lane", 3), ("stages", 1),
+                             ("stages", 9), ("consumer_warps", 33), ("slice_bytes", 4), ("store_mode", 4), ("wait_limit_ms", -1), ("withhold_copies", 2), ("average", 2), ("row_skew_lines", -2), ("copy_mode", 3),
                              ("traversal", 2), ("l2_policy", 3), ("launch_overlap", 3),
                              ("shard_cols", -1), ("shard_begin", 64), ("shard_cols", 11_173_963),
                              ("block_steps", -1), ("block_steps", 33), ("team_warps", -1), ("team_warps", 17)):
@@ -85,7 +85,7 @@ def test_options_pitch_and_state_errors(lib):
         assert lib.rps_configure(h, ctypes.byref(shard)) == -1
         shard.shard_begin, shard.shard_cols = 11_173_952, 10
         assert lib.rps_configure(h, ctypes.byref(shard)) == 0
-        assert lib.rps_pitch(h) == 32
+        assert lib.rps_pitch(h) == 256                                 # a shard of 10 floats: one kilobyte per row
         shard.shard_begin, shard.shard_cols = 0, 0
         shard.dtype = 1
         assert lib.rps_configure(h, ctypes.byref(shard)) == 0
