@@ -68,7 +68,7 @@ def blocked_kernel_digest() -> str:
 
 # rps_options fields that shape the kernels without changing what is computed (command-line flags of the same names)
 SHAPE_OPTIONS = ("kernel", "workers_per_lane", "stages", "consumer_warps", "copy_mode", "slice_bytes", "store_mode",
-                 "traversal", "l2_policy", "launch_overlap", "block_steps", "team_warps")
+                 "traversal", "l2_policy", "launch_overlap", "block_steps", "team_warps", "early_targets")
 
 
 def kernel_digest() -> str:
@@ -87,11 +87,12 @@ def fused_kernel_name(args, w) -> str:
     small = w.n * w.d * w.elem_bytes < 148 * 8192
     if args.kernel == 1 or (args.kernel == 0 and small):
         return "rps_fused_direct_kernel"
-    stream_built = w.n >= 2 and not (args.average_gradients or args.track)
+    stream_built = w.n >= 2 and not args.average_gradients
     staged_only = args.workers_per_lane or args.copy_mode or args.slice_bytes
-    if stream_built and (args.kernel == 4 or (args.kernel == 0 and w.dtype == "bf16" and w.n > 32 and not staged_only)):
+    wide = w.n > 32 or (args.track and w.n >= 32)
+    if stream_built and (args.kernel == 4 or (args.kernel == 0 and w.dtype == "bf16" and wide and not staged_only)):
         return "rps_fused_stream_kernel"
-    ring_built = w.dtype == "bf16" and w.n > 4 and not (args.average_gradients or args.track)
+    ring_built = w.dtype == "bf16" and w.n > 4 and not args.track
     staged_only = args.workers_per_lane or args.consumer_warps or args.copy_mode or args.slice_bytes
     if ring_built and (args.kernel == 3 or (args.kernel == 0 and not staged_only)):
         return "rps_fused_ring_kernel"
@@ -290,6 +291,8 @@ def measure(args, ctx, w, b, *, with_e2e, with_upwards, p_sweep=()):
     shape = {name: getattr(args, name) for name in SHAPE_OPTIONS}  # all 0 = the library's choice
     bytes_per_step = w.bytes_per_step * cols // w.d
 
+    mask_window = 32  # steps whose masks one launch of the mask kernel generates (rps_options.mask_window)
+
     def make(p, **more):
         r = binding.RPS(w.n, w.d, p, w.gamma, w.seed, dtype=w.dtype, sigma=w.sigma,
                         average_gradients=args.average_gradients, shard_begin=begin if sharded else 0,
@@ -311,7 +314,7 @@ def measure(args, ctx, w, b, *, with_e2e, with_upwards, p_sweep=()):
     with ClockSampler(local_rank) as clocks:
         r.step_n(max(args.warmup, 3))
         r.profile(True)
-        r.step_n(args.steps)
+        r.step_n(max(args.steps, mask_window + 1))  # long enough to see the mask kernel, which runs once per window
         fused_ms, fused_n, mask_ms, mask_n = r.profile_read()
         r.profile(False)
         total_ms, gpu_launches = timed_run(r)
@@ -342,7 +345,6 @@ def measure(args, ctx, w, b, *, with_e2e, with_upwards, p_sweep=()):
     if default_shape and NCU_TRAFFIC["kernel_digest"] == kernel_digest():
         traffic = NCU_TRAFFIC["bytes_per_launch"].get(w.name)
         traffic_cold = NCU_TRAFFIC["cold_bytes_per_launch"].get(w.name)
-    mask_window = 32  # steps whose masks one launch of the mask kernel generates (rps_options.mask_window)
     roofline = {
         "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
         "traffic": traffic, "traffic_cold_cache": traffic_cold, "peak_kind": f"of {peak_kind}",
@@ -581,6 +583,8 @@ def main(argv=None):
     ap.add_argument("--l2-policy", type=int, default=0, help="staged kernel: 1 plain loads, 2 targets evict-first")
     ap.add_argument("--launch-overlap", type=int, default=0,
                     help="staged kernel: 1 plain launches, 2 programmatic stream serialization (default)")
+    ap.add_argument("--early-targets", type=int, default=0,
+                    help="1: every copy waits for the kernel ahead in the stream; 2: the first stages' copies of b do not")
     ap.add_argument("--block-steps", type=int, default=0,
                     help="temporal blocking of rps_step_n: this many consecutive steps per pass over x and b (<= 32); "
                          "the pass is then bound by arithmetic, not by HBM (off by default)")

@@ -103,13 +103,15 @@ typedef struct rps_options {
                                  walks all n workers in order, two at a time, adding each v to the
                                  running sum and storing it at once where the return message is
                                  lost; the average is rounded once and stored to every receiver.
-                                 Every warp has a shared-memory ring of its own that it refills
-                                 itself; a warp reads and writes whole 512-byte pieces of rows
-                                 (plain untracked model averaging, n >= 2; any other step runs as
-                                 kernel 2).
-                                 0: kernel 1 for models too short to give every SM a tile, kernel 3
-                                 for bf16 replicas of more than 4 workers (unless an option that
-                                 shapes kernel 2 alone is set), else kernel 2                 */
+                                 Teams of warps share shared-memory rings of a few rows that they
+                                 refill themselves; a team reads whole 2 KB pieces of rows and a warp
+                                 writes whole 512-byte pieces (model averaging, tracked or not,
+                                 n >= 2, blocks of at least 16 bytes; any other step runs as
+                                 kernel 2 or 3).
+                                 0: kernel 1 for models too short to give every SM a tile, kernel 4
+                                 for bf16 replicas of more than 32 workers, kernel 3 for bf16
+                                 replicas of more than 4 workers (unless an option that shapes
+                                 kernel 2 alone is set), else kernel 2                        */
     int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */
     int32_t stages;           /* depth of the shared-memory ring(s) of kernels 2, 3 and 4 (2..8) */
     int32_t consumer_warps;   /* compute warps per CTA of kernel 2 (1..24; shapes that need
@@ -122,7 +124,9 @@ typedef struct rps_options {
                                  lane, 2: through an output tile in shared memory with TMA tensor
                                  stores, 3: in place in the stage, with TMA tensor stores from
                                  there (kernel 2: by a store warp; kernel 3: by the last warp of
-                                 a team to have written)                                      */
+                                 a team to have written).  Kernel 4: 1 from registers, 2 the
+                                 average through a 512-byte slot in shared memory and one bulk
+                                 copy per receiving row                                        */
     int32_t wait_limit_ms;    /* kernel 2: every wait of a warp on data or on a free stage gives
                                  up after this many milliseconds (0 = 2000); the next
                                  synchronising call then returns RPS_ECUDA                   */
@@ -163,7 +167,18 @@ typedef struct rps_options {
      * and only to untracked model averaging.                                                         */
     int32_t block_steps;
     int32_t team_warps;       /* kernel 3: warp slices per tile, 1..16 (0 = the library's choice: 8, or
-                                 fewer where the ring would otherwise be too shallow)             */
+                                 fewer where the ring would otherwise be too shallow); kernel 4: warps
+                                 per team, 1, 2 or 4 (0 = 4): a team's row piece is team_warps x 512 bytes */
+    int32_t early_targets;    /* kernels 2 and 4 under launch_overlap = 2: 2 = the copies of the targets b
+                                 for a CTA's first stages are issued BEFORE the CTA waits for the kernel
+                                 ahead of it in the stream, so they arrive while that kernel drains; only
+                                 the copies of x wait.  This relies on b not being written by that
+                                 kernel: no kernel of this library writes b, and the library's own
+                                 uploads (rps_set_targets, rps_step_host) are copies, which a kernel
+                                 launch never overtakes.  A caller whose OWN kernel writes b on the bound
+                                 stream directly before a step must set 1 (every copy waits) or put a
+                                 stream synchronisation or an event between the two.  0 = the library's
+                                 choice (2 for kernel 2, 1 for kernel 4).                          */
 } rps_options;
 
 /*
@@ -303,8 +318,7 @@ int rps_estimate_alpha(rps_handle* h, uint64_t t0, int64_t steps, double* alpha1
  * trace_dev[2k+1] the value sum_i ||x^(i) - xbar||^2 of the state x_{t+1} it produces (for bf16
  * replicas: of the rounded values it stores).  fp32 arithmetic relative to a per-column pivot
  * within a tile of columns, fp64 across tiles; the order of the fp64 additions is not fixed, so the
- * last bits vary from run to run.  Tracked steps run in the lane shape with 4 workers per lane
- * whatever workers_per_lane says.  trace_dev == NULL or capacity == 0 switches tracking off.
+ * last bits vary from run to run.  trace_dev == NULL or capacity == 0 switches tracking off.
  * Errors: RPS_ESTATE before rps_bind, RPS_EINVAL for a negative capacity or a misaligned pointer.
  */
 int rps_track(rps_handle* h, double* trace_dev, int64_t capacity);
@@ -361,7 +375,11 @@ int rps_profile_read(rps_handle* h, double* fused_ms, int64_t* fused_launches, d
  * needs clearing, but two calls that overlap on the GPU (different streams, or
  * different host threads on different streams) race on it: keep them on one
  * stream or order them with events.  Returns RPS_OK, RPS_EINVAL, RPS_ELIMIT or
- * RPS_ECUDA; asynchronous like rps_step().
+ * RPS_ECUDA; asynchronous like rps_step().  One difference from the handle path:
+ * there is no error word here for a kernel to write, so a bounded wait inside the
+ * fused kernel that gives up (which rps_read() on a handle reports as RPS_ECUDA)
+ * ends that kernel early WITHOUT any report, with x partly updated.  Callers that
+ * need that report use a handle.
  */
 int rps_step_static(int n, int64_t d, int dtype, void* x_dev, const void* b_dev, int64_t pitch, double p,
                     double gamma, double sigma, uint64_t seed, uint64_t t, void* cuda_stream);

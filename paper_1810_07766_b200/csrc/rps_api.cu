@@ -105,6 +105,7 @@ struct rps_handle {
         tune.l2_policy = opt.l2_policy;
         tune.launch_overlap = opt.launch_overlap;
         tune.team_warps = opt.team_warps;
+        tune.early_targets = opt.early_targets;
         return tune;
     }
     rps::StepMasks* window() const { return reinterpret_cast<rps::StepMasks*>(scratch + kDiagBytes); }
@@ -334,6 +335,7 @@ int rps_default_options(rps_options* opt)
     opt->shard_cols = 0;
     opt->block_steps = 0;
     opt->team_warps = 0;
+    opt->early_targets = 0;
     return RPS_OK;
 }
 
@@ -442,6 +444,8 @@ int rps_configure(rps_handle* h, const rps_options* opt)
         return fail(h, RPS_EINVAL, "block_steps must be in 0..mask_window");
     if (opt->team_warps < 0 || opt->team_warps > 16)
         return fail(h, RPS_EINVAL, "team_warps must be 0 (auto) or 1..16");
+    if (opt->early_targets < 0 || opt->early_targets > 2)
+        return fail(h, RPS_EINVAL, "early_targets must be 0 (auto), 1 or 2");
     h->opt = *opt;
     h->sigma = (float)opt->sigma;
     return RPS_OK;

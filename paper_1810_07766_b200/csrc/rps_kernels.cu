@@ -234,8 +234,9 @@ cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool b
     // bf16 replicas of more than 32 workers: workers streamed through the teams' rings (what is staged does not
     // grow with n, every row piece is 2 KB); measured side by side 5 % ahead of the ring kernel at n = 64 and
     // a third at n = 48, level with it or behind at n <= 32.
-    if (tune.kernel == 0 && bf16 && prm.n > 32 && stream_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 &&
-        tune.copy_mode == 0 && tune.slice_bytes == 0)
+    // Tracked steps take it from 32 workers on (0.64 against 0.73 ms per step at n = 32, 1.19 against 1.62 at n = 64).
+    if (tune.kernel == 0 && bf16 && (prm.n > 32 || (prm.trace != nullptr && prm.n >= 32)) &&
+        stream_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 && tune.copy_mode == 0 && tune.slice_bytes == 0)
         return launch_fused_stream(prm, tune, bf16, sm_count, stream);
     // bf16 replicas of more than 4 workers: the self-refilling ring (16 compute warps, no producer warp), unless an
     // option that shapes the staged kernel only was set.  Measured side by side it is 3-8 % ahead at every n.

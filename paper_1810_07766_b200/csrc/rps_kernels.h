@@ -114,6 +114,8 @@ struct FusedTuning {
     int32_t l2_policy;         // staged kernel: 1 plain loads, 2 targets loaded with the L2 evict-first hint
     int32_t launch_overlap;    // staged kernel: 1 plain launch, 2 programmatic stream serialization
     int32_t team_warps;        // ring kernel: warp slices per tile (1..16)
+    int32_t early_targets;     // staged and streamed kernels: 1 every copy waits for the kernel ahead in the stream,
+                               // 2 the copies of b for the first stages are issued before that wait
 };
 
 struct FusedParams {

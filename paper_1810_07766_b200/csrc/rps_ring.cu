@@ -116,7 +116,7 @@ struct RingCursor {
     }
 };
 
-template <typename T, int VEC, int WPT, int G>
+template <typename T, int VEC, int WPT, int G, bool GRAD>
 __global__ void __launch_bounds__(kRingWarps * 32, 1)
     rps_fused_ring_kernel(const FusedParams prm, const RingShape shape, const __grid_constant__ CUtensorMap map_x,
                           const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out)
@@ -257,6 +257,17 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
         unsigned char* x_base = x_ring + (size_t)at_x.stage * shape.array_bytes + lane_off;
         const unsigned char* b_base = b_ring + (size_t)at_b.stage * shape.array_bytes + lane_off;
 
+        auto hand_back = [&] {
+            __syncwarp();
+            if (lane == 0 && count_off(&bs.done[at_b.stage]) == (uint32_t)shape.team_warps - 1u) {
+                bs.done[at_b.stage] = 0;  // seen by the stage's next readers through the barrier the refill completes
+                const int64_t next = local + shape.b_stages;
+                if (next < my_tiles && !*abort_flag) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // reads before the unit's writes
+                    fill(next, !in_place, true);
+                }
+            }
+        };
         float v[WPT][VEC];
         {
             Raw raw_x[WPT], raw_b[WPT];
@@ -268,19 +279,24 @@ __global__ void __launch_bounds__(kRingWarps * 32, 1)
                 raw_b[w] = *reinterpret_cast<const Raw*>(b_base + (size_t)row * shape.row_bytes);
             }
             // This warp has everything it needs from the tile (from its b half, if results go back in place).
-            // The last warp to say so refills the stage with the tile that comes b_stages later.
-            __syncwarp();
-            if (lane == 0 && count_off(&bs.done[at_b.stage]) == (uint32_t)shape.team_warps - 1u) {
-                bs.done[at_b.stage] = 0;  // seen by the stage's next readers through the barrier the refill completes
-                const int64_t next = local + shape.b_stages;
-                if (next < my_tiles && !*abort_flag) {
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // reads before the unit's writes
-                    fill(next, !in_place, true);
-                }
-            }
-            local_sgd_raw<T, VEC, WPT, false>(raw_x, raw_b, v, c, w_first, prm);
+            // The last warp to say so refills the stage with the tile that comes b_stages later.  (Gradient
+            // averaging reads x a second time after the average and hands the tile back only then.)
+            if (!GRAD) hand_back();
+            local_sgd_raw<T, VEC, WPT, GRAD>(raw_x, raw_b, v, c, w_first, prm);
         }
         const uint32_t live_bits = average_and_select<VEC, WPT, G>(v, c, col_live, w_first, masks, cursor, prm);
+        if (GRAD) {
+            // v holds the update each worker applies (the average one where it arrived): x_{t+1} = x + update
+#pragma unroll
+            for (int w = 0; w < WPT; ++w) {
+                const int row = w_first + w < n ? w_first + w : n - 1;
+                float xv[VEC];
+                RowVec<T, VEC>::unpack(*reinterpret_cast<const Raw*>(x_base + (size_t)row * shape.row_bytes), xv);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) v[w][e] += xv[e];
+            }
+            hand_back();
+        }
         if (in_place || out_tiles) {
             unsigned char* out_base = x_base;
             const int out_slot = (int)((uint32_t)local % (uint32_t)shape.teams);
@@ -394,17 +410,19 @@ bool plan_ring(const FusedParams& prm, const FusedTuning& tune, int vec, int g, 
     return false;
 }
 
-template <typename T, int VEC, int WPT, int G>
+template <typename T, int VEC, int WPT, int G, bool GRAD = false>
 cudaError_t launch_ring_as(const FusedParams& prm, const FusedTuning& tune, int sm_count, cudaStream_t stream)
 {
-    auto kernel = rps_fused_ring_kernel<T, VEC, WPT, G>;
+    auto kernel = rps_fused_ring_kernel<T, VEC, WPT, G, GRAD>;
     static LaunchState state;  // of this instantiation, per device
     size_t smem_limit = 0;
     cudaError_t err = smem_limit_of_device(state, &smem_limit);
     if (err != cudaSuccess) return err;
     RingShape shape;
     uint32_t smem_bytes = 0;
-    if (!plan_ring(prm, tune, VEC, G, sizeof(T), smem_limit, &shape, &smem_bytes)) return cudaErrorInvalidConfiguration;
+    FusedTuning shaped = tune;
+    if (GRAD) shaped.store_mode = 1;  // gradient averaging is built with results leaving from registers
+    if (!plan_ring(prm, shaped, VEC, G, sizeof(T), smem_limit, &shape, &smem_bytes)) return cudaErrorInvalidConfiguration;
     constexpr bool bf16 = sizeof(T) == 2;
     alignas(64) CUtensorMap map_x, map_b, map_out;
     // loads may read up to the pitch (padding arrives and is ignored); stores end at column d
@@ -434,8 +452,8 @@ cudaError_t launch_ring_as(const FusedParams& prm, const FusedTuning& tune, int 
 
 bool ring_kernel_covers(const FusedParams& prm, bool bf16)
 {
-    // built for bf16 replicas with 8 workers per lane, plain model averaging, untracked; TMA coordinates are 32-bit
-    return bf16 && prm.n > 4 && prm.trace == nullptr && !prm.average_gradients && prm.pitch < ((int64_t)1 << 31);
+    // built for bf16 replicas with 8 workers per lane, untracked (models or gradients averaged); TMA coordinates are 32-bit
+    return bf16 && prm.n > 4 && prm.trace == nullptr && prm.pitch < ((int64_t)1 << 31);
 }
 
 cudaError_t launch_fused_ring(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
@@ -443,6 +461,12 @@ cudaError_t launch_fused_ring(const FusedParams& prm, const FusedTuning& tune, b
 {
     if (!ring_kernel_covers(prm, bf16)) return cudaErrorInvalidConfiguration;
     const int n = prm.n;
+    if (prm.average_gradients) {
+        if (n <= 8) return launch_ring_as<__nv_bfloat16, 8, 8, 1, true>(prm, tune, sm_count, stream);
+        if (n <= 16) return launch_ring_as<__nv_bfloat16, 8, 8, 2, true>(prm, tune, sm_count, stream);
+        if (n <= 32) return launch_ring_as<__nv_bfloat16, 8, 8, 4, true>(prm, tune, sm_count, stream);
+        return launch_ring_as<__nv_bfloat16, 8, 8, 8, true>(prm, tune, sm_count, stream);
+    }
     if (n <= 8) return launch_ring_as<__nv_bfloat16, 8, 8, 1>(prm, tune, sm_count, stream);
     if (n <= 16) return launch_ring_as<__nv_bfloat16, 8, 8, 2>(prm, tune, sm_count, stream);
     if (n <= 32) return launch_ring_as<__nv_bfloat16, 8, 8, 4>(prm, tune, sm_count, stream);

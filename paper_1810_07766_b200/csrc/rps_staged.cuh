@@ -47,6 +47,7 @@ constexpr uint32_t kAbortFlagOffset = kSmemHeaderBytes - 128;
 constexpr int kOutBuffers = 2;
 constexpr int kDefaultL2Policy = 1;
 constexpr int kDefaultLaunchOverlap = 2;
+constexpr int kDefaultEarlyTargets = 2;
 static_assert(kSmemHeaderBytes % 128 == 0, "tile data must start on a 128-byte boundary");
 
 struct StagedShape {
@@ -78,6 +79,10 @@ struct StagedShape {
     // on the columns the step before it touched last, which are still in L2 (and still dirty there).
     int32_t descending;
     int32_t evict_first_targets;  // 1: b is loaded with the L2 evict-first hint
+    // 1: the producer issues the copies of b for its first `stages` tiles BEFORE it waits for the kernel ahead of
+    // it in the stream (programmatic launch): the targets are not written by a step, so they can arrive while
+    // that kernel drains.  Only the copies of x wait.
+    int32_t early_targets;
 
     __device__ __forceinline__ int64_t tile_of_turn(int64_t turn) const { return descending ? tiles - 1 - turn : turn; }
 };
@@ -117,11 +122,70 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    constexpr uint32_t elem = (uint32_t)sizeof(T);
     // Launched with programmatic stream serialization this CTA may have been placed while the kernel before
     // it in the stream was still draining.  Let the kernel after this one do the same, then wait for the one
-    // before to complete (its writes visible) before reading anything from global memory: the masks here, x
-    // and b in the producer.  Both are no-ops in a plain launch.
+    // before to complete (its writes visible) before reading anything it may have written: the masks here, x
+    // in the producer.  Both are no-ops in a plain launch.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Copies of one tile into its stage, by the producer warp: the targets, the replicas, or both; `expect`
+    // announces the bytes of BOTH to the stage's barrier (once per tile, before its first copy).
+    auto copy_tile = [&](int stage, int64_t tile, bool with_x, bool with_b, bool expect) {
+        const unsigned char* x_bytes = static_cast<const unsigned char*>(prm.x);
+        const unsigned char* b_bytes = static_cast<const unsigned char*>(prm.b);
+        const uint64_t targets_policy = l2_evict_first_policy();
+        const int64_t c0 = tile * shape.tile_cols;
+        const uint32_t bar = smem_addr(&full[stage]);
+        const uint32_t dst = smem_addr(ring) + (uint32_t)stage * shape.stage_bytes;
+        if (shape.use_boxes) {
+            // one thread, a few copies: the TMA unit walks the n rows of each box itself.  Boxes are
+            // always delivered whole (zeros past the pitch), so the byte count is fixed.
+            if (lane == 0) {
+                if (expect) mbar_arrive_expect_tx(bar, 2u * (uint32_t)shape.boxes_per_tile * shape.box_tx_bytes);
+                for (int k = 0; k < shape.boxes_per_tile; ++k) {
+                    const int32_t col = (int32_t)c0 + k * shape.box_cols;
+                    if (with_x) tma_load_box(dst + (uint32_t)k * shape.box_bytes, &map_x, col, 0, bar);
+                    if (with_b) {
+                        if (shape.evict_first_targets)
+                            tma_load_box(dst + shape.array_bytes + (uint32_t)k * shape.box_bytes, &map_b, col, 0, bar,
+                                         targets_policy);
+                        else
+                            tma_load_box(dst + shape.array_bytes + (uint32_t)k * shape.box_bytes, &map_b, col, 0, bar);
+                    }
+                }
+            }
+        } else {
+            // one bulk copy per row and array, spread over the lanes; the last tile stops at the pitch
+            const int64_t cols_left = prm.cols_in_row - c0;
+            const uint32_t cols = (uint32_t)(cols_left < shape.tile_cols ? cols_left : shape.tile_cols);
+            const uint32_t bytes = cols * elem;
+            if (expect && lane == 0) mbar_arrive_expect_tx(bar, 2u * (uint32_t)n * bytes);
+            __syncwarp();
+            for (int i = lane; i < n; i += 32) {
+                const int64_t at = ((int64_t)i * prm.pitch + c0) * elem;
+                if (with_x) bulk_load_row(dst + (uint32_t)i * shape.row_bytes, x_bytes + at, bytes, bar);
+                if (with_b) {
+                    if (shape.evict_first_targets)
+                        bulk_load_row(dst + shape.array_bytes + (uint32_t)i * shape.row_bytes, b_bytes + at, bytes, bar,
+                                      targets_policy);
+                    else
+                        bulk_load_row(dst + shape.array_bytes + (uint32_t)i * shape.row_bytes, b_bytes + at, bytes, bar);
+                }
+            }
+        }
+    };
+    // the targets of the producer's first tiles, ahead of the wait (see StagedShape::early_targets)
+    int early_tiles = 0;
+    if (shape.early_targets && !shape.withhold_copies) {
+        __syncthreads();  // the barriers are initialised
+        if (warp == consumer_warps) {
+            if (shape.use_boxes && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+            for (int64_t turn = blockIdx.x; turn < shape.tiles && early_tiles < shape.stages; turn += gridDim.x) {
+                copy_tile(early_tiles, shape.tile_of_turn(turn), false, true, true);
+                ++early_tiles;
+            }
+        }
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kAbortFlagOffset);
     if (threadIdx.x == 0) *abort_flag = 0;
@@ -142,17 +206,13 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
     __syncthreads();
     // no CTA-wide barrier below this line: the producer warp runs ahead and leaves first
 
-    constexpr uint32_t elem = (uint32_t)sizeof(T);
     if (warp == consumer_warps) {
         // ---------------- producer warp: keeps the ring full
         if (shape.withhold_copies) return;
-        const unsigned char* x_bytes = static_cast<const unsigned char*>(prm.x);
-        const unsigned char* b_bytes = static_cast<const unsigned char*>(prm.b);
         if (shape.use_boxes && lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
         }
-        const uint64_t targets_policy = l2_evict_first_policy();
         int stage = 0;
         uint32_t phase = 0;
         int64_t issued = 0;
@@ -164,41 +224,9 @@ __global__ void __launch_bounds__((max_consumer_warps(WPT, VEC, (int)sizeof(T)) 
                 ok = false;
                 break;
             }
-            const int64_t c0 = tile * shape.tile_cols;
-            const uint32_t bar = smem_addr(&full[stage]);
-            const uint32_t dst = smem_addr(ring) + (uint32_t)stage * shape.stage_bytes;
-            if (shape.use_boxes) {
-                // one thread, a few copies: the TMA unit walks the n rows of each box itself.  Boxes are
-                // always delivered whole (zeros past the pitch), so the byte count is fixed.
-                if (lane == 0) {
-                    mbar_arrive_expect_tx(bar, 2u * (uint32_t)shape.boxes_per_tile * shape.box_tx_bytes);
-                    for (int k = 0; k < shape.boxes_per_tile; ++k) {
-                        const int32_t col = (int32_t)c0 + k * shape.box_cols;
-                        tma_load_box(dst + (uint32_t)k * shape.box_bytes, &map_x, col, 0, bar);
-                        if (shape.evict_first_targets)
-                            tma_load_box(dst + shape.array_bytes + (uint32_t)k * shape.box_bytes, &map_b, col, 0, bar,
-                                         targets_policy);
-                        else
-                            tma_load_box(dst + shape.array_bytes + (uint32_t)k * shape.box_bytes, &map_b, col, 0, bar);
-                    }
-                }
-            } else {
-                // one bulk copy per row and array, spread over the lanes; the last tile stops at the pitch
-                const int64_t cols_left = prm.cols_in_row - c0;
-                const uint32_t cols = (uint32_t)(cols_left < shape.tile_cols ? cols_left : shape.tile_cols);
-                const uint32_t bytes = cols * elem;
-                if (lane == 0) mbar_arrive_expect_tx(bar, 2u * (uint32_t)n * bytes);
-                __syncwarp();
-                for (int i = lane; i < n; i += 32) {
-                    const int64_t at = ((int64_t)i * prm.pitch + c0) * elem;
-                    bulk_load_row(dst + (uint32_t)i * shape.row_bytes, x_bytes + at, bytes, bar);
-                    if (shape.evict_first_targets)
-                        bulk_load_row(dst + shape.array_bytes + (uint32_t)i * shape.row_bytes, b_bytes + at, bytes, bar,
-                                      targets_policy);
-                    else
-                        bulk_load_row(dst + shape.array_bytes + (uint32_t)i * shape.row_bytes, b_bytes + at, bytes, bar);
-                }
-            }
+            // the targets of the first tiles are on their way already, and their bytes announced
+            const bool early = issued < early_tiles;
+            copy_tile(stage, tile, true, !early, !early);
             ++issued;
             if (++stage == shape.stages) {
                 stage = 0;
@@ -459,6 +487,7 @@ bool shape_for(const FusedParams& prm, const FusedTuning& tune, int vec, int g, 
     sh.withhold_copies = tune.withhold_copies;
     sh.descending = prm.descending;
     sh.evict_first_targets = (tune.l2_policy != 0 ? tune.l2_policy : kDefaultL2Policy) == 2;
+    sh.early_targets = (tune.early_targets != 0 ? tune.early_targets : kDefaultEarlyTargets) == 2;
     sh.out_offset = (uint32_t)stages * sh.stage_bytes;
     out->threads = (warps + (store_mode == 3 ? 2 : 1)) * 32;
     out->smem_bytes = kSmemHeaderBytes + (uint32_t)stages * sh.stage_bytes + (uint32_t)out_total;

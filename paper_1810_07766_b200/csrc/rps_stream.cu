@@ -14,12 +14,17 @@
 //     stores alike (the lane-group forms store 64-byte pieces at n = 64), and the shared memory a warp needs
 //     does not grow with n: what is staged is a worker pair, not a tile of all workers.
 //   * Warps work in teams of team_warps neighbours.  A team owns a ring in shared memory whose stage holds
-//     one worker pair of the team's tile: 2 rows x (team_warps x 512 bytes) of x and of b, fetched by two TMA box
-//     copies (the arrays are described to the unit in 8-byte units, so one box spans up to 2 KB of a row).  A
-//     warp copies its part of a stage to registers and counts itself off; the warp that counts last refills
-//     the stage with the pair that comes `stages` pairs later (of the same tile or of the team's next one).
-//     Nobody waits for a free stage; the only wait is the bounded one for a stage's copies to land.  Teams
-//     take the tiles in fixed turns, so every warp knows the whole sequence of pairs in advance.
+//     one or two worker pairs of the team's tile: ROWS rows x (team_warps x 512 bytes) of x and of b, fetched by
+//     two TMA box copies (the arrays are described to the unit in 8-byte units, so one box spans up to 2 KB of a
+//     row; with rows that start on 1 KB boundaries every row piece is a whole number of DRAM pages).  A warp
+//     works through its part of a stage and counts itself off; the warp that counts last refills the stage with
+//     the rows that come `stages` stages later (of the same tile or of the team's next one).  Nobody waits for
+//     a free stage; the only wait is the bounded one for a stage's copies to land.  Teams take the tiles in
+//     fixed turns, so every warp knows the whole sequence of stages in advance.
+//   * The arithmetic runs two columns at a time in the packed fp32 forms (fma / mul / add .f32x2): one issue
+//     slot, two IEEE operations, the same bits as the scalar forms of the other kernels.
+//   * Tracked steps (DIAG) get their sums from the same walk: every receiver holds the same value, so only
+//     the keepers have a deviation from it (see TrackCols).
 //
 // A lane whose slice straddles two blocks or the end of the row (at most n such lanes per step) takes a
 // per-column branch with the same arithmetic, so a column's result does not depend on where it lies.
@@ -42,7 +47,8 @@ constexpr uint32_t kPieceBytes = 512;                 // of one row per warp: 32
 // shared-memory header: a line per team (barriers, counters), the step's masks
 constexpr uint32_t kTeamLineBytes = 128;              // [8] mbarriers, then [8] int counters of warps done with a stage
 constexpr uint32_t kMaskOffset = kStreamMaxWarps * kTeamLineBytes;  // up[64], down[64] u64, inv[64] f32
-constexpr uint32_t kStreamHeaderBytes = kMaskOffset + 2 * kMaxWorkers * 8 + kMaxWorkers * 4 + 256;
+constexpr uint32_t kTrackOffset = kMaskOffset + 2 * kMaxWorkers * 8 + kMaxWorkers * 4;  // tracked steps: 2 doubles, a counter
+constexpr uint32_t kStreamHeaderBytes = kTrackOffset + 256;
 static_assert(kStreamHeaderBytes % 128 == 0, "stages start on 128-byte boundaries");
 static_assert(kStreamMaxStages * (8 + 4) <= kTeamLineBytes, "a team's barriers and counters fit its line");
 static_assert(kStreamMaxTeamWarps * kPieceBytes / 8 <= 256, "a team's row piece is one box");
@@ -55,6 +61,7 @@ struct StreamShape {
     int32_t withhold_copies;  // test aid: nothing is ever copied, so that the waits run out
     int32_t descending;       // 1: the tiles are taken from the last to the first (odd steps)
     int32_t bulk_stores;      // 1: the average leaves through shared memory and bulk copies (see the kernel)
+    int32_t early_targets;    // 1: the first stages' copies of b are issued before the wait for the kernel ahead in the stream
     uint32_t out_offset;      // of the warps' output slots from the start of the rings
     uint64_t wait_limit_ns;
 
@@ -64,14 +71,41 @@ struct StreamShape {
     }
 };
 
+// Tracked steps (distance of the averaged model to the optimum, consensus error; see Tracker in rps_device.cuh),
+// in the streamed form.  Every receiver of a block holds the same stored value P, so with P as the pivot
+// only the workers that keep their own v (down bit clear) have a deviation: per column a lane keeps
+//   bsum = sum_k b_k,  a0 = v of worker 0 (a provisional pivot, P is not known until the last worker),
+//   D0 = sum over keepers (v_k - a0),  Q0 = sum over keepers (v_k - a0)^2        (v_k as stored),
+// and closes the column with delta = a0 - P, m keepers:  D = D0 + m delta,  Q = Q0 + 2 delta D0 + m delta^2,
+//   mean x = P + D / n,   consensus = Q - D^2 / n.   Nothing large is squared and subtracted.
+template <int VEC>
+struct TrackCols {
+    float bsum[VEC], a0[VEC], d0[VEC], q0[VEC];
+};
+
+// One column's contribution to (|| mean x - mean b ||^2, consensus error).  `receivers` = workers that hold
+// `stored_avg`; with none of them the provisional pivot stays.
+__device__ __forceinline__ void close_tracked_column(float bsum, float a0, float d0, float q0, float stored_avg,
+                                                     int keepers, int receivers, float inv_n, float& dist2, float& cons)
+{
+    const float pivot = receivers > 0 ? stored_avg : a0;
+    const float delta = a0 - pivot, m = (float)keepers;
+    const float dev_sum = fmaf(m, delta, d0);
+    const float dev_sq = fmaf(m * delta, delta, fmaf(2.0f * delta, d0, q0));
+    const float gap = fmaf(dev_sum - bsum, inv_n, pivot);  // mean x - mean b of this column
+    dist2 = fmaf(gap, gap, dist2);
+    cons += fmaf(-dev_sum * inv_n, dev_sum, dev_sq);
+}
+
 // The two steps of a lane whose slice is cut by a block boundary or by the end of the row, per column:
 // columns [0, cut) of the slice belong to block j, columns [cut, VEC) to block j + 1, columns from live_n on
 // do not exist.  Same arithmetic as the regular path (predicated add in worker order, one multiplication).
 // Out of line and on copies of the caller's registers: this is rare.
-template <typename T, int VEC>
+template <typename T, int VEC, bool DIAG>
 __device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[2][VEC], int k, int j, int j_next,
                                             int cut, int live_n, uint64_t valid, const uint64_t* s_up,
-                                            const uint64_t* s_down, T* dst, int64_t pitch)
+                                            const uint64_t* s_down, T* dst, int64_t pitch, TrackCols<VEC>* track,
+                                            const float (*b)[VEC])
 {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -83,15 +117,27 @@ __device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[
         for (int e = 0; e < VEC; ++e) {
             const bool live = e < live_n, hi = e >= cut;
             add_if(sum[e], v[h][e], live ? (hi ? up_hi : up_lo) : 0u);
-            if (live && (hi ? keep_hi : keep_lo)) dst[(int64_t)w * pitch + e] = RowVec<T, VEC>::narrow(v[h][e]);
+            const bool kept = live && (hi ? keep_hi : keep_lo);
+            const T stored = RowVec<T, VEC>::narrow(v[h][e]);
+            if (kept) dst[(int64_t)w * pitch + e] = stored;
+            if (DIAG && live) {
+                track->bsum[e] += b[h][e];
+                if (w == 0) track->a0[e] = v[0][e];
+                if (kept) {
+                    const float dev = (float)stored - track->a0[e];
+                    track->d0[e] += dev;
+                    track->q0[e] = fmaf(dev, dev, track->q0[e]);
+                }
+            }
         }
     }
 }
 
-template <typename T, int VEC>
+template <typename T, int VEC, bool DIAG>
 __device__ __noinline__ void irregular_receivers(const float (&sum)[VEC], int n, int j, int j_next, int cut,
                                                  int live_n, const uint64_t* s_down, const float* s_inv, T* dst,
-                                                 int64_t pitch)
+                                                 int64_t pitch, const TrackCols<VEC>* track, float inv_n, float* dist2,
+                                                 float* cons)
 {
     T avg[VEC];
 #pragma unroll
@@ -103,6 +149,17 @@ __device__ __noinline__ void irregular_receivers(const float (&sum)[VEC], int n,
 #pragma unroll
         for (int e = 0; e < VEC; ++e)
             if (e < live_n && (e >= cut ? hi : lo)) dst[(int64_t)i * pitch + e] = avg[e];
+    }
+    if (DIAG) {
+        float dd = 0.0f, q = 0.0f;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e)
+            if (e < live_n) {
+                const int receivers = __popcll(e >= cut ? down_hi : down_lo);
+                close_tracked_column(track->bsum[e], track->a0[e], track->d0[e], track->q0[e], (float)avg[e],
+                                     n - receivers, receivers, inv_n, dd, q);
+            }
+        *dist2 = dd, *cons = q;
     }
 }
 
@@ -146,7 +203,7 @@ __device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity, uint6
     return mbar_wait(bar, parity, limit_ns);
 }
 
-template <typename T, int VEC, int MAXW, int ROWS>
+template <typename T, int VEC, int MAXW, int ROWS, bool DIAG>
 __global__ void __launch_bounds__(MAXW * 32, 1)
     rps_fused_stream_kernel(const __grid_constant__ FusedParams prm, const StreamShape shape,
                             const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_b)
@@ -163,6 +220,9 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
     uint64_t* s_up = reinterpret_cast<uint64_t*>(smem + kMaskOffset);
     uint64_t* s_down = s_up + kMaxWorkers;
     float* s_inv = reinterpret_cast<float*>(s_down + kMaxWorkers);
+    // tracked steps: the CTA's pair of sums and the count of warps that have added theirs
+    double* track_pair = reinterpret_cast<double*>(smem + kTrackOffset);
+    int* track_arrivals = reinterpret_cast<int*>(smem + kTrackOffset + 16);
     // a stage: ROWS rows of x, then ROWS rows of b, each row the team's piece (team_warps x 512 bytes)
     const uint32_t row_bytes = (uint32_t)shape.team_warps * kPieceBytes;
     const uint32_t array_bytes = ROWS * row_bytes;
@@ -189,11 +249,44 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
     if (threadIdx.x == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+        if (DIAG) {
+            track_pair[0] = 0.0;
+            track_pair[1] = 0.0;
+            *track_arrivals = 0;
+        }
     }
+    // Copies rows [ROWS * chunk, ROWS * chunk + ROWS) of the team's tile number `local` into `stage` (which must be
+    // free): one thread, one box per array (the replicas, the targets, or both); `expect` announces the bytes of
+    // BOTH to the stage's barrier.  Boxes arrive whole (rows past n and columns past the pitch as zeros), so the
+    // byte count is fixed.  The maps count columns in 8-byte units.
+    auto issue = [&](int stage, int local, int chunk, bool with_x, bool with_b, bool expect) {
+        if (shape.withhold_copies) return;
+        const int tile = shape.tile_of_turn((int64_t)g + (int64_t)local * teams_total);
+        const uint32_t bar = smem_addr(&full[stage]);
+        const uint32_t dst = ring_addr + (uint32_t)stage * stage_bytes;
+        if (expect) mbar_arrive_expect_tx(bar, stage_bytes);
+        if (with_x) tma_load_box(dst, &map_x, tile * units_per_tile, ROWS * chunk, bar);
+        if (with_b) tma_load_box(dst + array_bytes, &map_b, tile * units_per_tile, ROWS * chunk, bar);
+    };
+    // the stages the ring starts with, filled by the team's first thread: stage s holds the team's chunk number s
+    auto first_fills = [&](bool with_x, bool with_b, bool expect) {
+        if (member != 0 || lane != 0) return;
+        int local = 0, chunk = 0;
+        for (int s = 0; s < shape.stages && (uint32_t)s < total; ++s) {
+            issue(s, local, chunk, with_x, with_b, expect);
+            if (++chunk == chunks_per_tile) chunk = 0, ++local;
+        }
+    };
     // With programmatic stream serialization this CTA may have been placed while the kernel before it in
     // the stream was still draining: let the next kernel do the same, then wait for the one before to
-    // complete before reading anything from global memory.  Both are no-ops in a plain launch.
+    // complete before reading anything it may have written.  Both are no-ops in a plain launch.  The targets
+    // are not written by a step: the copies of b for the first stages go out before the wait (early_targets)
+    // and arrive while that kernel drains; only the copies of x wait.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (shape.early_targets) {
+        __syncthreads();  // the barriers are initialised
+        first_fills(false, true, true);
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int j = threadIdx.x; j < kMaxWorkers; j += blockDim.x) {
         const bool used = j < n;
@@ -201,26 +294,12 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
         s_down[j] = used ? prm.masks->down[j] : 0;
         s_inv[j] = used ? prm.masks->inv_cnt[j] : 0.0f;
     }
-    __syncthreads();  // the only CTA-wide barrier
-
-    // Copies rows [ROWS * chunk, ROWS * chunk + ROWS) of the team's tile number `local` into `stage` (which must be
-    // free): one thread, one box per array.  Boxes arrive whole (rows past n and columns past the pitch as
-    // zeros), so the byte count is fixed.  The maps count columns in 8-byte units.
-    auto issue = [&](int stage, int local, int chunk) {
-        if (shape.withhold_copies) return;
-        const int tile = shape.tile_of_turn((int64_t)g + (int64_t)local * teams_total);
-        const uint32_t bar = smem_addr(&full[stage]);
-        const uint32_t dst = ring_addr + (uint32_t)stage * stage_bytes;
-        mbar_arrive_expect_tx(bar, stage_bytes);
-        tma_load_box(dst, &map_x, tile * units_per_tile, ROWS * chunk, bar);
-        tma_load_box(dst + array_bytes, &map_b, tile * units_per_tile, ROWS * chunk, bar);
-    };
+    __syncthreads();  // the last CTA-wide barrier
+    first_fills(true, !shape.early_targets, !shape.early_targets);
     // where the filling stands: every warp keeps the count (the warp that frees a stage refills it)
     int fill_local = 0, fill_chunk = 0;
-    for (int s = 0; s < shape.stages; ++s) {
-        if ((uint32_t)s < total && member == 0 && lane == 0) issue(s, fill_local, fill_chunk);
+    for (int s = 0; s < shape.stages; ++s)
         if (++fill_chunk == chunks_per_tile) fill_chunk = 0, ++fill_local;
-    }
 
     T* __restrict__ xg = static_cast<T*>(prm.x);
     const uint64_t valid = n >= 64 ? ~(uint64_t)0 : (((uint64_t)1 << n) - 1);
@@ -230,6 +309,7 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
     const unsigned char* my_ring = ring + member * kPieceBytes + lane * 16;
     int stage = 0;
     uint32_t phase = 0, q = 0;
+    Tracker<VEC, 2, 1> tracker;  // this lane's sums over its tiles, and the hand-over to the CTA's pair
     for (int local = 0; local < my_tiles; ++local) {
         // ---- a new tile: this lane's columns, the masks of their block, an empty sum
         const int tile = shape.tile_of_turn((int64_t)g + (int64_t)local * teams_total);
@@ -255,6 +335,11 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
         Float2 sum[VEC / 2];
 #pragma unroll
         for (int m = 0; m < VEC / 2; ++m) sum[m] = 0ull;  // (+0, +0)
+        TrackCols<VEC> track;
+        if (DIAG) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) track.bsum[e] = track.a0[e] = track.d0[e] = track.q0[e] = 0.0f;
+        }
 
         for (int chunk = 0; chunk < chunks_per_tile; ++chunk, ++q) {
             if (!__all_sync(0xFFFFFFFFu, stream_wait(smem_addr(&full[stage]), phase, shape.wait_limit_ns))) {
@@ -289,11 +374,38 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                     for (int m = 0; m < VEC / 2; ++m) add2_if(sum[m], v[0][m], arrived & 1u);
 #pragma unroll
                     for (int m = 0; m < VEC / 2; ++m) add2_if(sum[m], v[1][m], arrived & 2u);
+                    if (DIAG) {
+                        // tracked: the sum of the targets (rows past n arrive as zeros), the provisional pivot
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            float bv[VEC];
+                            RowVec<T, VEC>::unpack(raw_b[h], bv);
+#pragma unroll
+                            for (int e = 0; e < VEC; ++e) track.bsum[e] += bv[e];
+                        }
+                        if (k == 0) {
+#pragma unroll
+                            for (int m = 0; m < VEC / 2; ++m) unpack2(v[0][m], track.a0[2 * m], track.a0[2 * m + 1]);
+                        }
+                    }
                     // AG, the workers whose return message is lost: they keep v, which can go out now
                     if (kept) {
-                        if (kept & 1u) __stcs(reinterpret_cast<uint4*>(dst + (int64_t)k * prm.pitch), pack_pairs<T, VEC>(v[0]));
-                        if (kept & 2u)
-                            __stcs(reinterpret_cast<uint4*>(dst + (int64_t)(k + 1) * prm.pitch), pack_pairs<T, VEC>(v[1]));
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if (!((kept >> h) & 1u)) continue;
+                            const uint4 packed_v = pack_pairs<T, VEC>(v[h]);
+                            __stcs(reinterpret_cast<uint4*>(dst + (int64_t)(k + h) * prm.pitch), packed_v);
+                            if (DIAG) {
+                                float stored[VEC];  // as it will read back
+                                RowVec<T, VEC>::unpack(packed_v, stored);
+#pragma unroll
+                                for (int e = 0; e < VEC; ++e) {
+                                    const float dev = stored[e] - track.a0[e];
+                                    track.d0[e] += dev;
+                                    track.q0[e] = fmaf(dev, dev, track.q0[e]);
+                                }
+                            }
+                        }
                     }
                 } else {
                     float sum_copy[VEC], v_copy[2][VEC];
@@ -303,7 +415,15 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                         unpack2(v[0][m], v_copy[0][2 * m], v_copy[0][2 * m + 1]);
                         unpack2(v[1][m], v_copy[1][2 * m], v_copy[1][2 * m + 1]);
                     }
-                    irregular_pair<T, VEC>(sum_copy, v_copy, k, j, j_next, cut, live_n, valid, s_up, s_down, dst, prm.pitch);
+                    float b_copy[2][VEC];
+                    TrackCols<VEC> track_copy = track;
+                    if (DIAG) {
+                        RowVec<T, VEC>::unpack(raw_b[0], b_copy[0]);
+                        RowVec<T, VEC>::unpack(raw_b[1], b_copy[1]);
+                    }
+                    irregular_pair<T, VEC, DIAG>(sum_copy, v_copy, k, j, j_next, cut, live_n, valid, s_up, s_down, dst,
+                                                 prm.pitch, &track_copy, b_copy);
+                    if (DIAG) track = track_copy;
 #pragma unroll
                     for (int m = 0; m < VEC / 2; ++m) sum[m] = pack2(sum_copy[2 * m], sum_copy[2 * m + 1]);
                 }
@@ -322,7 +442,7 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                 }
                 if (last && q + (uint32_t)shape.stages < total) {
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // reads before the unit's writes
-                    issue(stage, fill_local, fill_chunk);
+                    issue(stage, fill_local, fill_chunk, true, true, true);
                 }
             }
             if (++fill_chunk == chunks_per_tile) fill_chunk = 0, ++fill_local;
@@ -366,13 +486,31 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                 for (int i = 0; i < n; ++i, row += prm.pitch, rest >>= 1)
                     if (rest & 1u) __stcs(reinterpret_cast<uint4*>(row), packed);
             }
+            if (DIAG && live_n == VEC) {
+                float stored_avg[VEC], dd = 0.0f, qq = 0.0f;
+                RowVec<T, VEC>::unpack(packed, stored_avg);
+                const int receivers = __popcll(down);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e)
+                    close_tracked_column(track.bsum[e], track.a0[e], track.d0[e], track.q0[e], stored_avg[e],
+                                         n - receivers, receivers, prm.inv_n, dd, qq);
+                tracker.dist2 += (double)dd;
+                tracker.cons += (double)qq;
+            }
         } else {
-            float sum_copy[VEC];
+            float sum_copy[VEC], dd = 0.0f, qq = 0.0f;
 #pragma unroll
             for (int m = 0; m < VEC / 2; ++m) unpack2(sum[m], sum_copy[2 * m], sum_copy[2 * m + 1]);
-            irregular_receivers<T, VEC>(sum_copy, n, j, j_next, cut, live_n, s_down, s_inv, dst, prm.pitch);
+            const TrackCols<VEC> track_copy = track;
+            irregular_receivers<T, VEC, DIAG>(sum_copy, n, j, j_next, cut, live_n, s_down, s_inv, dst, prm.pitch,
+                                              &track_copy, prm.inv_n, &dd, &qq);
+            if (DIAG) {
+                tracker.dist2 += (double)dd;
+                tracker.cons += (double)qq;
+            }
         }
     }
+    if (DIAG) tracker.flush(track_pair, track_arrivals, (int)(blockDim.x >> 5), prm.trace);
     // the bulk copies issued by this thread still read this CTA's shared memory: see them through
     if (shape.bulk_stores && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
@@ -393,11 +531,11 @@ bool encode_row_boxes(CUtensorMap* map, const void* base, size_t elem, const Fus
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <typename T, int VEC, int MAXW, int ROWS>
+template <typename T, int VEC, int MAXW, int ROWS, bool DIAG = false>
 cudaError_t launch_stream_as(const FusedParams& prm, const FusedTuning& tune, int warps, int team_warps, int sm_count,
                              cudaStream_t stream)
 {
-    auto kernel = rps_fused_stream_kernel<T, VEC, MAXW, ROWS>;
+    auto kernel = rps_fused_stream_kernel<T, VEC, MAXW, ROWS, DIAG>;
     static LaunchState state;
     size_t smem_limit = 0;
     cudaError_t err = smem_limit_of_device(state, &smem_limit);
@@ -422,6 +560,9 @@ cudaError_t launch_stream_as(const FusedParams& prm, const FusedTuning& tune, in
     shape.wait_limit_ns = tune.wait_limit_ms > 0 ? (uint64_t)tune.wait_limit_ms * 1000000ull : kDefaultWaitLimitNs;
     shape.withhold_copies = tune.withhold_copies;
     shape.descending = prm.descending;
+    // early copies of the targets: built and bit-identical, but worth nothing here (cfg5: 1.036 ms per step with
+    // them, 1.024 without, three alternating pairs on one box); the staged kernel gains 0.7 % on the smallest model
+    shape.early_targets = tune.early_targets == 2;
     const uint32_t smem_bytes = kStreamHeaderBytes + (uint32_t)ring_bytes();
     if ((err = grant_smem(state, kernel, smem_bytes)) != cudaSuccess) return err;
     alignas(64) CUtensorMap map_x, map_b;
@@ -474,13 +615,29 @@ cudaError_t launch_stream_for_warps(const FusedParams& prm, const FusedTuning& t
     return launch_stream_as<T, VEC, 32, ROWS>(prm, tune, warps, team_warps, sm_count, stream);
 }
 
+// Tracked steps: stages of two worker pairs, 16 warps unless asked otherwise (the per-column sums take
+// registers: 20 warps spill and were 6 % slower at n = 64).
+template <typename T, int VEC>
+cudaError_t launch_stream_tracked(const FusedParams& prm, const FusedTuning& tune, int sm_count, cudaStream_t stream)
+{
+    int warps = tune.consumer_warps > 0 ? tune.consumer_warps : 16;
+    if (warps > 20) warps = 20;
+    int team_warps = tune.team_warps == 0 || tune.team_warps >= 4 ? 4 : (tune.team_warps >= 2 ? 2 : 1);
+    while (team_warps > warps) team_warps /= 2;
+    warps -= warps % team_warps;
+    if (warps <= 16) return launch_stream_as<T, VEC, 16, 4, true>(prm, tune, warps, team_warps, sm_count, stream);
+    return launch_stream_as<T, VEC, 20, 4, true>(prm, tune, warps, team_warps, sm_count, stream);
+}
+
 }  // namespace
 
 bool stream_kernel_covers(const FusedParams& prm, bool bf16)
 {
-    // plain model averaging, untracked, at least one worker pair, blocks at least as wide as a lane's slice
-    // (a slice then meets at most two blocks); TMA coordinates are 32-bit
-    return prm.n >= 2 && prm.trace == nullptr && !prm.average_gradients && prm.block_cols >= (bf16 ? 8 : 4) &&
+    // model averaging (tracked or not), at least one worker pair, blocks at least as wide as a lane's slice
+    // (a slice then meets at most two blocks); TMA coordinates are 32-bit.  Not gradient averaging: a receiver's
+    // new value x + (average update) needs its own x after all workers have been seen, which this form has
+    // let go of by then.
+    return prm.n >= 2 && !prm.average_gradients && prm.block_cols >= (bf16 ? 8 : 4) &&
            prm.pitch < ((int64_t)1 << 31);
 }
 
@@ -488,6 +645,9 @@ cudaError_t launch_fused_stream(const FusedParams& prm, const FusedTuning& tune,
                                 cudaStream_t stream)
 {
     if (!stream_kernel_covers(prm, bf16)) return cudaErrorInvalidConfiguration;
+    if (prm.trace != nullptr)
+        return bf16 ? launch_stream_tracked<__nv_bfloat16, 8>(prm, tune, sm_count, stream)
+                    : launch_stream_tracked<float, 4>(prm, tune, sm_count, stream);
     // rows per stage: two worker pairs, unless one pair is asked for (workers_per_lane = 2)
     const bool one_pair = tune.workers_per_lane == 2 || prm.n <= 2;
     if (bf16)

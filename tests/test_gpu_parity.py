@@ -485,6 +485,53 @@ def test_full_size_whole_run_sampled_columns(rps_mod, oracle, name):
     torch.cuda.empty_cache()
 
 
+# ------------------------------------------------------------------ every element: laps of the rings, full sizes
+
+@pytest.mark.parametrize("n,d,dtype", [(8, 3_000_011, "f32"), (16, 2_400_003, "f32"), (32, 2_000_037, "f32"),
+                                       (32, 1_500_007, "bf16"), (64, 1_048_584, "bf16")])
+def test_default_shapes_lap_their_rings_every_element(rps_mod, oracle, n, d, dtype):
+    """The library's own choice of kernel for each kind of workload (staged with 4 and with 8 workers per lane,
+    the ring kernel, the streamed kernel) on a model long enough that every CTA takes a dozen or more tiles, so
+    that every stage of its ring is reused many times: three free-running steps, which walk the columns up, down
+    and up again, compared with the oracle's run in EVERY element."""
+    w = wl.Workload("laps", n=n, d=d, dtype=dtype, p=0.1, gamma=0.05, sigma=0.1, seed=4321 + n, steps=3)
+    b = wl.make_targets(w)
+    want = wl.make_initial(w)
+    oracle.run(want, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps)
+    r = make(rps_mod, w)
+    r.set_targets(b)
+    r.step_n(w.steps)
+    got = r.read()
+    r.close()
+    assert_close(w, got, want, BF16_TOL if dtype == "bf16" else 3 * STEP_TOL)
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
+def test_full_size_one_step_every_element(rps_mod, oracle, name):
+    """One step of the workload at its full size from a state in which every replica differs (worker i starts
+    from the targets of worker n-1-i), library defaults: the WHOLE state against the oracle's step, row by row."""
+    w = wl.WORKLOADS[name]
+    b = wl.make_targets(w)
+    x0 = np.ascontiguousarray(b[::-1])
+    want = x0.copy()
+    oracle.step(want, b, dtype=w.dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t=7)
+    r = make(rps_mod, w)
+    r.set_targets(b)
+    r.write(x0)
+    del x0, b
+    r.set_step(7)
+    r.step()
+    got = r.read()
+    r.close()
+    tol = BF16_TOL if w.dtype == "bf16" else STEP_TOL
+    worst = 0.0
+    for i in range(w.n):  # a row at a time keeps the fp64 copies small
+        g, o = wl.as_float64(w, got[i:i + 1]), wl.as_float64(w, want[i:i + 1])
+        worst = max(worst, float((np.abs(g - o) / (1.0 + np.abs(o))).max()))
+    assert worst <= tol, worst
+    torch.cuda.empty_cache()
+
+
 # ------------------------------------------------------------------ bounded waits
 
 @pytest.mark.parametrize("store_mode", [1, 2, 3])

@@ -79,9 +79,30 @@ def test_ring_options_do_not_change_a_bit(rps_mod):
         assert (np.concatenate(parts, axis=1) == ref).all()
 
 
+@pytest.mark.parametrize("n,d", [(5, 70_003), (8, 262_144), (17, 4097), (33, 20_011), (48, 50_001), (64, 300_007)])
+def test_ring_gradient_averaging_matches_the_oracle(rps_mod, oracle, n, d):
+    """Section 5's comparison method in the ring form (x is read a second time from the tile after the average,
+    and the tile is handed back only then): against the oracle, and bit for bit across teams and ring depths."""
+    w = wl.Workload("ring", n=n, d=d, dtype="bf16", p=0.2, gamma=0.05, sigma=0.1, seed=900 + n, steps=5, hetero=True)
+    b = wl.make_targets(w)
+    x0 = wl.f32_to_bf16_bits(np.random.default_rng(n * 7 + 1).standard_normal((n, d)).astype(np.float32))
+    want = x0.copy()
+    oracle.run(want, b, dtype="bf16", gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=3, steps=w.steps,
+               average_gradients=True)
+    ref = run(rps_mod, w, b, x0, w.steps, t0=3, kernel=3, average_gradients=True)
+    g, o = wl.as_float64(w, ref), wl.as_float64(w, want)
+    assert (np.abs(g - o) / (1 + np.abs(o))).max() <= BF16_TOL
+    for team_warps, stages, traversal in ((1, 2, 0), (4, 3, 1), (8, 2, 0), (16, 0, 1), (3, 5, 0)):
+        got = run(rps_mod, w, b, x0, w.steps, t0=3, kernel=3, average_gradients=True, team_warps=team_warps,
+                  stages=stages, traversal=traversal)
+        assert (got == ref).all(), (team_warps, stages, traversal)
+    # the library's own choice for this step is the same kernel
+    assert (run(rps_mod, w, b, x0, w.steps, t0=3, average_gradients=True) == ref).all()
+
+
 def test_steps_the_ring_is_not_built_for_run_as_the_staged_kernel(rps_mod, oracle):
-    """fp32 replicas, few workers, gradient averaging and tracked steps are not built in the ring form: asking
-    for kernel 3 must still give the right step."""
+    """fp32 replicas, few workers and tracked steps are not built in the ring form: asking for kernel 3 must still
+    give the right step (gradient averaging is built: it runs as the ring kernel)."""
     for n, dtype, extra in ((8, "f32", {}), (3, "bf16", {}), (16, "bf16", dict(average_gradients=True))):
         w = wl.Workload("ring", n=n, d=30_011, dtype=dtype, p=0.2, gamma=0.1, sigma=0.1, seed=5, steps=3)
         b = wl.make_targets(w)

@@ -79,7 +79,8 @@ def test_stream_matches_the_oracle_and_its_options_change_no_bit(rps_mod, oracle
                                 (12, 3, 4), (30, 2, 3)):
         got = run_(rps_mod, w, b, x0, w.steps, t0=3, kernel=4, consumer_warps=warps, stages=stages, team_warps=team)
         assert (got == ref).all(), (warps, stages, team, int((got != ref).sum()))
-    for opts in (dict(traversal=1), dict(launch_overlap=1), dict(mask_window=1), dict(workers_per_lane=2),
+    for opts in (dict(traversal=1), dict(launch_overlap=1), dict(mask_window=1), dict(early_targets=1),
+                 dict(early_targets=1, launch_overlap=1), dict(workers_per_lane=2),
                  dict(workers_per_lane=2, team_warps=4, consumer_warps=20, stages=6), dict(store_mode=2),
                  dict(store_mode=2, team_warps=4, consumer_warps=20, traversal=1)):
         if ("workers_per_lane" in opts or "store_mode" in opts) and not covered:
@@ -191,3 +192,63 @@ def test_a_stream_wait_that_runs_out_is_reported_and_harmless(rps_mod):
     assert (r.x_dev[:, :w.d].view(torch.int16).cpu().numpy().view(np.uint16) == x0.view(np.uint16)).all()
     r.close()
     assert (run(rps_mod, w, b, x0, 1, kernel=4, wait_limit_ms=20) == run(rps_mod, w, b, x0, 1, kernel=4)).all()
+
+
+TRACE_RTOL = 1e-4
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("n,d,self_delivery,p", [(2, 50_001, True, 0.3), (5, 70_003, True, 0.2), (17, 40_970, False, 0.7),
+                                                 (48, 50_001, True, 0.05), (64, 300_007, True, 0.1),
+                                                 (64, 65_536, False, 0.95), (12, 90_011, True, 1.0), (9, 8_200, True, 0.0)])
+def test_stream_tracked_steps_report_the_oracle_diagnostics(rps_mod, oracle, dtype, n, d, self_delivery, p):
+    """Tracked steps in the streamed form: every entry of the trace against the oracle's diagnostics of the state
+    that step left in memory (lanes on block boundaries and on the end of the row included, blocks that nobody
+    averages, everything and nothing delivered), and tracking changes no bit of x."""
+    w = wl.Workload("stream", n=n, d=d, dtype=dtype, p=p, gamma=0.1, sigma=0.1, seed=77 + n, steps=4, hetero=True)
+    b = wl.make_targets(w)
+    x0 = start(w, 9)
+    untracked = run(rps_mod, w, b, x0, w.steps, kernel=4, self_delivery=self_delivery)
+    for warps, team in ((0, 0), (16, 2), (5, 1)):
+        r = rps_mod.RPS(n, d, w.p, w.gamma, w.seed, dtype=dtype, sigma=w.sigma, kernel=4, self_delivery=self_delivery,
+                        consumer_warps=warps, team_warps=team)
+        r.set_targets(b)
+        r.write(x0)
+        r.track(w.steps)
+        states = []
+        for _ in range(w.steps):
+            r.step()
+            states.append(r.read())
+        trace = r.read_trace()
+        r.close()
+        assert trace.shape == (w.steps, 2)
+        for k, x in enumerate(states):
+            dist2, cons = oracle.diag(x, b, dtype=dtype)
+            assert abs(trace[k, 0] - dist2) <= TRACE_RTOL * dist2 + 1e-12 * n * d, (warps, k, trace[k, 0], dist2)
+            assert abs(trace[k, 1] - cons) <= TRACE_RTOL * cons + 1e-12 * n * d, (warps, k, trace[k, 1], cons)
+        assert (states[-1] == untracked).all()
+
+
+@pytest.mark.parametrize("n,d,dtype", [(8, 300_010, "f32"), (16, 100_008, "f32"), (32, 100_005, "f32"), (64, 65_536, "bf16"),
+                                       (3, 70_001, "bf16")])
+def test_targets_copied_ahead_of_the_wait_change_no_bit(rps_mod, n, d, dtype):
+    """The first stages' copies of b may be issued before a CTA waits for the step before it (early_targets):
+    with them, without them, in a plain launch and with targets replaced between steps by the library's own
+    upload, the staged and the streamed kernel give the same bits."""
+    w = wl.Workload("early", n=n, d=d, dtype=dtype, p=0.1, gamma=0.05, sigma=0.1, seed=11, steps=6)
+    b = wl.make_targets(w)
+    b2 = wl.make_targets(wl.Workload("early", n=n, d=d, dtype=dtype, p=0.1, gamma=0.05, sigma=0.1, seed=12, steps=6))
+    x0 = start(w, 4)
+    for kernel in (2, 4):
+        outs = []
+        for opts in (dict(early_targets=1), dict(early_targets=2), dict(early_targets=2, launch_overlap=1), dict()):
+            r = rps_mod.RPS(n, d, w.p, w.gamma, w.seed, dtype=dtype, sigma=w.sigma, kernel=kernel, **opts)
+            r.set_targets(b)
+            r.write(x0)
+            r.step_n(3)
+            r.set_targets(b2)  # an upload between two steps: the next step's early copies must see it
+            r.step_n(3)
+            outs.append(r.read())
+            r.close()
+        for other in outs[1:]:
+            assert (other == outs[0]).all(), kernel

@@ -50,7 +50,7 @@ def test_trace_equals_the_oracle_diagnostics_of_the_state_left_behind(rps_mod, o
                     hetero=True)
     b = wl.make_targets(w)
     worst = 0.0
-    for kernel, store_mode, copy_mode in ((1, 0, 0), (2, 1, 1), (2, 2, 2), (2, 3, 0)):
+    for kernel, store_mode, copy_mode in ((1, 0, 0), (2, 1, 1), (2, 2, 2), (2, 3, 0), (4, 0, 0)):
         r = rps_mod.RPS(n, d, w.p, w.gamma, w.seed, dtype=dtype, sigma=w.sigma, kernel=kernel, store_mode=store_mode,
                         copy_mode=copy_mode, average_gradients=average_gradients)
         r.set_targets(b)
