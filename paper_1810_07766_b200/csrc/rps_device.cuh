@@ -321,12 +321,22 @@ __device__ __forceinline__ Float2 add_noise_pair(Float2 v, uint32_t word, const 
     return fma2(pack2(z.radius, z.radius), pack2(z.c, z.s), v);
 }
 
+__device__ __forceinline__ Float2 add2(Float2 a, Float2 b)
+{
+    Float2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
 // Local SGD step of one lane on a worker pair (k even) x VEC columns from column c, from the raw slices, two
 // columns at a time: v = x + gamma (b - x) - (gamma sigma) xi.  Same bits as local_sgd_raw<T, VEC, 2, false>.
-template <typename T, int VEC>
+// TARGETS: also add the pair's targets to target_sum, as (b - x) + x from the values the step holds anyway
+// (equal to b up to one rounding of the difference; for the tracked steps' mean of the targets).
+template <typename T, int VEC, bool TARGETS = false>
 __device__ __forceinline__ void local_sgd_pair_packed(const uint4 (&raw_x)[2], const uint4 (&raw_b)[2],
                                                       Float2 (&v)[2][VEC / 2], int64_t c, int k,
-                                                      const FusedParams& prm, const PackedScalars& scalars)
+                                                      const FusedParams& prm, const PackedScalars& scalars,
+                                                      Float2* target_sum = nullptr)
 {
     static_assert(VEC * sizeof(T) == 16, "a slice is 16 bytes");
 #pragma unroll
@@ -337,7 +347,9 @@ __device__ __forceinline__ void local_sgd_pair_packed(const uint4 (&raw_x)[2], c
 #pragma unroll
             for (int m = 0; m < 2; ++m) {
                 const Float2 x2 = pack2(wx[2 * m], wx[2 * m + 1]);
-                v[h][m % (VEC / 2)] = fma2(scalars.gamma, sub2(pack2(wb[2 * m], wb[2 * m + 1]), x2), x2);
+                const Float2 b2 = pack2(wb[2 * m], wb[2 * m + 1]);
+                v[h][m % (VEC / 2)] = fma2(scalars.gamma, sub2(b2, x2), x2);
+                if (TARGETS) target_sum[m % (VEC / 2)] = add2(target_sum[m % (VEC / 2)], b2);
             }
         } else {
 #pragma unroll
@@ -345,7 +357,9 @@ __device__ __forceinline__ void local_sgd_pair_packed(const uint4 (&raw_x)[2], c
                 const float x_lo = __uint_as_float(wx[m] << 16), x_hi = __uint_as_float(wx[m] & 0xFFFF0000u);
                 float d_lo, d_hi;
                 bf16_pair_minus(wb[m], x_lo, x_hi, d_lo, d_hi);
-                v[h][m % (VEC / 2)] = fma2(scalars.gamma, pack2(d_lo, d_hi), pack2(x_lo, x_hi));
+                const Float2 d2 = pack2(d_lo, d_hi), x2 = pack2(x_lo, x_hi);
+                v[h][m % (VEC / 2)] = fma2(scalars.gamma, d2, x2);
+                if (TARGETS) target_sum[m % (VEC / 2)] = add2(target_sum[m % (VEC / 2)], add2(d2, x2));
             }
         }
     }

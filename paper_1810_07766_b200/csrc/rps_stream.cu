@@ -336,9 +336,12 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
 #pragma unroll
         for (int m = 0; m < VEC / 2; ++m) sum[m] = 0ull;  // (+0, +0)
         TrackCols<VEC> track;
+        Float2 target_sum[VEC / 2];  // tracked, regular lanes: the sum of the targets, two columns at a time
         if (DIAG) {
 #pragma unroll
             for (int e = 0; e < VEC; ++e) track.bsum[e] = track.a0[e] = track.d0[e] = track.q0[e] = 0.0f;
+#pragma unroll
+            for (int m = 0; m < VEC / 2; ++m) target_sum[m] = 0ull;
         }
 
         for (int chunk = 0; chunk < chunks_per_tile; ++chunk, ++q) {
@@ -366,7 +369,7 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                 raw_b[0] = *reinterpret_cast<const uint4*>(src + array_bytes + (2 * half) * row_bytes);
                 raw_b[1] = *reinterpret_cast<const uint4*>(src + array_bytes + (2 * half + 1) * row_bytes);
                 Float2 v[2][VEC / 2];
-                local_sgd_pair_packed<T, VEC>(raw_x, raw_b, v, c, k, prm, scalars);
+                local_sgd_pair_packed<T, VEC, DIAG>(raw_x, raw_b, v, c, k, prm, scalars, target_sum);
                 if (regular) {
                     const uint32_t arrived = (uint32_t)(up >> k), kept = (uint32_t)(keep >> k) & 3u;
                     // RS: the running sum over the workers whose copy arrived, in worker order
@@ -375,14 +378,8 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
 #pragma unroll
                     for (int m = 0; m < VEC / 2; ++m) add2_if(sum[m], v[1][m], arrived & 2u);
                     if (DIAG) {
-                        // tracked: the sum of the targets (rows past n arrive as zeros), the provisional pivot
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            float bv[VEC];
-                            RowVec<T, VEC>::unpack(raw_b[h], bv);
-#pragma unroll
-                            for (int e = 0; e < VEC; ++e) track.bsum[e] += bv[e];
-                        }
+                        // tracked: the provisional pivot (the targets were summed with the step: rows past n arrive
+                        // as zeros and add nothing)
                         if (k == 0) {
 #pragma unroll
                             for (int m = 0; m < VEC / 2; ++m) unpack2(v[0][m], track.a0[2 * m], track.a0[2 * m + 1]);
@@ -418,6 +415,7 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                     float b_copy[2][VEC];
                     TrackCols<VEC> track_copy = track;
                     if (DIAG) {
+                        // (an irregular lane's targets are summed per column there, not in the packed sum)
                         RowVec<T, VEC>::unpack(raw_b[0], b_copy[0]);
                         RowVec<T, VEC>::unpack(raw_b[1], b_copy[1]);
                     }
@@ -489,6 +487,8 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
             if (DIAG && live_n == VEC) {
                 float stored_avg[VEC], dd = 0.0f, qq = 0.0f;
                 RowVec<T, VEC>::unpack(packed, stored_avg);
+#pragma unroll
+                for (int m = 0; m < VEC / 2; ++m) unpack2(target_sum[m], track.bsum[2 * m], track.bsum[2 * m + 1]);
                 const int receivers = __popcll(down);
 #pragma unroll
                 for (int e = 0; e < VEC; ++e)
