@@ -40,12 +40,12 @@ FALLBACK_HBM_GBS = 6650.0
 # of this benchmark at full size with the caches left as the launch before left them (one-pass
 # capture), which is the state the timed steps run in: a step starts on the columns that the step
 # before it touched last, so part of x and b is still in L2 and the traffic is below the
-# algorithmic bytes.  "cold_bytes_per_launch": one launch alone with the caches flushed first
-# (cfg3 and cfg5 from captures at d/4 and d/8, scaled by 4 and 8).
+# algorithmic bytes.  "cold_bytes_per_launch": one launch alone at full size with the caches flushed first
+# (also a one-pass capture; the writes of the last lines are still in L2 when the launch ends).
 NCU_TRAFFIC = {
-    "kernel_digest": "fca028b86cf7191c",
-    "bytes_per_launch": {"cfg2": 953715942, "cfg3": 4804074214, "cfg4": 1432305587, "cfg5": 6350427366},
-    "cold_bytes_per_launch": {"cfg2": 1021500928, "cfg3": 4713249792, "cfg4": 1486095952, "cfg5": 6061942784},
+    "kernel_digest": "e1905f700f57feea",
+    "bytes_per_launch": {"cfg2": 963785472, "cfg3": 4806406886, "cfg4": 1432377165, "cfg5": 6413996672},
+    "cold_bytes_per_launch": {"cfg2": 1023124480, "cfg3": 4859331072, "cfg4": 1486761728, "cfg5": 6387706368},
 }
 
 
