@@ -68,7 +68,7 @@ def blocked_kernel_digest() -> str:
 
 # rps_options fields that shape the kernels without changing what is computed (command-line flags of the same names)
 SHAPE_OPTIONS = ("kernel", "workers_per_lane", "stages", "consumer_warps", "copy_mode", "slice_bytes", "store_mode",
-                 "traversal", "l2_policy", "launch_overlap", "block_steps", "team_warps", "early_targets")
+                 "traversal", "l2_policy", "launch_overlap", "block_steps", "team_warps", "early_targets", "fuse_steps")
 
 
 def kernel_digest() -> str:
@@ -314,7 +314,8 @@ def measure(args, ctx, w, b, *, with_e2e, with_upwards, p_sweep=()):
     with ClockSampler(local_rank) as clocks:
         r.step_n(max(args.warmup, 3))
         r.profile(True)
-        r.step_n(max(args.steps, mask_window + 1))  # long enough to see the mask kernel, which runs once per window
+        profile_steps = max(args.steps, mask_window + 1)  # long enough to see the mask kernel, which runs once per window
+        r.step_n(profile_steps)
         fused_ms, fused_n, mask_ms, mask_n = r.profile_read()
         r.profile(False)
         total_ms, gpu_launches = timed_run(r)
@@ -336,8 +337,10 @@ def measure(args, ctx, w, b, *, with_e2e, with_upwards, p_sweep=()):
 
     ms_per_step = total_ms / args.steps
     peak, peak_kind = measured_peak_gbs()
+    # a launch may run several steps (rps_options.fuse_steps): bytes per launch = bytes per step x steps per launch
     fused_avg_ms = fused_ms / max(fused_n, 1)
-    achieved = bytes_per_step / (fused_avg_ms * 1e-3) / 1e9
+    steps_per_launch = profile_steps / max(fused_n, 1)
+    achieved = bytes_per_step * steps_per_launch / (fused_avg_ms * 1e-3) / 1e9
     whole_step = bytes_per_step / (ms_per_step * 1e-3) / 1e9
     traffic = traffic_cold = None
     default_shape = not (any(shape.values()) or args.average_gradients or args.track or sharded or
@@ -347,14 +350,17 @@ def measure(args, ctx, w, b, *, with_e2e, with_upwards, p_sweep=()):
         traffic_cold = NCU_TRAFFIC["cold_bytes_per_launch"].get(w.name)
     roofline = {
         "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "traffic": traffic, "traffic_cold_cache": traffic_cold, "peak_kind": f"of {peak_kind}",
+        # per launch, like `achieved`: the recorded bytes are per step
+        "traffic": traffic * steps_per_launch if traffic else None, "traffic_per_step": traffic,
+        "traffic_cold_cache": traffic_cold, "peak_kind": f"of {peak_kind}",
         "kernel": fused_kernel_name(args, w), "avg_launch_ms": fused_avg_ms, "launches_timed": fused_n,
+        "steps_per_launch": steps_per_launch,
         # the same bytes over the time of a whole step inside a train of steps (launch overlap kept, mask kernel in)
         "whole_step_achieved": whole_step, "whole_step_frac": whole_step / peak,
         "whole_step_frac_of_8TBs_nominal": whole_step / 8000.0,
         # what crossed the HBM interface (ncu, when recorded for these sources) over the same times
-        "dram_achieved": traffic / (fused_avg_ms * 1e-3) / 1e9 if traffic else None,
-        "dram_frac": traffic / (fused_avg_ms * 1e-3) / 1e9 / peak if traffic else None,
+        "dram_achieved": traffic * steps_per_launch / (fused_avg_ms * 1e-3) / 1e9 if traffic else None,
+        "dram_frac": traffic * steps_per_launch / (fused_avg_ms * 1e-3) / 1e9 / peak if traffic else None,
         "dram_whole_step_achieved": traffic / (ms_per_step * 1e-3) / 1e9 if traffic else None,
         "dram_whole_step_frac_of_8TBs_nominal": traffic / (ms_per_step * 1e-3) / 8e12 if traffic else None,
         "note": "avg_launch_ms brackets every launch with events, which serialises the launches and loses the "
@@ -403,7 +409,7 @@ def blocked_roofline(args, ctx, w, cols, entry):
     torch, device = ctx["torch"], ctx["device"]
     old = entry["roofline"]
     fused_avg_ms, fused_n = old["avg_launch_ms"], old["launches_timed"]
-    steps_per_launch = args.steps / max(fused_n, 1)
+    steps_per_launch = old["steps_per_launch"]
     rp_steps_per_s = w.n * cols * steps_per_launch / (fused_avg_ms * 1e-3)
     sm_count = torch.cuda.get_device_properties(device).multi_processor_count
     mhz = entry["clocks"].get("sm_max_mhz") or 1965
@@ -585,6 +591,8 @@ def main(argv=None):
                     help="staged kernel: 1 plain launches, 2 programmatic stream serialization (default)")
     ap.add_argument("--early-targets", type=int, default=0,
                     help="1: every copy waits for the kernel ahead in the stream; 2: the first stages' copies of b do not")
+    ap.add_argument("--fuse-steps", type=int, default=0,
+                    help="rps_step_n: 1 one launch per step; 2 several steps per launch where the kernel takes them")
     ap.add_argument("--block-steps", type=int, default=0,
                     help="temporal blocking of rps_step_n: this many consecutive steps per pass over x and b (<= 32); "
                          "the pass is then bound by arithmetic, not by HBM (off by default)")

@@ -179,6 +179,14 @@ typedef struct rps_options {
                                  stream directly before a step must set 1 (every copy waits) or put a
                                  stream synchronisation or an event between the two.  0 = the library's
                                  choice (2 for kernel 2, 1 for kernel 4).                          */
+    int32_t fuse_steps;       /* rps_step_n: 2 = consecutive untracked steps are issued as ONE launch of the
+                                 fused kernel (up to the steps left in the window of masks) where the
+                                 kernel that serves this handle can go from step to step by itself
+                                 (kernel 4: a team of warps works on the same tiles in every step, and a
+                                 column's next step needs only that column's last step, so a team sees
+                                 its own stores done, fences, and goes on; no launch boundary, no wait
+                                 for the rest of the GPU).  Results are bit for bit those of single
+                                 steps.  1 = one launch per step.  0 = the library's choice (2).     */
 } rps_options;
 
 /*

@@ -44,7 +44,7 @@ class rps_options(ctypes.Structure):
                 ("withhold_copies", ctypes.c_int32), ("average", ctypes.c_int32),
                 ("traversal", ctypes.c_int32), ("l2_policy", ctypes.c_int32), ("launch_overlap", ctypes.c_int32),
                 ("shard_begin", ctypes.c_int64), ("shard_cols", ctypes.c_int64), ("block_steps", ctypes.c_int32),
-                ("team_warps", ctypes.c_int32), ("early_targets", ctypes.c_int32)]
+                ("team_warps", ctypes.c_int32), ("early_targets", ctypes.c_int32), ("fuse_steps", ctypes.c_int32)]
 
 
 def shard_columns(d: int, world: int, rank: int, align: int = 64) -> Tuple[int, int]:
@@ -150,7 +150,7 @@ class RPS:
                  average_gradients: bool = False, shard_begin: int = 0, shard_cols: int = 0, block_steps: int = 0,
                  kernel: int = 0, workers_per_lane: int = 0, stages: int = 0, consumer_warps: int = 0,
                  row_skew_lines: int = -1, copy_mode: int = 0, slice_bytes: int = 0, store_mode: int = 0,
-                 early_targets: int = 0,
+                 early_targets: int = 0, fuse_steps: int = 0,
                  traversal: int = 0, l2_policy: int = 0, launch_overlap: int = 0, team_warps: int = 0,
                  wait_limit_ms: int = 0, withhold_copies: bool = False,
                  device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
@@ -176,6 +176,7 @@ class RPS:
         opt.shard_begin, opt.shard_cols, opt.block_steps = shard_begin, shard_cols, block_steps
         opt.team_warps = team_warps
         opt.early_targets = early_targets
+        opt.fuse_steps = fuse_steps
         self._check(self._lib.rps_configure(self._h, ctypes.byref(opt)), "rps_configure")
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
         self.pitch = int(self._lib.rps_pitch(self._h))

@@ -106,6 +106,7 @@ struct rps_handle {
         tune.launch_overlap = opt.launch_overlap;
         tune.team_warps = opt.team_warps;
         tune.early_targets = opt.early_targets;
+        tune.fuse_steps = opt.fuse_steps;
         return tune;
     }
     rps::StepMasks* window() const { return reinterpret_cast<rps::StepMasks*>(scratch + kDiagBytes); }
@@ -336,6 +337,7 @@ int rps_default_options(rps_options* opt)
     opt->block_steps = 0;
     opt->team_warps = 0;
     opt->early_targets = 0;
+    opt->fuse_steps = 0;
     return RPS_OK;
 }
 
@@ -446,6 +448,7 @@ int rps_configure(rps_handle* h, const rps_options* opt)
         return fail(h, RPS_EINVAL, "team_warps must be 0 (auto) or 1..16");
     if (opt->early_targets < 0 || opt->early_targets > 2)
         return fail(h, RPS_EINVAL, "early_targets must be 0 (auto), 1 or 2");
+    if (opt->fuse_steps < 0 || opt->fuse_steps > 2) return fail(h, RPS_EINVAL, "fuse_steps must be 0 (auto), 1 or 2");
     h->opt = *opt;
     h->sigma = (float)opt->sigma;
     return RPS_OK;
@@ -540,6 +543,33 @@ int rps_step_n(rps_handle* h, int64_t T)
             rps::FusedParams prm = fused_params(h, masks, 0, h->cols());
             rc = timed_launch(h, 0, [&] {
                 return rps::launch_fused_blocked(prm, (int)chunk, h->opt.dtype == RPS_BF16, h->sm_count, h->stream);
+            });
+            if (rc != RPS_OK) return rc;
+            h->t += (uint64_t)chunk;
+            done += chunk;
+        }
+        return RPS_OK;
+    }
+    if (h && h->bound && h->opt.fuse_steps != 1) {
+        // as many steps per launch as the window of masks holds, where the kernel that serves this handle's steps can
+        // go from step to step inside one launch (a tracked step, or a kernel that cannot, runs singly)
+        int64_t done = 0;
+        while (done < T) {
+            int rc = need_bound(h);
+            if (rc != RPS_OK) return rc;
+            const rps::StepMasks* masks = nullptr;
+            if ((rc = masks_of_step(h, &masks)) != RPS_OK) return rc;
+            rps::FusedParams prm = fused_params(h, masks, 0, h->cols());
+            int64_t chunk = (int64_t)h->opt.mask_window - (int64_t)(h->t - h->window_t0);
+            if (chunk > T - done) chunk = T - done;
+            if (chunk < 2 || !rps::fused_steps_supported(prm, h->tuning(), h->opt.dtype == RPS_BF16, h->sm_count)) {
+                if ((rc = run_fused(h, masks)) != RPS_OK) return rc;
+                done += 1;
+                continue;
+            }
+            rc = timed_launch(h, 0, [&] {
+                return rps::launch_fused_steps(prm, h->tuning(), (int)chunk, h->opt.dtype == RPS_BF16, h->sm_count,
+                                               h->stream);
             });
             if (rc != RPS_OK) return rc;
             h->t += (uint64_t)chunk;

@@ -330,13 +330,14 @@ __device__ __forceinline__ Float2 add2(Float2 a, Float2 b)
 
 // Local SGD step of one lane on a worker pair (k even) x VEC columns from column c, from the raw slices, two
 // columns at a time: v = x + gamma (b - x) - (gamma sigma) xi.  Same bits as local_sgd_raw<T, VEC, 2, false>.
+// The step index (t_hi, t_lo) is the caller's: a launch may run several steps.
 // TARGETS: also add the pair's targets to target_sum, as (b - x) + x from the values the step holds anyway
 // (equal to b up to one rounding of the difference; for the tracked steps' mean of the targets).
 template <typename T, int VEC, bool TARGETS = false>
 __device__ __forceinline__ void local_sgd_pair_packed(const uint4 (&raw_x)[2], const uint4 (&raw_b)[2],
                                                       Float2 (&v)[2][VEC / 2], int64_t c, int k,
                                                       const FusedParams& prm, const PackedScalars& scalars,
-                                                      Float2* target_sum = nullptr)
+                                                      uint32_t t_lo, uint32_t t_hi, Float2* target_sum = nullptr)
 {
     static_assert(VEC * sizeof(T) == 16, "a slice is 16 bytes");
 #pragma unroll
@@ -366,7 +367,7 @@ __device__ __forceinline__ void local_sgd_pair_packed(const uint4 (&raw_x)[2], c
     if (!prm.noisy) return;
 #pragma unroll
     for (int q = 0; q < VEC / 4; ++q) {
-        const Philox4 r = philox4x32_keyed<kNoiseRounds>(prm.t_lo, prm.t_hi, (uint32_t)((c + prm.col_offset) >> 2) + q,
+        const Philox4 r = philox4x32_keyed<kNoiseRounds>(t_lo, t_hi, (uint32_t)((c + prm.col_offset) >> 2) + q,
                                                          kStreamNoise | ((uint32_t)(k >> 1) << 8), prm.round_key);
         // words 0,1 -> the pair's first worker (columns 0,1 and 2,3 of the four), words 2,3 -> its second
         v[0][2 * q] = add_noise_pair(v[0][2 * q], r.x, scalars);

@@ -218,18 +218,21 @@ cudaError_t launch_fused_direct(const FusedParams& prm, const FusedTuning& tune,
     return launch_direct_for_n<float, 4>(prm, tune.workers_per_lane, sm_count, stream, overlap);
 }
 
-cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
-                         cudaStream_t stream)
+namespace {
+
+enum class FusedKernel { kDirect, kStaged, kRing, kStream };
+
+// Which form of the fused step runs: the one asked for where it is built for this step, else the library's choice.
+FusedKernel choose_fused_kernel(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count)
 {
-    if (tune.kernel == 1) return launch_fused_direct(prm, tune, bf16, sm_count, stream);
-    if (tune.kernel == 3 && ring_kernel_covers(prm, bf16)) return launch_fused_ring(prm, tune, bf16, sm_count, stream);
-    if (tune.kernel == 4 && stream_kernel_covers(prm, bf16)) return launch_fused_stream(prm, tune, bf16, sm_count, stream);
+    if (tune.kernel == 1) return FusedKernel::kDirect;
+    if (tune.kernel == 3 && ring_kernel_covers(prm, bf16)) return FusedKernel::kRing;
+    if (tune.kernel == 4 && stream_kernel_covers(prm, bf16)) return FusedKernel::kStream;
     if (tune.kernel == 0) {
         // A model this short gives the staged kernel's ring less than a tile per SM: there
         // is nothing to pipeline and its set-up dominates; the step is launch bound and L2 resident.
         const int64_t bytes_per_column = (int64_t)prm.n * (bf16 ? 2 : 4);
-        if (prm.d * bytes_per_column < (int64_t)sm_count * 8192)
-            return launch_fused_direct(prm, tune, bf16, sm_count, stream);
+        if (prm.d * bytes_per_column < (int64_t)sm_count * 8192) return FusedKernel::kDirect;
     }
     // bf16 replicas of more than 32 workers: workers streamed through the teams' rings (what is staged does not
     // grow with n, every row piece is 2 KB); measured side by side 5 % ahead of the ring kernel at n = 64 and
@@ -237,13 +240,39 @@ cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool b
     // Tracked steps take it from 32 workers on (0.64 against 0.73 ms per step at n = 32, 1.19 against 1.62 at n = 64).
     if (tune.kernel == 0 && bf16 && (prm.n > 32 || (prm.trace != nullptr && prm.n >= 32)) &&
         stream_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 && tune.copy_mode == 0 && tune.slice_bytes == 0)
-        return launch_fused_stream(prm, tune, bf16, sm_count, stream);
+        return FusedKernel::kStream;
     // bf16 replicas of more than 4 workers: the self-refilling ring (16 compute warps, no producer warp), unless an
     // option that shapes the staged kernel only was set.  Measured side by side it is 3-8 % ahead at every n.
     if (tune.kernel == 0 && bf16 && ring_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 &&
         tune.consumer_warps == 0 && tune.copy_mode == 0 && tune.slice_bytes == 0)
-        return launch_fused_ring(prm, tune, bf16, sm_count, stream);
-    return launch_fused_staged(prm, tune, bf16, sm_count, stream);
+        return FusedKernel::kRing;
+    return FusedKernel::kStaged;
+}
+
+}  // namespace
+
+cudaError_t launch_fused(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
+                         cudaStream_t stream)
+{
+    switch (choose_fused_kernel(prm, tune, bf16, sm_count)) {
+        case FusedKernel::kDirect: return launch_fused_direct(prm, tune, bf16, sm_count, stream);
+        case FusedKernel::kRing: return launch_fused_ring(prm, tune, bf16, sm_count, stream);
+        case FusedKernel::kStream: return launch_fused_stream(prm, tune, bf16, sm_count, stream);
+        default: return launch_fused_staged(prm, tune, bf16, sm_count, stream);
+    }
+}
+
+bool fused_steps_supported(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count)
+{
+    // untracked steps of the streamed kernel: its teams go from step to step on their own tiles
+    return prm.trace == nullptr && choose_fused_kernel(prm, tune, bf16, sm_count) == FusedKernel::kStream;
+}
+
+cudaError_t launch_fused_steps(const FusedParams& prm, const FusedTuning& tune, int steps, bool bf16, int sm_count,
+                               cudaStream_t stream)
+{
+    if (!fused_steps_supported(prm, tune, bf16, sm_count)) return cudaErrorInvalidConfiguration;
+    return launch_fused_stream(prm, tune, bf16, sm_count, stream, steps);
 }
 
 void set_philox_key(FusedParams& prm, uint64_t seed)

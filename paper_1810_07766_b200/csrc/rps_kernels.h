@@ -116,6 +116,7 @@ struct FusedTuning {
     int32_t team_warps;        // ring kernel: warp slices per tile (1..16)
     int32_t early_targets;     // staged and streamed kernels: 1 every copy waits for the kernel ahead in the stream,
                                // 2 the copies of b for the first stages are issued before that wait
+    int32_t fuse_steps;        // rps_step_n: 1 one launch per step, 2 as many steps per launch as the kernel takes
 };
 
 struct FusedParams {
@@ -178,8 +179,14 @@ cudaError_t launch_fused_ring(const FusedParams& prm, const FusedTuning& tune, b
                               cudaStream_t stream);
 // Workers streamed through per-warp rings (rps_stream.cu): whether it is built for this step, and its launch.
 bool stream_kernel_covers(const FusedParams& prm, bool bf16);
+// `steps` consecutive steps from step (prm.t_hi, prm.t_lo) in one launch, with the mask records of those steps at
+// prm.masks[0 .. steps-1] (untracked steps; each team of warps goes from step to step on its own tiles).
 cudaError_t launch_fused_stream(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
-                                cudaStream_t stream);
+                                cudaStream_t stream, int steps = 1);
+// Whether launch_fused would run this step as a kernel that can take several steps per launch, and that launch.
+bool fused_steps_supported(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count);
+cudaError_t launch_fused_steps(const FusedParams& prm, const FusedTuning& tune, int steps, bool bf16, int sm_count,
+                               cudaStream_t stream);
 // The optional forms of the fused step, built in one family of lane shapes, each group in a
 // translation unit of its own: gradient averaging (prm.average_gradients) and tracked steps
 // (prm.trace != NULL, with either kind of averaging).

@@ -25,6 +25,10 @@
 //     slot, two IEEE operations, the same bits as the scalar forms of the other kernels.
 //   * Tracked steps (DIAG) get their sums from the same walk: every receiver holds the same value, so only
 //     the keepers have a deviation from it (see TrackCols).
+//   * One launch can run several consecutive steps (rps_step_n): a team has the same tiles in every step and a
+//     column's next step needs only that column's last step, so a team goes on to the next step by itself once
+//     its own stores are done and fenced.  There is no launch boundary between the steps and no wait for the
+//     rest of the GPU; odd steps walk the team's tiles backwards, onto what is still in L2.
 //
 // A lane whose slice straddles two blocks or the end of the row (at most n such lanes per step) takes a
 // per-column branch with the same arithmetic, so a column's result does not depend on where it lies.
@@ -45,12 +49,13 @@ constexpr int kStreamDefaultStoreMode = 1;            // 1: 16-byte stores from 
 constexpr int kStreamMaxTeamWarps = 4;                // a team's row piece is one TMA box: at most 256 8-byte units
 constexpr uint32_t kPieceBytes = 512;                 // of one row per warp: 32 lanes x 16 bytes
 // shared-memory header: a line per team (barriers, counters), the step's masks
-constexpr uint32_t kTeamLineBytes = 128;              // [8] mbarriers, then [8] int counters of warps done with a stage
+constexpr uint32_t kTeamLineBytes = 128;              // [8] mbarriers, [8] int counters of warps done with a stage, the step barrier
+constexpr uint32_t kStepBarOffset = kStreamMaxStages * (8 + 4);  // in a team's line
 constexpr uint32_t kMaskOffset = kStreamMaxWarps * kTeamLineBytes;  // up[64], down[64] u64, inv[64] f32
 constexpr uint32_t kTrackOffset = kMaskOffset + 2 * kMaxWorkers * 8 + kMaxWorkers * 4;  // tracked steps: 2 doubles, a counter
 constexpr uint32_t kStreamHeaderBytes = kTrackOffset + 256;
 static_assert(kStreamHeaderBytes % 128 == 0, "stages start on 128-byte boundaries");
-static_assert(kStreamMaxStages * (8 + 4) <= kTeamLineBytes, "a team's barriers and counters fit its line");
+static_assert(kStepBarOffset + 8 <= kTeamLineBytes && kStepBarOffset % 8 == 0, "a team's barriers and counters fit its line");
 static_assert(kStreamMaxTeamWarps * kPieceBytes / 8 <= 256, "a team's row piece is one box");
 
 struct StreamShape {
@@ -59,16 +64,13 @@ struct StreamShape {
     int32_t team_warps;       // warps per team: a tile is team_warps x 32 slices wide
     int32_t teams;            // teams per CTA
     int32_t withhold_copies;  // test aid: nothing is ever copied, so that the waits run out
-    int32_t descending;       // 1: the tiles are taken from the last to the first (odd steps)
+    int32_t steps;            // consecutive steps this launch runs, each with the mask record that follows the last one's
+    int32_t alternate;        // 1: in odd steps a team takes ITS tiles from the last to the first (FusedTuning::traversal = 0)
     int32_t bulk_stores;      // 1: the average leaves through shared memory and bulk copies (see the kernel)
     int32_t early_targets;    // 1: the first stages' copies of b are issued before the wait for the kernel ahead in the stream
     uint32_t out_offset;      // of the warps' output slots from the start of the rings
     uint64_t wait_limit_ns;
 
-    __device__ __forceinline__ int tile_of_turn(int64_t turn) const
-    {
-        return descending ? tiles - 1 - (int)turn : (int)turn;
-    }
 };
 
 // Tracked steps (distance of the averaged model to the optimum, consensus error; see Tracker in rps_device.cuh),
@@ -217,9 +219,7 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
     const int team = warp / shape.team_warps, member = warp - team * shape.team_warps;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + team * kTeamLineBytes);         // [stages] the rows have landed
     int* done = reinterpret_cast<int*>(smem + team * kTeamLineBytes + kStreamMaxStages * 8);  // [stages] warps done with them
-    uint64_t* s_up = reinterpret_cast<uint64_t*>(smem + kMaskOffset);
-    uint64_t* s_down = s_up + kMaxWorkers;
-    float* s_inv = reinterpret_cast<float*>(s_down + kMaxWorkers);
+    uint64_t* step_bar = reinterpret_cast<uint64_t*>(smem + team * kTeamLineBytes + kStepBarOffset);  // between two steps
     // tracked steps: the CTA's pair of sums and the count of warps that have added theirs
     double* track_pair = reinterpret_cast<double*>(smem + kTrackOffset);
     int* track_arrivals = reinterpret_cast<int*>(smem + kTrackOffset + 16);
@@ -237,13 +237,20 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
     const int g = (int)blockIdx.x * shape.teams + team;
     const int my_tiles = g < shape.tiles ? (shape.tiles - g + teams_total - 1) / teams_total : 0;
     const int chunks_per_tile = (n + ROWS - 1) / ROWS;
-    const uint32_t total = (uint32_t)my_tiles * (uint32_t)chunks_per_tile;  // stages' worth of rows this team goes through
+    const uint32_t total = (uint32_t)my_tiles * (uint32_t)chunks_per_tile;  // stages' worth of rows this team goes through per step
+    const uint64_t t_first = ((uint64_t)prm.t_hi << 32) | prm.t_lo;
+    auto walks_down = [&](int step) { return shape.alternate != 0 && ((t_first + (uint64_t)step) & 1u) != 0; };
+    // The team's tile number `local` of a step: the same set of tiles in every step (a team depends on nobody else's
+    // stores from one step to the next), walked upwards or downwards, so that a step starts on the tiles the step
+    // before it touched last, which are still in L2.
+    auto tile_of = [&](int local, bool down) { return g + (down ? my_tiles - 1 - local : local) * teams_total; };
 
     if (member == 0 && lane == 0) {
         for (int s = 0; s < shape.stages; ++s) {
             mbar_init(smem_addr(&full[s]), 1);
             done[s] = 0;
         }
+        mbar_init(smem_addr(step_bar), (uint32_t)shape.team_warps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x == 0) {
@@ -259,21 +266,22 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
     // free): one thread, one box per array (the replicas, the targets, or both); `expect` announces the bytes of
     // BOTH to the stage's barrier.  Boxes arrive whole (rows past n and columns past the pitch as zeros), so the
     // byte count is fixed.  The maps count columns in 8-byte units.
-    auto issue = [&](int stage, int local, int chunk, bool with_x, bool with_b, bool expect) {
+    auto issue = [&](int stage, bool down, int local, int chunk, bool with_x, bool with_b, bool expect) {
         if (shape.withhold_copies) return;
-        const int tile = shape.tile_of_turn((int64_t)g + (int64_t)local * teams_total);
+        const int tile = tile_of(local, down);
         const uint32_t bar = smem_addr(&full[stage]);
         const uint32_t dst = ring_addr + (uint32_t)stage * stage_bytes;
         if (expect) mbar_arrive_expect_tx(bar, stage_bytes);
         if (with_x) tma_load_box(dst, &map_x, tile * units_per_tile, ROWS * chunk, bar);
         if (with_b) tma_load_box(dst + array_bytes, &map_b, tile * units_per_tile, ROWS * chunk, bar);
     };
-    // the stages the ring starts with, filled by the team's first thread: stage s holds the team's chunk number s
-    auto first_fills = [&](bool with_x, bool with_b, bool expect) {
+    // the stages a step starts with, filled by the team's first thread: the ring goes on from `stage`
+    auto first_fills = [&](int stage, bool down, bool with_x, bool with_b, bool expect) {
         if (member != 0 || lane != 0) return;
         int local = 0, chunk = 0;
         for (int s = 0; s < shape.stages && (uint32_t)s < total; ++s) {
-            issue(s, local, chunk, with_x, with_b, expect);
+            issue(stage, down, local, chunk, with_x, with_b, expect);
+            if (++stage == shape.stages) stage = 0;
             if (++chunk == chunks_per_tile) chunk = 0, ++local;
         }
     };
@@ -283,23 +291,10 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
     // are not written by a step: the copies of b for the first stages go out before the wait (early_targets)
     // and arrive while that kernel drains; only the copies of x wait.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (shape.early_targets) {
-        __syncthreads();  // the barriers are initialised
-        first_fills(false, true, true);
-    }
+    __syncthreads();  // the barriers are initialised; the only CTA-wide barrier
+    if (shape.early_targets) first_fills(0, walks_down(0), false, true, true);
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    for (int j = threadIdx.x; j < kMaxWorkers; j += blockDim.x) {
-        const bool used = j < n;
-        s_up[j] = used ? prm.masks->up[j] : 0;
-        s_down[j] = used ? prm.masks->down[j] : 0;
-        s_inv[j] = used ? prm.masks->inv_cnt[j] : 0.0f;
-    }
-    __syncthreads();  // the last CTA-wide barrier
-    first_fills(true, !shape.early_targets, !shape.early_targets);
-    // where the filling stands: every warp keeps the count (the warp that frees a stage refills it)
-    int fill_local = 0, fill_chunk = 0;
-    for (int s = 0; s < shape.stages; ++s)
-        if (++fill_chunk == chunks_per_tile) fill_chunk = 0, ++fill_local;
+    first_fills(0, walks_down(0), true, !shape.early_targets, !shape.early_targets);
 
     T* __restrict__ xg = static_cast<T*>(prm.x);
     const uint64_t valid = n >= 64 ? ~(uint64_t)0 : (((uint64_t)1 << n) - 1);
@@ -308,11 +303,27 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
     unsigned char* out_slots = smem + kStreamHeaderBytes + shape.out_offset + (size_t)warp * 2 * kPieceBytes;
     const unsigned char* my_ring = ring + member * kPieceBytes + lane * 16;
     int stage = 0;
-    uint32_t phase = 0, q = 0;
+    uint32_t phase = 0;
     Tracker<VEC, 2, 1> tracker;  // this lane's sums over its tiles, and the hand-over to the CTA's pair
+    // Several steps in one launch: a team's tiles are the same in every step, and a column's next step needs
+    // only that column's last step, so a team goes from step to step on its own.  Between two steps it sees
+    // its stores done and ordered ahead of the unit's next reads (below); no other team is waited for.
+    for (int step = 0; step < shape.steps; ++step) {
+    const bool down_step = walks_down(step);
+    const uint64_t t_now = t_first + (uint64_t)step;
+    const uint32_t t_lo = (uint32_t)t_now, t_hi = (uint32_t)(t_now >> 32);
+    const StepMasks* rec = prm.masks + step;  // this step's drop masks
+    const uint64_t* s_up = rec->up;
+    const uint64_t* s_down = rec->down;
+    const float* s_inv = rec->inv_cnt;
+    // where the filling stands: every warp keeps the count (the warp that frees a stage refills it)
+    int fill_local = 0, fill_chunk = 0;
+    for (int s = 0; s < shape.stages; ++s)
+        if (++fill_chunk == chunks_per_tile) fill_chunk = 0, ++fill_local;
+    uint32_t q = 0;
     for (int local = 0; local < my_tiles; ++local) {
         // ---- a new tile: this lane's columns, the masks of their block, an empty sum
-        const int tile = shape.tile_of_turn((int64_t)g + (int64_t)local * teams_total);
+        const int tile = tile_of(local, down_step);
         const int64_t c = (int64_t)tile * team_cols + member * WARP_COLS + lane * VEC;
         T* dst = xg + c;
         const int64_t left = prm.d - c;
@@ -369,7 +380,7 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                 raw_b[0] = *reinterpret_cast<const uint4*>(src + array_bytes + (2 * half) * row_bytes);
                 raw_b[1] = *reinterpret_cast<const uint4*>(src + array_bytes + (2 * half + 1) * row_bytes);
                 Float2 v[2][VEC / 2];
-                local_sgd_pair_packed<T, VEC, DIAG>(raw_x, raw_b, v, c, k, prm, scalars, target_sum);
+                local_sgd_pair_packed<T, VEC, DIAG>(raw_x, raw_b, v, c, k, prm, scalars, t_lo, t_hi, target_sum);
                 if (regular) {
                     const uint32_t arrived = (uint32_t)(up >> k), kept = (uint32_t)(keep >> k) & 3u;
                     // RS: the running sum over the workers whose copy arrived, in worker order
@@ -440,7 +451,7 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                 }
                 if (last && q + (uint32_t)shape.stages < total) {
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // reads before the unit's writes
-                    issue(stage, fill_local, fill_chunk, true, true, true);
+                    issue(stage, down_step, fill_local, fill_chunk, true, true, true);
                 }
             }
             if (++fill_chunk == chunks_per_tile) fill_chunk = 0, ++fill_local;
@@ -510,6 +521,25 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
             }
         }
     }
+    if (step + 1 < shape.steps) {
+        // ---- between two steps.  The next step reads, through the TMA unit, what this team's warps have just
+        // stored: every lane sees its own stores done (bulk copies first, then a fence over global memory), the
+        // team meets on its barrier (bounded like every other wait), and the thread that starts the next step's
+        // copies orders them behind all that with a proxy fence.  The ring has run empty by itself (nothing
+        // is refilled past the end of a step), so the team's pipeline restarts: a few microseconds per step and
+        // team, at a different time for every team, instead of a launch boundary for the whole GPU.
+        if (shape.bulk_stores && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_addr(step_bar));
+        if (!__all_sync(0xFFFFFFFFu, stream_wait(smem_addr(step_bar), (uint32_t)step & 1u, shape.wait_limit_ns))) {
+            report_timeout(prm, 3);
+            return;
+        }
+        if (member == 0 && lane == 0) asm volatile("fence.proxy.async;" ::: "memory");
+        first_fills(stage, walks_down(step + 1), true, true, true);
+    }
+    }
     if (DIAG) tracker.flush(track_pair, track_arrivals, (int)(blockDim.x >> 5), prm.trace);
     // the bulk copies issued by this thread still read this CTA's shared memory: see them through
     if (shape.bulk_stores && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
@@ -532,8 +562,8 @@ bool encode_row_boxes(CUtensorMap* map, const void* base, size_t elem, const Fus
 }
 
 template <typename T, int VEC, int MAXW, int ROWS, bool DIAG = false>
-cudaError_t launch_stream_as(const FusedParams& prm, const FusedTuning& tune, int warps, int team_warps, int sm_count,
-                             cudaStream_t stream)
+cudaError_t launch_stream_as(const FusedParams& prm, const FusedTuning& tune, int warps, int team_warps, int steps,
+                             int sm_count, cudaStream_t stream)
 {
     auto kernel = rps_fused_stream_kernel<T, VEC, MAXW, ROWS, DIAG>;
     static LaunchState state;
@@ -559,7 +589,8 @@ cudaError_t launch_stream_as(const FusedParams& prm, const FusedTuning& tune, in
     shape.tiles = (int32_t)((prm.d + team_cols - 1) / team_cols);
     shape.wait_limit_ns = tune.wait_limit_ms > 0 ? (uint64_t)tune.wait_limit_ms * 1000000ull : kDefaultWaitLimitNs;
     shape.withhold_copies = tune.withhold_copies;
-    shape.descending = prm.descending;
+    shape.steps = steps;
+    shape.alternate = tune.traversal == 0;
     // early copies of the targets: built and bit-identical, but worth nothing here (cfg5: 1.036 ms per step with
     // them, 1.024 without, three alternating pairs on one box); the staged kernel gains 0.7 % on the smallest model
     shape.early_targets = tune.early_targets == 2;
@@ -599,7 +630,8 @@ cudaError_t launch_stream_as(const FusedParams& prm, const FusedTuning& tune, in
 }
 
 template <typename T, int VEC, int ROWS>
-cudaError_t launch_stream_for_warps(const FusedParams& prm, const FusedTuning& tune, int sm_count, cudaStream_t stream)
+cudaError_t launch_stream_for_warps(const FusedParams& prm, const FusedTuning& tune, int steps, int sm_count,
+                                    cudaStream_t stream)
 {
     // the register file is shared out by launch bound: 32 warps of 64 registers, 24 of 80, 20 of 96, 16 of 128
     // defaults from sweeps on B200 (n = 64, bf16): 5 teams of 4 warps; 16 warps leave issue slots idle, 24 and
@@ -609,10 +641,10 @@ cudaError_t launch_stream_for_warps(const FusedParams& prm, const FusedTuning& t
     int team_warps = tune.team_warps == 0 || tune.team_warps >= 4 ? 4 : (tune.team_warps >= 2 ? 2 : 1);
     while (team_warps > warps) team_warps /= 2;
     warps -= warps % team_warps;  // whole teams
-    if (warps <= 16) return launch_stream_as<T, VEC, 16, ROWS>(prm, tune, warps, team_warps, sm_count, stream);
-    if (warps <= 20) return launch_stream_as<T, VEC, 20, ROWS>(prm, tune, warps, team_warps, sm_count, stream);
-    if (warps <= 24) return launch_stream_as<T, VEC, 24, ROWS>(prm, tune, warps, team_warps, sm_count, stream);
-    return launch_stream_as<T, VEC, 32, ROWS>(prm, tune, warps, team_warps, sm_count, stream);
+    if (warps <= 16) return launch_stream_as<T, VEC, 16, ROWS>(prm, tune, warps, team_warps, steps, sm_count, stream);
+    if (warps <= 20) return launch_stream_as<T, VEC, 20, ROWS>(prm, tune, warps, team_warps, steps, sm_count, stream);
+    if (warps <= 24) return launch_stream_as<T, VEC, 24, ROWS>(prm, tune, warps, team_warps, steps, sm_count, stream);
+    return launch_stream_as<T, VEC, 32, ROWS>(prm, tune, warps, team_warps, steps, sm_count, stream);
 }
 
 // Tracked steps: stages of two worker pairs, 16 warps unless asked otherwise (the per-column sums take
@@ -625,8 +657,8 @@ cudaError_t launch_stream_tracked(const FusedParams& prm, const FusedTuning& tun
     int team_warps = tune.team_warps == 0 || tune.team_warps >= 4 ? 4 : (tune.team_warps >= 2 ? 2 : 1);
     while (team_warps > warps) team_warps /= 2;
     warps -= warps % team_warps;
-    if (warps <= 16) return launch_stream_as<T, VEC, 16, 4, true>(prm, tune, warps, team_warps, sm_count, stream);
-    return launch_stream_as<T, VEC, 20, 4, true>(prm, tune, warps, team_warps, sm_count, stream);
+    if (warps <= 16) return launch_stream_as<T, VEC, 16, 4, true>(prm, tune, warps, team_warps, 1, sm_count, stream);
+    return launch_stream_as<T, VEC, 20, 4, true>(prm, tune, warps, team_warps, 1, sm_count, stream);
 }
 
 }  // namespace
@@ -642,19 +674,21 @@ bool stream_kernel_covers(const FusedParams& prm, bool bf16)
 }
 
 cudaError_t launch_fused_stream(const FusedParams& prm, const FusedTuning& tune, bool bf16, int sm_count,
-                                cudaStream_t stream)
+                                cudaStream_t stream, int steps)
 {
-    if (!stream_kernel_covers(prm, bf16)) return cudaErrorInvalidConfiguration;
-    if (prm.trace != nullptr)
+    if (!stream_kernel_covers(prm, bf16) || steps < 1) return cudaErrorInvalidConfiguration;
+    if (prm.trace != nullptr) {
+        if (steps != 1) return cudaErrorInvalidConfiguration;  // tracked steps run one per launch
         return bf16 ? launch_stream_tracked<__nv_bfloat16, 8>(prm, tune, sm_count, stream)
                     : launch_stream_tracked<float, 4>(prm, tune, sm_count, stream);
+    }
     // rows per stage: two worker pairs, unless one pair is asked for (workers_per_lane = 2)
     const bool one_pair = tune.workers_per_lane == 2 || prm.n <= 2;
     if (bf16)
-        return one_pair ? launch_stream_for_warps<__nv_bfloat16, 8, 2>(prm, tune, sm_count, stream)
-                        : launch_stream_for_warps<__nv_bfloat16, 8, 4>(prm, tune, sm_count, stream);
-    return one_pair ? launch_stream_for_warps<float, 4, 2>(prm, tune, sm_count, stream)
-                    : launch_stream_for_warps<float, 4, 4>(prm, tune, sm_count, stream);
+        return one_pair ? launch_stream_for_warps<__nv_bfloat16, 8, 2>(prm, tune, steps, sm_count, stream)
+                        : launch_stream_for_warps<__nv_bfloat16, 8, 4>(prm, tune, steps, sm_count, stream);
+    return one_pair ? launch_stream_for_warps<float, 4, 2>(prm, tune, steps, sm_count, stream)
+                    : launch_stream_for_warps<float, 4, 4>(prm, tune, steps, sm_count, stream);
 }
 
 }  // namespace rps

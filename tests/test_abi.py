@@ -61,7 +61,7 @@ def test_options_pitch_and_state_errors(lib):
         assert opt.wait_limit_ms == 0 and opt.withhold_copies == 0 and opt.average == 0
         assert opt.traversal == 0 and opt.l2_policy == 0 and opt.launch_overlap == 0
         assert opt.shard_begin == 0 and opt.shard_cols == 0 and opt.block_steps == 0 and opt.team_warps == 0
-        assert opt.early_targets == 0
+        assert opt.early_targets == 0 and opt.fuse_steps == 0
         assert lib.rps_scratch_bytes(h) == 256 + 34 * 1792
         opt.dtype = 1
         assert lib.rps_configure(h, ctypes.byref(opt)) == 0
@@ -72,7 +72,7 @@ def test_options_pitch_and_state_errors(lib):
                              ("traversal", 2), ("l2_policy", 3), ("launch_overlap", 3),
                              ("shard_cols", -1), ("shard_begin", 64), ("shard_cols", 11_173_963),
                              ("block_steps", -1), ("block_steps", 33), ("team_warps", -1), ("team_warps", 17),
-                             ("early_targets", -1), ("early_targets", 3)):
+                             ("early_targets", -1), ("early_targets", 3), ("fuse_steps", -1), ("fuse_steps", 3)):
             bad = rps_options()
             lib.rps_default_options(ctypes.byref(bad))
             setattr(bad, field, value)

@@ -252,3 +252,46 @@ def test_targets_copied_ahead_of_the_wait_change_no_bit(rps_mod, n, d, dtype):
             r.close()
         for other in outs[1:]:
             assert (other == outs[0]).all(), kernel
+
+
+@pytest.mark.parametrize("n,d,dtype", [(64, 300_007, "bf16"), (48, 50_001, "bf16"), (5, 70_003, "f32"), (33, 20_011, "bf16"),
+                                       (64, 2_048, "bf16"), (2, 1_300, "f32")])
+def test_several_steps_in_one_launch_equal_single_steps(rps_mod, oracle, n, d, dtype):
+    """rps_step_n issues consecutive steps as one launch of the streamed kernel (fuse_steps): its teams go from step
+    to step on their own tiles.  Bit for bit the result of one launch per step, across windows of masks, across
+    t = 2^32, in shards, upwards only, with a ring longer than a step's tiles, and against the oracle's run."""
+    w = wl.Workload("fused", n=n, d=d, dtype=dtype, p=0.15, gamma=0.05, sigma=0.1, seed=21 + n, steps=11)
+    b = wl.make_targets(w)
+    x0 = start(w, 6)
+    for t0 in (0, 27, (1 << 32) - 5):
+        single = run(rps_mod, w, b, x0, w.steps, t0=t0, kernel=4, fuse_steps=1)
+        for opts in (dict(), dict(mask_window=4), dict(traversal=1), dict(stages=8, consumer_warps=8, team_warps=2),
+                     dict(store_mode=2), dict(workers_per_lane=2, consumer_warps=3, team_warps=1)):
+            ref = single if "traversal" not in opts else run(rps_mod, w, b, x0, w.steps, t0=t0, kernel=4, fuse_steps=1,
+                                                             traversal=1)
+            got = run(rps_mod, w, b, x0, w.steps, t0=t0, kernel=4, fuse_steps=2, **opts)
+            assert (got == ref).all(), (t0, opts, int((got != ref).sum()))
+    want = x0.copy()
+    oracle.run(want, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=27, steps=w.steps)
+    got = run(rps_mod, w, b, x0, w.steps, t0=27, kernel=4)
+    assert rel_err(w, got, want) <= (BF16_TOL if dtype == "bf16" else RUN_TOL)
+    # shards
+    if d > 100_000:
+        pieces = [(0, 64_000), (64_000, 36_032), (100_032, d - 100_032)]
+        parts = [run(rps_mod, w, b, x0, w.steps, t0=27, shard=piece, kernel=4) for piece in pieces]
+        assert (np.concatenate(parts, axis=1) == got).all()
+
+
+def test_fused_launches_are_counted_and_tracked_steps_stay_single(rps_mod):
+    w = wl.Workload("fused", n=64, d=65_536, dtype="bf16", p=0.1, gamma=0.05, sigma=0.1, seed=3, steps=40)
+    b = wl.make_targets(w)
+    r = rps_mod.RPS(w.n, w.d, w.p, w.gamma, w.seed, dtype="bf16", sigma=w.sigma, kernel=4)
+    r.set_targets(b)
+    before = r.launch_count()
+    r.step_n(40)  # masks of 32 steps, 32 steps in one launch; masks again, 8 steps in one launch
+    assert r.launch_count() - before == 4 and r.get_step() == 40
+    r.track(3)
+    before = r.launch_count()
+    r.step_n(5)   # three tracked steps singly, then two in one launch (no new masks: steps 40..44 of the window 32..63)
+    assert r.launch_count() - before == 4 and r.read_trace().shape == (3, 2)
+    r.close()
