@@ -41,11 +41,13 @@ FALLBACK_HBM_GBS = 6650.0
 # capture), which is the state the timed steps run in: a step starts on the columns that the step
 # before it touched last, so part of x and b is still in L2 and the traffic is below the
 # algorithmic bytes.  "cold_bytes_per_launch": one launch alone at full size with the caches flushed first
-# (also a one-pass capture; the writes of the last lines are still in L2 when the launch ends).
+# (also a one-pass capture; the writes of the last lines are still in L2 when the launch ends).  Both are bytes PER
+# STEP: cfg5's steps go out several per launch, and its figure is one launch of 32 steps divided by 32 (one step per
+# launch, --fuse-steps 1, moves the same: 6,414,904,269 B).
 NCU_TRAFFIC = {
-    "kernel_digest": "e1905f700f57feea",
-    "bytes_per_launch": {"cfg2": 963785472, "cfg3": 4806406886, "cfg4": 1432377165, "cfg5": 6413996672},
-    "cold_bytes_per_launch": {"cfg2": 1023124480, "cfg3": 4859331072, "cfg4": 1486761728, "cfg5": 6387706368},
+    "kernel_digest": "aa90357af9cdd844",
+    "bytes_per_launch": {"cfg2": 964004557, "cfg3": 4809354061, "cfg4": 1432287565, "cfg5": 6413415424},
+    "cold_bytes_per_launch": {"cfg2": 1021588480, "cfg3": 4861362176, "cfg4": 1487245824, "cfg5": 6387514624},
 }
 
 
@@ -121,7 +123,7 @@ class ClockSampler:
 
     def __init__(self, index: int, period_s: float = 0.002):
         self.index, self.period = index, period_s
-        self.samples, self.reason_bits = [], 0
+        self.samples, self.reason_bits, self.power_w = [], 0, []
         self.max_mhz = None
         self._stop = threading.Event()
         self._thread = None
@@ -154,6 +156,7 @@ class ClockSampler:
             try:
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._dev, nv.NVML_CLOCK_SM)))
                 self.reason_bits |= self._reasons() & ~0x1
+                self.power_w.append(nv.nvmlDeviceGetPowerUsage(self._dev) / 1000.0)
             except Exception:
                 pass
             time.sleep(self.period)
@@ -167,7 +170,9 @@ class ClockSampler:
     def summary(self):
         reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit]
         return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
-                "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(self.samples)}
+                "sm_min_mhz": min(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(self.samples),
+                "power_w_max": max(self.power_w) if self.power_w else None}
 
 
 # ----------------------------------------------------------------------------- multi-rank plumbing

@@ -257,7 +257,13 @@ int rps_get_step(const rps_handle* h, uint64_t* t);
  */
 int rps_step(rps_handle* h);
 
-/* T consecutive rps_step calls. */
+/*
+ * rps_step_n: T consecutive steps (the loop over t of Algorithm 1), with the results of T calls of
+ * rps_step bit for bit.  Where the kernel that serves the handle allows it (rps_options.fuse_steps),
+ * consecutive untracked steps go out as one launch per window of masks: x and b are still read once
+ * and x written once PER STEP, only the launch boundaries between the steps are gone.  (Several steps per
+ * PASS over x and b, which changes the traffic, is rps_options.block_steps.)  T < 0: RPS_EINVAL.
+ */
 int rps_step_n(rps_handle* h, int64_t T);
 
 /*
