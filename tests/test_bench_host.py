@@ -122,3 +122,32 @@ def test_bench_refuses_to_run_the_product_arm_without_a_gpu():
         return
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--steps", "1"], capture_output=True, text=True)
     assert out.returncode != 0 and "CUDA" in (out.stderr + out.stdout)
+
+
+def test_default_suite_and_kernel_names():
+    """The default run times every configuration with the largest fp32 model (d >= 11M) as the headline, and names the
+    kernel the library picks for each (the names are what the profiler's launch list shows)."""
+    sys.path.insert(0, ROOT)
+    import argparse
+
+    import bench
+    from paper_1810_07766_b200 import workloads as wl
+
+    assert bench.DEFAULT_SUITE[0] == bench.HEADLINE == "cfg3"
+    assert set(bench.DEFAULT_SUITE) == {"cfg2", "cfg3", "cfg4", "cfg5"}
+    head = wl.WORKLOADS[bench.HEADLINE]
+    assert head.dtype == "f32" and head.d >= 11_000_000
+    assert all(wl.WORKLOADS[c].n * wl.WORKLOADS[c].d <= head.n * head.d for c in bench.DEFAULT_SUITE if wl.WORKLOADS[c].dtype == "f32")
+    args = argparse.Namespace(kernel=0, average_gradients=False, track=False, workers_per_lane=0, consumer_warps=0,
+                              copy_mode=0, slice_bytes=0, d=None, sigma=None, n=None)
+    names = {c: bench.fused_kernel_name(args, wl.WORKLOADS[c]) for c in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5")}
+    assert names == {"cfg1": "rps_fused_direct_kernel", "cfg2": "rps_fused_staged_kernel", "cfg3": "rps_fused_staged_kernel",
+                     "cfg4": "rps_fused_staged_kernel", "cfg5": "rps_fused_stream_kernel"}
+    from dataclasses import replace
+    assert bench.fused_kernel_name(args, replace(wl.WORKLOADS["cfg5"], n=32)) == "rps_fused_ring_kernel"
+    args.track = True
+    assert bench.fused_kernel_name(args, replace(wl.WORKLOADS["cfg5"], n=32)) == "rps_fused_stream_kernel"
+    args.track, args.average_gradients = False, True
+    assert bench.fused_kernel_name(args, wl.WORKLOADS["cfg5"]) == "rps_fused_ring_kernel"
+    w = bench.resolve_workload(argparse.Namespace(d=1000, sigma=0.0, n=6), "cfg2", p=0.3)
+    assert (w.n, w.d, w.p, w.sigma, w.gamma, w.seed) == (6, 1000, 0.3, 0.0, 0.05, 1)
