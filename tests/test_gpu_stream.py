@@ -146,8 +146,7 @@ def test_stream_shards_reproduce_the_whole_model(rps_mod):
         assert (np.concatenate(parts, axis=1) == ref).all()
 
 
-@pytest.mark.parametrize("n,d,dtype,warps", [(8, 3_000_011, "f32", 0), (16, 2_400_003, "f32", 0),
-                                             (32, 2_000_037, "f32", 0), (64, 1_048_584, "bf16", 6),
+@pytest.mark.parametrize("n,d,dtype,warps", [(8, 3_000_011, "f32", 0), (64, 1_048_584, "bf16", 6),
                                              (64, 600_007, "bf16", 0)])
 def test_stream_laps_its_rings_many_times_every_element(rps_mod, oracle, n, d, dtype, warps):
     """Three free-running steps (up, down, up) on a model long enough that every warp takes several tiles, one
@@ -263,10 +262,11 @@ def test_several_steps_in_one_launch_equal_single_steps(rps_mod, oracle, n, d, d
     w = wl.Workload("fused", n=n, d=d, dtype=dtype, p=0.15, gamma=0.05, sigma=0.1, seed=21 + n, steps=11)
     b = wl.make_targets(w)
     x0 = start(w, 6)
+    every = (dict(), dict(mask_window=4), dict(traversal=1), dict(stages=8, consumer_warps=8, team_warps=2),
+             dict(store_mode=2), dict(workers_per_lane=2, consumer_warps=3, team_warps=1))
     for t0 in (0, 27, (1 << 32) - 5):
         single = run(rps_mod, w, b, x0, w.steps, t0=t0, kernel=4, fuse_steps=1)
-        for opts in (dict(), dict(mask_window=4), dict(traversal=1), dict(stages=8, consumer_warps=8, team_warps=2),
-                     dict(store_mode=2), dict(workers_per_lane=2, consumer_warps=3, team_warps=1)):
+        for opts in (every if t0 == 27 else every[:2]):
             ref = single if "traversal" not in opts else run(rps_mod, w, b, x0, w.steps, t0=t0, kernel=4, fuse_steps=1,
                                                              traversal=1)
             got = run(rps_mod, w, b, x0, w.steps, t0=t0, kernel=4, fuse_steps=2, **opts)
