@@ -48,12 +48,11 @@ constexpr int kStreamDefaultStages = 3;
 constexpr int kStreamDefaultStoreMode = 1;            // 1: 16-byte stores from registers; 2: bulk copies from shared memory
 constexpr int kStreamMaxTeamWarps = 4;                // a team's row piece is one TMA box: at most 256 8-byte units
 constexpr uint32_t kPieceBytes = 512;                 // of one row per warp: 32 lanes x 16 bytes
-// shared-memory header: a line per team (barriers, counters), the step's masks
+// shared-memory header: a line per team (barriers, counters), then the tracked steps' sums
 constexpr uint32_t kTeamLineBytes = 128;              // [8] mbarriers, [8] int counters of warps done with a stage, the step barrier
 constexpr uint32_t kStepBarOffset = kStreamMaxStages * (8 + 4);  // in a team's line
-constexpr uint32_t kMaskOffset = kStreamMaxWarps * kTeamLineBytes;  // up[64], down[64] u64, inv[64] f32
-constexpr uint32_t kTrackOffset = kMaskOffset + 2 * kMaxWorkers * 8 + kMaxWorkers * 4;  // tracked steps: 2 doubles, a counter
-constexpr uint32_t kStreamHeaderBytes = kTrackOffset + 256;
+constexpr uint32_t kTrackOffset = kStreamMaxWarps * kTeamLineBytes;  // tracked steps: 2 doubles, a counter
+constexpr uint32_t kStreamHeaderBytes = kTrackOffset + 128;
 static_assert(kStreamHeaderBytes % 128 == 0, "stages start on 128-byte boundaries");
 static_assert(kStepBarOffset + 8 <= kTeamLineBytes && kStepBarOffset % 8 == 0, "a team's barriers and counters fit its line");
 static_assert(kStreamMaxTeamWarps * kPieceBytes / 8 <= 256, "a team's row piece is one box");
@@ -76,13 +75,14 @@ struct StreamShape {
 // Tracked steps (distance of the averaged model to the optimum, consensus error; see Tracker in rps_device.cuh),
 // in the streamed form.  Every receiver of a block holds the same stored value P, so with P as the pivot
 // only the workers that keep their own v (down bit clear) have a deviation: per column a lane keeps
-//   bsum = sum_k b_k,  a0 = v of worker 0 (a provisional pivot, P is not known until the last worker),
+//   the sum of the targets (two columns at a time, with the step: local_sgd_pair_packed),
+//   a0 = v of worker 0 (a provisional pivot, P is not known until the last worker),
 //   D0 = sum over keepers (v_k - a0),  Q0 = sum over keepers (v_k - a0)^2        (v_k as stored),
 // and closes the column with delta = a0 - P, m keepers:  D = D0 + m delta,  Q = Q0 + 2 delta D0 + m delta^2,
 //   mean x = P + D / n,   consensus = Q - D^2 / n.   Nothing large is squared and subtracted.
 template <int VEC>
 struct TrackCols {
-    float bsum[VEC], a0[VEC], d0[VEC], q0[VEC];
+    float a0[VEC], d0[VEC], q0[VEC];
 };
 
 // One column's contribution to (|| mean x - mean b ||^2, consensus error).  `receivers` = workers that hold
@@ -106,8 +106,7 @@ __device__ __forceinline__ void close_tracked_column(float bsum, float a0, float
 template <typename T, int VEC, bool DIAG>
 __device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[2][VEC], int k, int j, int j_next,
                                             int cut, int live_n, uint64_t valid, const uint64_t* s_up,
-                                            const uint64_t* s_down, T* dst, int64_t pitch, TrackCols<VEC>* track,
-                                            const float (*b)[VEC])
+                                            const uint64_t* s_down, T* dst, int64_t pitch, TrackCols<VEC>* track)
 {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -123,7 +122,6 @@ __device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[
             const T stored = RowVec<T, VEC>::narrow(v[h][e]);
             if (kept) dst[(int64_t)w * pitch + e] = stored;
             if (DIAG && live) {
-                track->bsum[e] += b[h][e];
                 if (w == 0) track->a0[e] = v[0][e];
                 if (kept) {
                     const float dev = (float)stored - track->a0[e];
@@ -138,8 +136,8 @@ __device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[
 template <typename T, int VEC, bool DIAG>
 __device__ __noinline__ void irregular_receivers(const float (&sum)[VEC], int n, int j, int j_next, int cut,
                                                  int live_n, const uint64_t* s_down, const float* s_inv, T* dst,
-                                                 int64_t pitch, const TrackCols<VEC>* track, float inv_n, float* dist2,
-                                                 float* cons)
+                                                 int64_t pitch, const TrackCols<VEC>* track, const float (&target_sum)[VEC],
+                                                 float inv_n, float* dist2, float* cons)
 {
     T avg[VEC];
 #pragma unroll
@@ -158,7 +156,7 @@ __device__ __noinline__ void irregular_receivers(const float (&sum)[VEC], int n,
         for (int e = 0; e < VEC; ++e)
             if (e < live_n) {
                 const int receivers = __popcll(e >= cut ? down_hi : down_lo);
-                close_tracked_column(track->bsum[e], track->a0[e], track->d0[e], track->q0[e], (float)avg[e],
+                close_tracked_column(target_sum[e], track->a0[e], track->d0[e], track->q0[e], (float)avg[e],
                                      n - receivers, receivers, inv_n, dd, q);
             }
         *dist2 = dd, *cons = q;
@@ -350,7 +348,7 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
         Float2 target_sum[VEC / 2];  // tracked, regular lanes: the sum of the targets, two columns at a time
         if (DIAG) {
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) track.bsum[e] = track.a0[e] = track.d0[e] = track.q0[e] = 0.0f;
+            for (int e = 0; e < VEC; ++e) track.a0[e] = track.d0[e] = track.q0[e] = 0.0f;
 #pragma unroll
             for (int m = 0; m < VEC / 2; ++m) target_sum[m] = 0ull;
         }
@@ -423,15 +421,9 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                         unpack2(v[0][m], v_copy[0][2 * m], v_copy[0][2 * m + 1]);
                         unpack2(v[1][m], v_copy[1][2 * m], v_copy[1][2 * m + 1]);
                     }
-                    float b_copy[2][VEC];
                     TrackCols<VEC> track_copy = track;
-                    if (DIAG) {
-                        // (an irregular lane's targets are summed per column there, not in the packed sum)
-                        RowVec<T, VEC>::unpack(raw_b[0], b_copy[0]);
-                        RowVec<T, VEC>::unpack(raw_b[1], b_copy[1]);
-                    }
                     irregular_pair<T, VEC, DIAG>(sum_copy, v_copy, k, j, j_next, cut, live_n, valid, s_up, s_down, dst,
-                                                 prm.pitch, &track_copy, b_copy);
+                                                 prm.pitch, &track_copy);
                     if (DIAG) track = track_copy;
 #pragma unroll
                     for (int m = 0; m < VEC / 2; ++m) sum[m] = pack2(sum_copy[2 * m], sum_copy[2 * m + 1]);
@@ -496,14 +488,14 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                     if (rest & 1u) __stcs(reinterpret_cast<uint4*>(row), packed);
             }
             if (DIAG && live_n == VEC) {
-                float stored_avg[VEC], dd = 0.0f, qq = 0.0f;
+                float stored_avg[VEC], targets[VEC], dd = 0.0f, qq = 0.0f;
                 RowVec<T, VEC>::unpack(packed, stored_avg);
 #pragma unroll
-                for (int m = 0; m < VEC / 2; ++m) unpack2(target_sum[m], track.bsum[2 * m], track.bsum[2 * m + 1]);
+                for (int m = 0; m < VEC / 2; ++m) unpack2(target_sum[m], targets[2 * m], targets[2 * m + 1]);
                 const int receivers = __popcll(down);
 #pragma unroll
                 for (int e = 0; e < VEC; ++e)
-                    close_tracked_column(track.bsum[e], track.a0[e], track.d0[e], track.q0[e], stored_avg[e],
+                    close_tracked_column(targets[e], track.a0[e], track.d0[e], track.q0[e], stored_avg[e],
                                          n - receivers, receivers, prm.inv_n, dd, qq);
                 tracker.dist2 += (double)dd;
                 tracker.cons += (double)qq;
@@ -513,8 +505,14 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
 #pragma unroll
             for (int m = 0; m < VEC / 2; ++m) unpack2(sum[m], sum_copy[2 * m], sum_copy[2 * m + 1]);
             const TrackCols<VEC> track_copy = track;
+            float targets[VEC];  // (of the columns that exist: the others hold whatever the padding held)
+#pragma unroll
+            for (int m = 0; m < VEC / 2; ++m) {
+                if (DIAG) unpack2(target_sum[m], targets[2 * m], targets[2 * m + 1]);
+                else targets[2 * m] = targets[2 * m + 1] = 0.0f;
+            }
             irregular_receivers<T, VEC, DIAG>(sum_copy, n, j, j_next, cut, live_n, s_down, s_inv, dst, prm.pitch,
-                                              &track_copy, prm.inv_n, &dd, &qq);
+                                              &track_copy, targets, prm.inv_n, &dd, &qq);
             if (DIAG) {
                 tracker.dist2 += (double)dd;
                 tracker.cons += (double)qq;
@@ -634,8 +632,9 @@ cudaError_t launch_stream_for_warps(const FusedParams& prm, const FusedTuning& t
                                     cudaStream_t stream)
 {
     // the register file is shared out by launch bound: 32 warps of 64 registers, 24 of 80, 20 of 96, 16 of 128
-    // defaults from sweeps on B200 (n = 64, bf16): 5 teams of 4 warps; 16 warps leave issue slots idle, 24 and
-    // more lose more to the memory system than they gain
+    // defaults from sweeps on B200 (n = 64, bf16): 5 teams of 4 warps (whose rings of 16 KB stages are two stages deep:
+    // a third does not fit in shared memory, and made no difference where it did); 16 warps leave issue slots idle,
+    // 24 and more lose more to the memory system than they gain
     int warps = tune.consumer_warps > 0 ? tune.consumer_warps : 20;
     if (warps > kStreamMaxWarps) warps = kStreamMaxWarps;
     int team_warps = tune.team_warps == 0 || tune.team_warps >= 4 ? 4 : (tune.team_warps >= 2 ? 2 : 1);
