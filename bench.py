@@ -89,9 +89,9 @@ def fused_kernel_name(args, w) -> str:
     small = w.n * w.d * w.elem_bytes < 148 * 8192
     if args.kernel == 1 or (args.kernel == 0 and small):
         return "rps_fused_direct_kernel"
-    stream_built = w.n >= 2 and not args.average_gradients
+    stream_built = w.n >= 2 and not (args.average_gradients and args.track)
     staged_only = args.workers_per_lane or args.copy_mode or args.slice_bytes
-    wide = w.n > 32 or (args.track and w.n >= 32)
+    wide = 32 < w.n <= 60 if args.average_gradients else w.n > 32 or (args.track and w.n >= 32)
     if stream_built and (args.kernel == 4 or (args.kernel == 0 and w.dtype == "bf16" and wide and not staged_only)):
         return "rps_fused_stream_kernel"
     ring_built = w.dtype == "bf16" and w.n > 4 and not args.track

@@ -97,21 +97,24 @@ typedef struct rps_options {
                                  3: the same staging with no producer warp: all 16 warps of a
                                  CTA compute, each taking the next slice of the next tile from a
                                  counter, and the last warp to have read a stage refills it (built for bf16 replicas
-                                 with more than 4 workers, plain untracked model averaging;
-                                 any other step runs as kernel 2);
+                                 with more than 4 workers, untracked steps; any other step runs
+                                 as kernel 2);
                                  4: workers streamed: a lane owns one 16-byte slice of columns and
                                  walks all n workers in order, two at a time, adding each v to the
                                  running sum and storing it at once where the return message is
                                  lost; the average is rounded once and stored to every receiver.
                                  Teams of warps share shared-memory rings of a few rows that they
                                  refill themselves; a team reads whole 2 KB pieces of rows and a warp
-                                 writes whole 512-byte pieces (model averaging, tracked or not,
-                                 n >= 2, blocks of at least 16 bytes; any other step runs as
-                                 kernel 2 or 3).
+                                 writes whole 512-byte pieces.  Gradient averaging sums the
+                                 updates instead and reads a tile's rows of x a second time for
+                                 the receivers (n >= 2, blocks of at least 16 bytes, tracked
+                                 steps in model averaging only; any other step runs as kernel
+                                 2 or 3).
                                  0: kernel 1 for models too short to give every SM a tile, kernel 4
-                                 for bf16 replicas of more than 32 workers, kernel 3 for bf16
-                                 replicas of more than 4 workers (unless an option that shapes
-                                 kernel 2 alone is set), else kernel 2                        */
+                                 for bf16 replicas of more than 32 workers (gradient averaging:
+                                 33 to 60), kernel 3 for bf16 replicas of more than 4 workers
+                                 (unless an option that shapes kernel 2 alone is set), else
+                                 kernel 2                                                     */
     int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */
     int32_t stages;           /* depth of the shared-memory ring(s) of kernels 2, 3 and 4 (2..8) */
     int32_t consumer_warps;   /* compute warps per CTA of kernel 2 (1..24; shapes that need

@@ -333,7 +333,8 @@ __device__ __forceinline__ Float2 add2(Float2 a, Float2 b)
 // The step index (t_hi, t_lo) is the caller's: a launch may run several steps.
 // TARGETS: also add the pair's targets to target_sum, as (b - x) + x from the values the step holds anyway
 // (equal to b up to one rounding of the difference; for the tracked steps' mean of the targets).
-template <typename T, int VEC, bool TARGETS = false>
+// UPDATE: leave the update v - x = gamma (b - x) - (gamma sigma) xi in v instead (gradient averaging).
+template <typename T, int VEC, bool TARGETS = false, bool UPDATE = false>
 __device__ __forceinline__ void local_sgd_pair_packed(const uint4 (&raw_x)[2], const uint4 (&raw_b)[2],
                                                       Float2 (&v)[2][VEC / 2], int64_t c, int k,
                                                       const FusedParams& prm, const PackedScalars& scalars,
@@ -349,7 +350,7 @@ __device__ __forceinline__ void local_sgd_pair_packed(const uint4 (&raw_x)[2], c
             for (int m = 0; m < 2; ++m) {
                 const Float2 x2 = pack2(wx[2 * m], wx[2 * m + 1]);
                 const Float2 b2 = pack2(wb[2 * m], wb[2 * m + 1]);
-                v[h][m % (VEC / 2)] = fma2(scalars.gamma, sub2(b2, x2), x2);
+                v[h][m % (VEC / 2)] = UPDATE ? mul2(scalars.gamma, sub2(b2, x2)) : fma2(scalars.gamma, sub2(b2, x2), x2);
                 if (TARGETS) target_sum[m % (VEC / 2)] = add2(target_sum[m % (VEC / 2)], b2);
             }
         } else {
@@ -359,7 +360,7 @@ __device__ __forceinline__ void local_sgd_pair_packed(const uint4 (&raw_x)[2], c
                 float d_lo, d_hi;
                 bf16_pair_minus(wb[m], x_lo, x_hi, d_lo, d_hi);
                 const Float2 d2 = pack2(d_lo, d_hi), x2 = pack2(x_lo, x_hi);
-                v[h][m % (VEC / 2)] = fma2(scalars.gamma, d2, x2);
+                v[h][m % (VEC / 2)] = UPDATE ? mul2(scalars.gamma, d2) : fma2(scalars.gamma, d2, x2);
                 if (TARGETS) target_sum[m % (VEC / 2)] = add2(target_sum[m % (VEC / 2)], add2(d2, x2));
             }
         }

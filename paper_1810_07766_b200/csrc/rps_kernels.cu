@@ -238,8 +238,13 @@ FusedKernel choose_fused_kernel(const FusedParams& prm, const FusedTuning& tune,
     // grow with n, every row piece is 2 KB); measured side by side 5 % ahead of the ring kernel at n = 64 and
     // a third at n = 48, level with it or behind at n <= 32.
     // Tracked steps take it from 32 workers on (0.64 against 0.73 ms per step at n = 32, 1.19 against 1.62 at n = 64).
-    if (tune.kernel == 0 && bf16 && (prm.n > 32 || (prm.trace != nullptr && prm.n >= 32)) &&
-        stream_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 && tune.copy_mode == 0 && tune.slice_bytes == 0)
+    // Gradient averaging reads x twice in this form, a third of it from DRAM again at n = 64 (1.25 ms per step against
+    // 1.18 for the ring kernel, which holds the tile); the ring kernel's lane groups of 8 workers are full only at
+    // n = 64, though: at n = 48 the streamed form is ahead (0.98 against 1.12 ms), so it takes 33..60 workers.
+    const bool many_workers = prm.average_gradients ? (prm.n > 32 && prm.n <= 60)
+                                                    : (prm.n > 32 || (prm.trace != nullptr && prm.n >= 32));
+    if (tune.kernel == 0 && bf16 && many_workers && stream_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 &&
+        tune.copy_mode == 0 && tune.slice_bytes == 0)
         return FusedKernel::kStream;
     // bf16 replicas of more than 4 workers: the self-refilling ring (16 compute warps, no producer warp), unless an
     // option that shapes the staged kernel only was set.  Measured side by side it is 3-8 % ahead at every n.

@@ -30,6 +30,10 @@
 //     its own stores are done and fenced.  There is no launch boundary between the steps and no wait for the
 //     rest of the GPU; odd steps walk the team's tiles backwards, onto what is still in L2.
 //
+//   * Gradient averaging (GRAD) sums the updates v - x instead, and a receiver's new value x + (average update)
+//     needs its own x after the last worker: the tile's rows of x go through the ring a second time, last rows
+//     first (what was read last is still in L2), and each receiver's row is finished then.  Keepers are stored in the first pass as always.
+//
 // A lane whose slice straddles two blocks or the end of the row (at most n such lanes per step) takes a
 // per-column branch with the same arithmetic, so a column's result does not depend on where it lies.
 //
@@ -103,10 +107,13 @@ __device__ __forceinline__ void close_tracked_column(float bsum, float a0, float
 // columns [0, cut) of the slice belong to block j, columns [cut, VEC) to block j + 1, columns from live_n on
 // do not exist.  Same arithmetic as the regular path (predicated add in worker order, one multiplication).
 // Out of line and on copies of the caller's registers: this is rare.
+// `v` is what the sum takes and `own` what a keeper stores: the same values in model averaging, the update and
+// x + the update in gradient averaging.
 template <typename T, int VEC, bool DIAG>
-__device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[2][VEC], int k, int j, int j_next,
-                                            int cut, int live_n, uint64_t valid, const uint64_t* s_up,
-                                            const uint64_t* s_down, T* dst, int64_t pitch, TrackCols<VEC>* track)
+__device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[2][VEC], const float (&own)[2][VEC],
+                                            int k, int j, int j_next, int cut, int live_n, uint64_t valid,
+                                            const uint64_t* s_up, const uint64_t* s_down, T* dst, int64_t pitch,
+                                            TrackCols<VEC>* track)
 {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -119,10 +126,10 @@ __device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[
             const bool live = e < live_n, hi = e >= cut;
             add_if(sum[e], v[h][e], live ? (hi ? up_hi : up_lo) : 0u);
             const bool kept = live && (hi ? keep_hi : keep_lo);
-            const T stored = RowVec<T, VEC>::narrow(v[h][e]);
+            const T stored = RowVec<T, VEC>::narrow(own[h][e]);
             if (kept) dst[(int64_t)w * pitch + e] = stored;
             if (DIAG && live) {
-                if (w == 0) track->a0[e] = v[0][e];
+                if (w == 0) track->a0[e] = own[0][e];
                 if (kept) {
                     const float dev = (float)stored - track->a0[e];
                     track->d0[e] += dev;
@@ -187,6 +194,34 @@ __device__ __forceinline__ uint4 pack_pairs(const Float2 (&v)[VEC / 2])
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// 16 bytes of a row as VEC / 2 column pairs in fp32.
+template <typename T, int VEC>
+__device__ __forceinline__ void unpack_pairs(const uint4 raw, Float2 (&x)[VEC / 2])
+{
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+    if (sizeof(T) == 4) {
+#pragma unroll
+        for (int m = 0; m < 2; ++m) x[m % (VEC / 2)] = pack2(w[2 * m], w[2 * m + 1]);
+    } else {
+#pragma unroll
+        for (int m = 0; m < 4; ++m) x[m % (VEC / 2)] = pack2(w[m] << 16, w[m] & 0xFFFF0000u);
+    }
+}
+
+// Gradient averaging, second pass, a lane whose slice is cut by a block boundary or the end of the row: worker w
+// takes x + (average update) in the columns whose block's average reached it.
+template <typename T, int VEC>
+__device__ __noinline__ void irregular_update_row(const uint4 raw_x, const float (&avg)[VEC], int w, int j, int j_next,
+                                                  int cut, int live_n, const uint64_t* s_down, T* row)
+{
+    float x[VEC];
+    RowVec<T, VEC>::unpack(raw_x, x);
+    const bool lo = (s_down[j] >> w) & 1u, hi = (s_down[j_next] >> w) & 1u;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e)
+        if (e < live_n && (e >= cut ? hi : lo)) row[e] = RowVec<T, VEC>::narrow(x[e] + avg[e]);
+}
+
 // Waits for the phase with the given parity: one cheap test first (the data has usually landed long ago), then
 // the bounded wait.
 __device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns)
@@ -203,13 +238,14 @@ __device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity, uint6
     return mbar_wait(bar, parity, limit_ns);
 }
 
-template <typename T, int VEC, int MAXW, int ROWS, bool DIAG>
+template <typename T, int VEC, int MAXW, int ROWS, bool DIAG, bool GRAD>
 __global__ void __launch_bounds__(MAXW * 32, 1)
     rps_fused_stream_kernel(const __grid_constant__ FusedParams prm, const StreamShape shape,
                             const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_b)
 {
     constexpr int WARP_COLS = 32 * VEC;
     static_assert(ROWS == 2 || ROWS == 4, "a stage holds one or two worker pairs");
+    static_assert(!(DIAG && GRAD), "tracked steps are model averaging");
     extern __shared__ __align__(128) unsigned char smem[];
     const int n = prm.n;
     const int lane = threadIdx.x & 31;
@@ -234,7 +270,10 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
     const int teams_total = (int)gridDim.x * shape.teams;
     const int g = (int)blockIdx.x * shape.teams + team;
     const int my_tiles = g < shape.tiles ? (shape.tiles - g + teams_total - 1) / teams_total : 0;
-    const int chunks_per_tile = (n + ROWS - 1) / ROWS;
+    // Gradient averaging goes through a tile's rows twice: a receiver's new value x + (average update) needs its
+    // own x once all workers have been seen, so the rows of x come round again (from L2, mostly) in a second pass.
+    const int pass_chunks = (n + ROWS - 1) / ROWS;
+    const int chunks_per_tile = GRAD ? 2 * pass_chunks : pass_chunks;
     const uint32_t total = (uint32_t)my_tiles * (uint32_t)chunks_per_tile;  // stages' worth of rows this team goes through per step
     const uint64_t t_first = ((uint64_t)prm.t_hi << 32) | prm.t_lo;
     auto walks_down = [&](int step) { return shape.alternate != 0 && ((t_first + (uint64_t)step) & 1u) != 0; };
@@ -269,9 +308,17 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
         const int tile = tile_of(local, down);
         const uint32_t bar = smem_addr(&full[stage]);
         const uint32_t dst = ring_addr + (uint32_t)stage * stage_bytes;
-        if (expect) mbar_arrive_expect_tx(bar, stage_bytes);
-        if (with_x) tma_load_box(dst, &map_x, tile * units_per_tile, ROWS * chunk, bar);
-        if (with_b) tma_load_box(dst + array_bytes, &map_b, tile * units_per_tile, ROWS * chunk, bar);
+        // The second pass of gradient averaging takes the replicas only, from the last rows to the first: what the
+        // first pass read last is read again first, while it is still in L2.  The targets of that form are loaded
+        // with the evict-first hint, so that they do not push the replicas out meanwhile.
+        const bool again = GRAD && chunk >= pass_chunks;
+        const int first_row = ROWS * (again ? 2 * pass_chunks - 1 - chunk : chunk);
+        if (expect) mbar_arrive_expect_tx(bar, again ? array_bytes : stage_bytes);
+        if (with_x) tma_load_box(dst, &map_x, tile * units_per_tile, first_row, bar);
+        if (with_b && !again) {
+            if (GRAD) tma_load_box(dst + array_bytes, &map_b, tile * units_per_tile, first_row, bar, l2_evict_first_policy());
+            else tma_load_box(dst + array_bytes, &map_b, tile * units_per_tile, first_row, bar);
+        }
     };
     // the stages a step starts with, filled by the team's first thread: the ring goes on from `stage`
     auto first_fills = [&](int stage, bool down, bool with_x, bool with_b, bool expect) {
@@ -319,6 +366,43 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
     for (int s = 0; s < shape.stages; ++s)
         if (++fill_chunk == chunks_per_tile) fill_chunk = 0, ++fill_local;
     uint32_t q = 0;
+    // Waits (bounded) for the ring's current stage to have landed.
+    auto await_stage = [&]() -> bool {
+        if (__all_sync(0xFFFFFFFFu, stream_wait(smem_addr(&full[stage]), phase, shape.wait_limit_ns))) return true;
+        // Something this warp waited for never came: say so, and see the copies that may have been issued
+        // into the team's ring land (bounded) before this warp's part of the shared memory is given up.
+        report_timeout(prm, 2);
+        if (!shape.withhold_copies && lane == 0) {
+            for (int s = 1; s < shape.stages && q + (uint32_t)s < total; ++s) {
+                if (++stage == shape.stages) stage = 0, phase ^= 1u;
+                if (!mbar_wait(smem_addr(&full[stage]), phase, shape.wait_limit_ns)) break;
+            }
+        }
+        if (shape.bulk_stores && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        return false;
+    };
+    // This warp is done with the stage (its values have been used, so its reads have completed).  The last
+    // warp of the team to say so refills the stage with the rows that come `stages` stages later.
+    auto release_stage = [&]() {
+        __syncwarp();
+        if (lane == 0) {
+            bool last = true;
+            if (shape.team_warps > 1) {
+                uint32_t before;
+                asm volatile("atom.relaxed.cta.shared::cta.add.u32 %0, [%1], 1;"
+                             : "=r"(before) : "r"(smem_addr(&done[stage])) : "memory");
+                last = before == (uint32_t)shape.team_warps - 1u;
+                if (last) done[stage] = 0;  // seen by the stage's next readers through the barrier the refill completes
+            }
+            if (last && q + (uint32_t)shape.stages < total) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // reads before the unit's writes
+                issue(stage, down_step, fill_local, fill_chunk, true, true, true);
+            }
+        }
+        if (++fill_chunk == chunks_per_tile) fill_chunk = 0, ++fill_local;
+        if (++stage == shape.stages) stage = 0, phase ^= 1u;
+        ++q;
+    };
     for (int local = 0; local < my_tiles; ++local) {
         // ---- a new tile: this lane's columns, the masks of their block, an empty sum
         const int tile = tile_of(local, down_step);
@@ -353,20 +437,8 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
             for (int m = 0; m < VEC / 2; ++m) target_sum[m] = 0ull;
         }
 
-        for (int chunk = 0; chunk < chunks_per_tile; ++chunk, ++q) {
-            if (!__all_sync(0xFFFFFFFFu, stream_wait(smem_addr(&full[stage]), phase, shape.wait_limit_ns))) {
-                // Something this warp waited for never came: say so, and see the copies that may have been issued
-                // into the team's ring land (bounded) before this warp's part of the shared memory is given up.
-                report_timeout(prm, 2);
-                if (!shape.withhold_copies && lane == 0) {
-                    for (int s = 1; s < shape.stages && q + (uint32_t)s < total; ++s) {
-                        if (++stage == shape.stages) stage = 0, phase ^= 1u;
-                        if (!mbar_wait(smem_addr(&full[stage]), phase, shape.wait_limit_ns)) break;
-                    }
-                }
-                if (shape.bulk_stores && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-                return;
-            }
+        for (int chunk = 0; chunk < pass_chunks; ++chunk) {
+            if (!await_stage()) return;
             const unsigned char* src = my_ring + (size_t)stage * stage_bytes;
 #pragma unroll
             for (int half = 0; half < ROWS / 2; ++half) {
@@ -378,7 +450,7 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                 raw_b[0] = *reinterpret_cast<const uint4*>(src + array_bytes + (2 * half) * row_bytes);
                 raw_b[1] = *reinterpret_cast<const uint4*>(src + array_bytes + (2 * half + 1) * row_bytes);
                 Float2 v[2][VEC / 2];
-                local_sgd_pair_packed<T, VEC, DIAG>(raw_x, raw_b, v, c, k, prm, scalars, t_lo, t_hi, target_sum);
+                local_sgd_pair_packed<T, VEC, DIAG, GRAD>(raw_x, raw_b, v, c, k, prm, scalars, t_lo, t_hi, target_sum);
                 if (regular) {
                     const uint32_t arrived = (uint32_t)(up >> k), kept = (uint32_t)(keep >> k) & 3u;
                     // RS: the running sum over the workers whose copy arrived, in worker order
@@ -399,6 +471,12 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             if (!((kept >> h) & 1u)) continue;
+                            if (GRAD) {  // v holds the update: the worker keeps x + its own
+                                Float2 x2[VEC / 2];
+                                unpack_pairs<T, VEC>(raw_x[h], x2);
+#pragma unroll
+                                for (int m = 0; m < VEC / 2; ++m) v[h][m] = add2(x2[m], v[h][m]);
+                            }
                             const uint4 packed_v = pack_pairs<T, VEC>(v[h]);
                             __stcs(reinterpret_cast<uint4*>(dst + (int64_t)(k + h) * prm.pitch), packed_v);
                             if (DIAG) {
@@ -422,34 +500,71 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                         unpack2(v[1][m], v_copy[1][2 * m], v_copy[1][2 * m + 1]);
                     }
                     TrackCols<VEC> track_copy = track;
-                    irregular_pair<T, VEC, DIAG>(sum_copy, v_copy, k, j, j_next, cut, live_n, valid, s_up, s_down, dst,
-                                                 prm.pitch, &track_copy);
+                    if (GRAD) {
+                        float own_copy[2][VEC];
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            RowVec<T, VEC>::unpack(raw_x[h], own_copy[h]);
+#pragma unroll
+                            for (int e = 0; e < VEC; ++e) own_copy[h][e] += v_copy[h][e];
+                        }
+                        irregular_pair<T, VEC, DIAG>(sum_copy, v_copy, own_copy, k, j, j_next, cut, live_n, valid, s_up,
+                                                     s_down, dst, prm.pitch, &track_copy);
+                    } else {
+                        irregular_pair<T, VEC, DIAG>(sum_copy, v_copy, v_copy, k, j, j_next, cut, live_n, valid, s_up,
+                                                     s_down, dst, prm.pitch, &track_copy);
+                    }
                     if (DIAG) track = track_copy;
 #pragma unroll
                     for (int m = 0; m < VEC / 2; ++m) sum[m] = pack2(sum_copy[2 * m], sum_copy[2 * m + 1]);
                 }
             }
-            // This warp is done with the stage (its values have been used, so its reads have completed).  The
-            // last warp of the team to say so refills the stage with the rows that come `stages` stages later.
-            __syncwarp();
-            if (lane == 0) {
-                bool last = true;
-                if (shape.team_warps > 1) {
-                    uint32_t before;
-                    asm volatile("atom.relaxed.cta.shared::cta.add.u32 %0, [%1], 1;"
-                                 : "=r"(before) : "r"(smem_addr(&done[stage])) : "memory");
-                    last = before == (uint32_t)shape.team_warps - 1u;
-                    if (last) done[stage] = 0;  // seen by the stage's next readers through the barrier the refill completes
-                }
-                if (last && q + (uint32_t)shape.stages < total) {
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // reads before the unit's writes
-                    issue(stage, down_step, fill_local, fill_chunk, true, true, true);
-                }
-            }
-            if (++fill_chunk == chunks_per_tile) fill_chunk = 0, ++fill_local;
-            if (++stage == shape.stages) stage = 0, phase ^= 1u;
+            release_stage();
         }
 
+        if (GRAD) {
+            // ---- AG of gradient averaging: the average UPDATE of the lane's columns, then the rows of x once
+            // more: worker k takes x_k + that average where the return message arrived.
+            Float2 avg[VEC / 2];
+            if (regular) {
+                const Float2 inv2 = pack2(inv, inv);
+#pragma unroll
+                for (int m = 0; m < VEC / 2; ++m) avg[m] = mul2(sum[m], inv2);
+            } else {
+                const float inv_next = s_inv[j_next];
+#pragma unroll
+                for (int m = 0; m < VEC / 2; ++m) {
+                    float lo, hi;
+                    unpack2(sum[m], lo, hi);
+                    avg[m] = pack2(lo * (2 * m >= cut ? inv_next : inv), hi * (2 * m + 1 >= cut ? inv_next : inv));
+                }
+            }
+            for (int chunk = 0; chunk < pass_chunks; ++chunk) {
+                if (!await_stage()) return;
+                const unsigned char* src = my_ring + (size_t)stage * stage_bytes;
+#pragma unroll
+                for (int r = 0; r < ROWS; ++r) {
+                    const int k = ROWS * (pass_chunks - 1 - chunk) + r;  // the rows come back last chunk first
+                    if (k >= n) break;
+                    if (regular) {
+                        if (!((down >> k) & 1u)) continue;
+                        Float2 x2[VEC / 2];
+                        unpack_pairs<T, VEC>(*reinterpret_cast<const uint4*>(src + r * row_bytes), x2);
+#pragma unroll
+                        for (int m = 0; m < VEC / 2; ++m) x2[m] = add2(x2[m], avg[m]);
+                        __stcs(reinterpret_cast<uint4*>(dst + (int64_t)k * prm.pitch), pack_pairs<T, VEC>(x2));
+                    } else {
+                        float avg_copy[VEC];
+#pragma unroll
+                        for (int m = 0; m < VEC / 2; ++m) unpack2(avg[m], avg_copy[2 * m], avg_copy[2 * m + 1]);
+                        irregular_update_row<T, VEC>(*reinterpret_cast<const uint4*>(src + r * row_bytes), avg_copy, k, j,
+                                                     j_next, cut, live_n, s_down, dst + (int64_t)k * prm.pitch);
+                    }
+                }
+                release_stage();
+            }
+            continue;
+        }
         // ---- AG, the receivers: one average, rounded and packed once, to every row whose down bit is set
         if (regular) {
             const Float2 inv2 = pack2(inv, inv);
@@ -559,11 +674,11 @@ bool encode_row_boxes(CUtensorMap* map, const void* base, size_t elem, const Fus
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <typename T, int VEC, int MAXW, int ROWS, bool DIAG = false>
+template <typename T, int VEC, int MAXW, int ROWS, bool DIAG = false, bool GRAD = false>
 cudaError_t launch_stream_as(const FusedParams& prm, const FusedTuning& tune, int warps, int team_warps, int steps,
                              int sm_count, cudaStream_t stream)
 {
-    auto kernel = rps_fused_stream_kernel<T, VEC, MAXW, ROWS, DIAG>;
+    auto kernel = rps_fused_stream_kernel<T, VEC, MAXW, ROWS, DIAG, GRAD>;
     static LaunchState state;
     size_t smem_limit = 0;
     cudaError_t err = smem_limit_of_device(state, &smem_limit);
@@ -574,7 +689,7 @@ cudaError_t launch_stream_as(const FusedParams& prm, const FusedTuning& tune, in
     shape.teams = warps / team_warps;
     shape.stages = tune.stages > 0 ? tune.stages : kStreamDefaultStages;
     if (shape.stages > kStreamMaxStages) shape.stages = kStreamMaxStages;
-    shape.bulk_stores = (tune.store_mode != 0 ? tune.store_mode : kStreamDefaultStoreMode) == 2;
+    shape.bulk_stores = !GRAD && (tune.store_mode != 0 ? tune.store_mode : kStreamDefaultStoreMode) == 2;
     // the rings, then (bulk stores) two 512-byte output slots per warp
     auto ring_bytes = [&] {
         return (size_t)shape.teams * team_warps * (shape.stages * (2 * ROWS * kPieceBytes) + (shape.bulk_stores ? 2 * kPieceBytes : 0));
@@ -660,15 +775,28 @@ cudaError_t launch_stream_tracked(const FusedParams& prm, const FusedTuning& tun
     return launch_stream_as<T, VEC, 20, 4, true>(prm, tune, warps, team_warps, 1, sm_count, stream);
 }
 
+// Gradient averaging: stages of two worker pairs, 16 or 20 warps.
+template <typename T, int VEC>
+cudaError_t launch_stream_gradients(const FusedParams& prm, const FusedTuning& tune, int steps, int sm_count,
+                                    cudaStream_t stream)
+{
+    int warps = tune.consumer_warps > 0 ? tune.consumer_warps : 20;
+    if (warps > 20) warps = 20;
+    int team_warps = tune.team_warps == 0 || tune.team_warps >= 4 ? 4 : (tune.team_warps >= 2 ? 2 : 1);
+    while (team_warps > warps) team_warps /= 2;
+    warps -= warps % team_warps;
+    if (warps <= 16)
+        return launch_stream_as<T, VEC, 16, 4, false, true>(prm, tune, warps, team_warps, steps, sm_count, stream);
+    return launch_stream_as<T, VEC, 20, 4, false, true>(prm, tune, warps, team_warps, steps, sm_count, stream);
+}
+
 }  // namespace
 
 bool stream_kernel_covers(const FusedParams& prm, bool bf16)
 {
-    // model averaging (tracked or not), at least one worker pair, blocks at least as wide as a lane's slice
-    // (a slice then meets at most two blocks); TMA coordinates are 32-bit.  Not gradient averaging: a receiver's
-    // new value x + (average update) needs its own x after all workers have been seen, which this form has
-    // let go of by then.
-    return prm.n >= 2 && !prm.average_gradients && prm.block_cols >= (bf16 ? 8 : 4) &&
+    // at least one worker pair, blocks at least as wide as a lane's slice (a slice then meets at most two
+    // blocks); TMA coordinates are 32-bit.  Tracked steps are model averaging.
+    return prm.n >= 2 && !(prm.average_gradients && prm.trace != nullptr) && prm.block_cols >= (bf16 ? 8 : 4) &&
            prm.pitch < ((int64_t)1 << 31);
 }
 
@@ -681,6 +809,9 @@ cudaError_t launch_fused_stream(const FusedParams& prm, const FusedTuning& tune,
         return bf16 ? launch_stream_tracked<__nv_bfloat16, 8>(prm, tune, sm_count, stream)
                     : launch_stream_tracked<float, 4>(prm, tune, sm_count, stream);
     }
+    if (prm.average_gradients)
+        return bf16 ? launch_stream_gradients<__nv_bfloat16, 8>(prm, tune, steps, sm_count, stream)
+                    : launch_stream_gradients<float, 4>(prm, tune, steps, sm_count, stream);
     // rows per stage: two worker pairs, unless one pair is asked for (workers_per_lane = 2)
     const bool one_pair = tune.workers_per_lane == 2 || prm.n <= 2;
     if (bf16)

@@ -161,16 +161,48 @@ def test_stream_laps_its_rings_many_times_every_element(rps_mod, oracle, n, d, d
 
 
 def test_steps_the_stream_kernel_is_not_built_for_still_run(rps_mod, oracle):
-    """One worker, gradient averaging: asking for kernel 4 must still give the right step."""
-    for n, dtype, extra in ((1, "f32", {}), (16, "bf16", dict(average_gradients=True))):
-        w = wl.Workload("stream", n=n, d=30_011, dtype=dtype, p=0.2, gamma=0.1, sigma=0.1, seed=5, steps=3)
+    """One worker, blocks narrower than a lane's slice: asking for kernel 4 must still give the right step."""
+    for n, d, dtype in ((1, 30_011, "f32"), (16, 100, "bf16")):
+        w = wl.Workload("stream", n=n, d=d, dtype=dtype, p=0.2, gamma=0.1, sigma=0.1, seed=5, steps=3)
         b = wl.make_targets(w)
         x0 = wl.make_initial(w)
         want = x0.copy()
-        oracle.run(want, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps,
-                   average_gradients=bool(extra))
-        got = run(rps_mod, w, b, x0, w.steps, kernel=4, strict_padding=False, **extra)
+        oracle.run(want, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=0, steps=w.steps)
+        got = run(rps_mod, w, b, x0, w.steps, kernel=4, strict_padding=False)
         assert rel_err(w, got, want) <= (BF16_TOL if dtype == "bf16" else RUN_TOL)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("n,d", [(2, 50_001), (3, 4097), (5, 70_003), (8, 262_144), (17, 40_970), (33, 20_011),
+                                 (48, 50_001), (64, 300_007), (64, 7), (7, 255)])
+def test_stream_gradient_averaging_matches_the_oracle(rps_mod, oracle, dtype, n, d):
+    """Section 5's comparison method in the streamed form (the updates are summed, and a tile's rows of x go through
+    the ring a second time for the receivers): against the oracle's run, and bit for bit across warps, teams, ring
+    depths, traversal, launch mode and steps per launch; the padding stays untouched."""
+    w = wl.Workload("stream", n=n, d=d, dtype=dtype, p=0.2, gamma=0.05, sigma=0.1, seed=700 + n, steps=7, hetero=True)
+    b = wl.make_targets(w)
+    x0 = start(w, n * 5 + 2)
+    want = x0.copy()
+    oracle.run(want, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=3, steps=w.steps,
+               average_gradients=True)
+    covered = -(-d // n) >= (8 if dtype == "bf16" else 4)
+    ref = run(rps_mod, w, b, x0, w.steps, t0=3, kernel=4, average_gradients=True, strict_padding=covered)
+    assert rel_err(w, ref, want) <= (BF16_TOL if dtype == "bf16" else RUN_TOL)
+    if not covered:
+        return
+    for opts in (dict(consumer_warps=1, team_warps=1, stages=2), dict(consumer_warps=16, stages=3, traversal=1),
+                 dict(team_warps=2, consumer_warps=6, stages=5, launch_overlap=1), dict(fuse_steps=1),
+                 dict(fuse_steps=2, mask_window=3), dict(early_targets=2, stages=8)):
+        base = ref if "traversal" not in opts else run(rps_mod, w, b, x0, w.steps, t0=3, kernel=4,
+                                                       average_gradients=True, traversal=1, fuse_steps=1)
+        got = run(rps_mod, w, b, x0, w.steps, t0=3, kernel=4, average_gradients=True, **opts)
+        assert (got == base).all(), (opts, int((got != base).sum()))
+    # one step, forced to the other kernels' tolerance: the single-step bound
+    one = x0.copy()
+    oracle.run(one, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=3, steps=1,
+               average_gradients=True)
+    got = run(rps_mod, w, b, x0, 1, t0=3, kernel=4, average_gradients=True)
+    assert rel_err(w, got, one) <= (BF16_TOL if dtype == "bf16" else STEP_TOL)
 
 
 def test_a_stream_wait_that_runs_out_is_reported_and_harmless(rps_mod):
