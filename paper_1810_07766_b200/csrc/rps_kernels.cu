@@ -237,7 +237,7 @@ FusedKernel choose_fused_kernel(const FusedParams& prm, const FusedTuning& tune,
     // bf16 replicas of more than 32 workers: workers streamed through the teams' rings (what is staged does not
     // grow with n, every row piece is 2 KB); measured side by side 5 % ahead of the ring kernel at n = 64 and
     // a third at n = 48, level with it or behind at n <= 32.
-    // Tracked steps take it from 32 workers on (0.57 against 0.73 ms per step at n = 32, 1.19 against 1.62 at n = 64).
+    // Tracked steps take it from 32 workers on (0.55 against 0.73 ms per step at n = 32, 1.16 against 1.62 at n = 64).
     // Gradient averaging reads x twice in this form, a third of it from DRAM again at n = 64 (1.25 ms per step against
     // 1.18 for the ring kernel, which holds the tile); the ring kernel's lane groups of 8 workers are full only at
     // n = 64, though: at n = 48 the streamed form is ahead (0.98 against 1.12 ms), so it takes 33..60 workers.

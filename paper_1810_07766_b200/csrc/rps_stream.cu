@@ -23,8 +23,8 @@
 //     fixed turns, so every warp knows the whole sequence of stages in advance.
 //   * The arithmetic runs two columns at a time in the packed fp32 forms (fma / mul / add .f32x2): one issue
 //     slot, two IEEE operations, the same bits as the scalar forms of the other kernels.
-//   * Tracked steps (DIAG) get their sums from the same walk: every receiver holds the same value, so only
-//     the keepers have a deviation from it (see TrackCols).
+//   * Tracked steps (DIAG) need little more than the walk: every receiver holds the same value, so only the
+//     keepers have a deviation from it, and their rows are read back when the tile's average is known.
 //   * One launch can run several consecutive steps (rps_step_n): a team has the same tiles in every step and a
 //     column's next step needs only that column's last step, so a team goes on to the next step by itself once
 //     its own stores are done and fenced.  There is no launch boundary between the steps and no wait for the
@@ -77,27 +77,19 @@ struct StreamShape {
 };
 
 // Tracked steps (distance of the averaged model to the optimum, consensus error; see Tracker in rps_device.cuh),
-// in the streamed form.  Every receiver of a block holds the same stored value P, so with P as the pivot
-// only the workers that keep their own v (down bit clear) have a deviation: per column a lane keeps
-//   the sum of the targets (two columns at a time, with the step: local_sgd_pair_packed),
-//   a0 = v of worker 0 (a provisional pivot, P is not known until the last worker),
-//   D0 = sum over keepers (v_k - a0),  Q0 = sum over keepers (v_k - a0)^2        (v_k as stored),
-// and closes the column with delta = a0 - P, m keepers:  D = D0 + m delta,  Q = Q0 + 2 delta D0 + m delta^2,
+// in the streamed form.  Every receiver of a block holds the same stored value P, so with P as the pivot only
+// the workers that keep their own v (down bit clear, a fraction p of them) have a deviation.  The walk itself
+// carries only the sum of the targets (two columns at a time, with the step: local_sgd_pair_packed).  When a tile's
+// average has been stored the lane reads its keepers' rows back (its own stores of a moment ago) and forms
+//   D = sum over keepers (v_k - P),  Q = sum over keepers (v_k - P)^2          (v_k as stored),
 //   mean x = P + D / n,   consensus = Q - D^2 / n.   Nothing large is squared and subtracted.
-template <int VEC>
-struct TrackCols {
-    float a0[VEC], d0[VEC], q0[VEC];
-};
+// With no receiver at all every worker is a keeper and worker 0's stored value is the pivot.
 
-// One column's contribution to (|| mean x - mean b ||^2, consensus error).  `receivers` = workers that hold
-// `stored_avg`; with none of them the provisional pivot stays.
-__device__ __forceinline__ void close_tracked_column(float bsum, float a0, float d0, float q0, float stored_avg,
-                                                     int keepers, int receivers, float inv_n, float& dist2, float& cons)
+// One column's contribution to (|| mean x - mean b ||^2, consensus error) from the keepers' deviations from the
+// pivot: their sum and the sum of their squares.
+__device__ __forceinline__ void close_tracked_column(float bsum, float pivot, float dev_sum, float dev_sq, float inv_n,
+                                                     float& dist2, float& cons)
 {
-    const float pivot = receivers > 0 ? stored_avg : a0;
-    const float delta = a0 - pivot, m = (float)keepers;
-    const float dev_sum = fmaf(m, delta, d0);
-    const float dev_sq = fmaf(m * delta, delta, fmaf(2.0f * delta, d0, q0));
     const float gap = fmaf(dev_sum - bsum, inv_n, pivot);  // mean x - mean b of this column
     dist2 = fmaf(gap, gap, dist2);
     cons += fmaf(-dev_sum * inv_n, dev_sum, dev_sq);
@@ -109,11 +101,10 @@ __device__ __forceinline__ void close_tracked_column(float bsum, float a0, float
 // Out of line and on copies of the caller's registers: this is rare.
 // `v` is what the sum takes and `own` what a keeper stores: the same values in model averaging, the update and
 // x + the update in gradient averaging.
-template <typename T, int VEC, bool DIAG>
+template <typename T, int VEC>
 __device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[2][VEC], const float (&own)[2][VEC],
                                             int k, int j, int j_next, int cut, int live_n, uint64_t valid,
-                                            const uint64_t* s_up, const uint64_t* s_down, T* dst, int64_t pitch,
-                                            TrackCols<VEC>* track)
+                                            const uint64_t* s_up, const uint64_t* s_down, T* dst, int64_t pitch)
 {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -126,16 +117,7 @@ __device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[
             const bool live = e < live_n, hi = e >= cut;
             add_if(sum[e], v[h][e], live ? (hi ? up_hi : up_lo) : 0u);
             const bool kept = live && (hi ? keep_hi : keep_lo);
-            const T stored = RowVec<T, VEC>::narrow(own[h][e]);
-            if (kept) dst[(int64_t)w * pitch + e] = stored;
-            if (DIAG && live) {
-                if (w == 0) track->a0[e] = own[0][e];
-                if (kept) {
-                    const float dev = (float)stored - track->a0[e];
-                    track->d0[e] += dev;
-                    track->q0[e] = fmaf(dev, dev, track->q0[e]);
-                }
-            }
+            if (kept) dst[(int64_t)w * pitch + e] = RowVec<T, VEC>::narrow(own[h][e]);
         }
     }
 }
@@ -143,8 +125,8 @@ __device__ __noinline__ void irregular_pair(float (&sum)[VEC], const float (&v)[
 template <typename T, int VEC, bool DIAG>
 __device__ __noinline__ void irregular_receivers(const float (&sum)[VEC], int n, int j, int j_next, int cut,
                                                  int live_n, const uint64_t* s_down, const float* s_inv, T* dst,
-                                                 int64_t pitch, const TrackCols<VEC>* track, const float (&target_sum)[VEC],
-                                                 float inv_n, float* dist2, float* cons)
+                                                 int64_t pitch, const float (&target_sum)[VEC], float inv_n,
+                                                 float* dist2, float* cons)
 {
     T avg[VEC];
 #pragma unroll
@@ -158,13 +140,22 @@ __device__ __noinline__ void irregular_receivers(const float (&sum)[VEC], int n,
             if (e < live_n && (e >= cut ? hi : lo)) dst[(int64_t)i * pitch + e] = avg[e];
     }
     if (DIAG) {
+        // the keepers' rows as this lane stored them, against what the receivers hold
+        const uint64_t valid = n >= 64 ? ~(uint64_t)0 : (((uint64_t)1 << n) - 1);
         float dd = 0.0f, q = 0.0f;
 #pragma unroll
         for (int e = 0; e < VEC; ++e)
             if (e < live_n) {
-                const int receivers = __popcll(e >= cut ? down_hi : down_lo);
-                close_tracked_column(target_sum[e], track->a0[e], track->d0[e], track->q0[e], (float)avg[e],
-                                     n - receivers, receivers, inv_n, dd, q);
+                const uint64_t down = (e >= cut ? down_hi : down_lo) & valid;
+                const float pivot = down != 0 ? (float)avg[e] : (float)dst[e];
+                float dev_sum = 0.0f, dev_sq = 0.0f;
+                for (uint64_t rest = ~down & valid; rest != 0; rest &= rest - 1) {
+                    const int i = __ffsll((long long)rest) - 1;
+                    const float dev = (float)dst[(int64_t)i * pitch + e] - pivot;
+                    dev_sum += dev;
+                    dev_sq = fmaf(dev, dev, dev_sq);
+                }
+                close_tracked_column(target_sum[e], pivot, dev_sum, dev_sq, inv_n, dd, q);
             }
         *dist2 = dd, *cons = q;
     }
@@ -428,11 +419,8 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
         Float2 sum[VEC / 2];
 #pragma unroll
         for (int m = 0; m < VEC / 2; ++m) sum[m] = 0ull;  // (+0, +0)
-        TrackCols<VEC> track;
-        Float2 target_sum[VEC / 2];  // tracked, regular lanes: the sum of the targets, two columns at a time
+        Float2 target_sum[VEC / 2];  // tracked: the sum of the targets, two columns at a time
         if (DIAG) {
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) track.a0[e] = track.d0[e] = track.q0[e] = 0.0f;
 #pragma unroll
             for (int m = 0; m < VEC / 2; ++m) target_sum[m] = 0ull;
         }
@@ -458,14 +446,6 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                     for (int m = 0; m < VEC / 2; ++m) add2_if(sum[m], v[0][m], arrived & 1u);
 #pragma unroll
                     for (int m = 0; m < VEC / 2; ++m) add2_if(sum[m], v[1][m], arrived & 2u);
-                    if (DIAG) {
-                        // tracked: the provisional pivot (the targets were summed with the step: rows past n arrive
-                        // as zeros and add nothing)
-                        if (k == 0) {
-#pragma unroll
-                            for (int m = 0; m < VEC / 2; ++m) unpack2(v[0][m], track.a0[2 * m], track.a0[2 * m + 1]);
-                        }
-                    }
                     // AG, the workers whose return message is lost: they keep v, which can go out now
                     if (kept) {
 #pragma unroll
@@ -479,16 +459,6 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                             }
                             const uint4 packed_v = pack_pairs<T, VEC>(v[h]);
                             __stcs(reinterpret_cast<uint4*>(dst + (int64_t)(k + h) * prm.pitch), packed_v);
-                            if (DIAG) {
-                                float stored[VEC];  // as it will read back
-                                RowVec<T, VEC>::unpack(packed_v, stored);
-#pragma unroll
-                                for (int e = 0; e < VEC; ++e) {
-                                    const float dev = stored[e] - track.a0[e];
-                                    track.d0[e] += dev;
-                                    track.q0[e] = fmaf(dev, dev, track.q0[e]);
-                                }
-                            }
                         }
                     }
                 } else {
@@ -499,7 +469,6 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                         unpack2(v[0][m], v_copy[0][2 * m], v_copy[0][2 * m + 1]);
                         unpack2(v[1][m], v_copy[1][2 * m], v_copy[1][2 * m + 1]);
                     }
-                    TrackCols<VEC> track_copy = track;
                     if (GRAD) {
                         float own_copy[2][VEC];
 #pragma unroll
@@ -508,13 +477,12 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
 #pragma unroll
                             for (int e = 0; e < VEC; ++e) own_copy[h][e] += v_copy[h][e];
                         }
-                        irregular_pair<T, VEC, DIAG>(sum_copy, v_copy, own_copy, k, j, j_next, cut, live_n, valid, s_up,
-                                                     s_down, dst, prm.pitch, &track_copy);
+                        irregular_pair<T, VEC>(sum_copy, v_copy, own_copy, k, j, j_next, cut, live_n, valid, s_up, s_down,
+                                               dst, prm.pitch);
                     } else {
-                        irregular_pair<T, VEC, DIAG>(sum_copy, v_copy, v_copy, k, j, j_next, cut, live_n, valid, s_up,
-                                                     s_down, dst, prm.pitch, &track_copy);
+                        irregular_pair<T, VEC>(sum_copy, v_copy, v_copy, k, j, j_next, cut, live_n, valid, s_up, s_down,
+                                               dst, prm.pitch);
                     }
-                    if (DIAG) track = track_copy;
 #pragma unroll
                     for (int m = 0; m < VEC / 2; ++m) sum[m] = pack2(sum_copy[2 * m], sum_copy[2 * m + 1]);
                 }
@@ -603,15 +571,28 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                     if (rest & 1u) __stcs(reinterpret_cast<uint4*>(row), packed);
             }
             if (DIAG && live_n == VEC) {
-                float stored_avg[VEC], targets[VEC], dd = 0.0f, qq = 0.0f;
-                RowVec<T, VEC>::unpack(packed, stored_avg);
+                // the keepers' rows as this lane stored them a moment ago, against what the receivers hold
+                float pivot[VEC], targets[VEC], dev_sum[VEC], dev_sq[VEC], dd = 0.0f, qq = 0.0f;
+                if (down != 0) RowVec<T, VEC>::unpack(packed, pivot);
+                else RowVec<T, VEC>::unpack(__ldcg(reinterpret_cast<const uint4*>(dst)), pivot);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) dev_sum[e] = dev_sq[e] = 0.0f;
+                for (uint64_t rest = keep; rest != 0; rest &= rest - 1) {
+                    const int i = __ffsll((long long)rest) - 1;
+                    float kept_v[VEC];
+                    RowVec<T, VEC>::unpack(__ldcg(reinterpret_cast<const uint4*>(dst + (int64_t)i * prm.pitch)), kept_v);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) {
+                        const float dev = kept_v[e] - pivot[e];
+                        dev_sum[e] += dev;
+                        dev_sq[e] = fmaf(dev, dev, dev_sq[e]);
+                    }
+                }
 #pragma unroll
                 for (int m = 0; m < VEC / 2; ++m) unpack2(target_sum[m], targets[2 * m], targets[2 * m + 1]);
-                const int receivers = __popcll(down);
 #pragma unroll
                 for (int e = 0; e < VEC; ++e)
-                    close_tracked_column(targets[e], track.a0[e], track.d0[e], track.q0[e], stored_avg[e],
-                                         n - receivers, receivers, prm.inv_n, dd, qq);
+                    close_tracked_column(targets[e], pivot[e], dev_sum[e], dev_sq[e], prm.inv_n, dd, qq);
                 tracker.dist2 += (double)dd;
                 tracker.cons += (double)qq;
             }
@@ -619,7 +600,6 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
             float sum_copy[VEC], dd = 0.0f, qq = 0.0f;
 #pragma unroll
             for (int m = 0; m < VEC / 2; ++m) unpack2(sum[m], sum_copy[2 * m], sum_copy[2 * m + 1]);
-            const TrackCols<VEC> track_copy = track;
             float targets[VEC];  // (of the columns that exist: the others hold whatever the padding held)
 #pragma unroll
             for (int m = 0; m < VEC / 2; ++m) {
@@ -627,7 +607,7 @@ __global__ void __launch_bounds__(MAXW * 32, 1)
                 else targets[2 * m] = targets[2 * m + 1] = 0.0f;
             }
             irregular_receivers<T, VEC, DIAG>(sum_copy, n, j, j_next, cut, live_n, s_down, s_inv, dst, prm.pitch,
-                                              &track_copy, targets, prm.inv_n, &dd, &qq);
+                                              targets, prm.inv_n, &dd, &qq);
             if (DIAG) {
                 tracker.dist2 += (double)dd;
                 tracker.cons += (double)qq;
@@ -761,12 +741,12 @@ cudaError_t launch_stream_for_warps(const FusedParams& prm, const FusedTuning& t
     return launch_stream_as<T, VEC, 32, ROWS>(prm, tune, warps, team_warps, steps, sm_count, stream);
 }
 
-// Tracked steps: stages of two worker pairs, 16 warps unless asked otherwise (the per-column sums take
-// registers: 20 warps spill and were 6 % slower at n = 64).
+// Tracked steps: stages of two worker pairs, 20 warps like the plain step (the walk carries only the sum of the
+// targets on top of it; bf16, n = 64: 1.11 ms per launch against 1.16 with 16 warps).
 template <typename T, int VEC>
 cudaError_t launch_stream_tracked(const FusedParams& prm, const FusedTuning& tune, int sm_count, cudaStream_t stream)
 {
-    int warps = tune.consumer_warps > 0 ? tune.consumer_warps : 16;
+    int warps = tune.consumer_warps > 0 ? tune.consumer_warps : 20;
     if (warps > 20) warps = 20;
     int team_warps = tune.team_warps == 0 || tune.team_warps >= 4 ? 4 : (tune.team_warps >= 2 ? 2 : 1);
     while (team_warps > warps) team_warps /= 2;
