@@ -91,7 +91,7 @@ def fused_kernel_name(args, w) -> str:
         return "rps_fused_direct_kernel"
     stream_built = w.n >= 2 and not (args.average_gradients and args.track)
     staged_only = args.workers_per_lane or args.copy_mode or args.slice_bytes
-    wide = 32 < w.n <= 60 if args.average_gradients else w.n > 32 or (args.track and w.n >= 32)
+    wide = 32 < w.n <= 52 if args.average_gradients else w.n > 32 or (args.track and w.n >= 32)
     if stream_built and (args.kernel == 4 or (args.kernel == 0 and w.dtype == "bf16" and wide and not staged_only)):
         return "rps_fused_stream_kernel"
     ring_built = w.dtype == "bf16" and w.n > 4 and not args.track

@@ -112,7 +112,7 @@ typedef struct rps_options {
                                  2 or 3).
                                  0: kernel 1 for models too short to give every SM a tile, kernel 4
                                  for bf16 replicas of more than 32 workers (gradient averaging:
-                                 33 to 60), kernel 3 for bf16 replicas of more than 4 workers
+                                 33 to 52), kernel 3 for bf16 replicas of more than 4 workers
                                  (unless an option that shapes kernel 2 alone is set), else
                                  kernel 2                                                     */
     int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */

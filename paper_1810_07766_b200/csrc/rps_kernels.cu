@@ -240,8 +240,9 @@ FusedKernel choose_fused_kernel(const FusedParams& prm, const FusedTuning& tune,
     // Tracked steps take it from 32 workers on (0.55 against 0.73 ms per step at n = 32, 1.16 against 1.62 at n = 64).
     // Gradient averaging reads x twice in this form, a third of it from DRAM again at n = 64 (1.25 ms per step against
     // 1.18 for the ring kernel, which holds the tile); the ring kernel's lane groups of 8 workers are full only at
-    // n = 64, though: at n = 48 the streamed form is ahead (0.98 against 1.12 ms), so it takes 33..60 workers.
-    const bool many_workers = prm.average_gradients ? (prm.n > 32 && prm.n <= 60)
+    // n = 64, though, and take 1.11-1.19 ms from n = 40 on: the streamed form is ahead up to n = 48 (0.83 against 1.11 ms
+    // at n = 40, 0.98 against 1.12 at 48) and level at 56 (1.17 against 1.15), so it takes 33..52 workers.
+    const bool many_workers = prm.average_gradients ? (prm.n > 32 && prm.n <= 52)
                                                     : (prm.n > 32 || (prm.trace != nullptr && prm.n >= 32));
     if (tune.kernel == 0 && bf16 && many_workers && stream_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 &&
         tune.copy_mode == 0 && tune.slice_bytes == 0)

@@ -96,8 +96,8 @@ def test_ring_gradient_averaging_matches_the_oracle(rps_mod, oracle, n, d):
         got = run(rps_mod, w, b, x0, w.steps, t0=3, kernel=3, average_gradients=True, team_warps=team_warps,
                   stages=stages, traversal=traversal)
         assert (got == ref).all(), (team_warps, stages, traversal)
-    # the library's own choice for this step: the same kernel, except the streamed one from 33 to 60 workers
-    if 32 < n <= 60:
+    # the library's own choice for this step: the same kernel, except the streamed one from 33 to 52 workers
+    if 32 < n <= 52:
         ref = run(rps_mod, w, b, x0, w.steps, t0=3, kernel=4, average_gradients=True)
     assert (run(rps_mod, w, b, x0, w.steps, t0=3, average_gradients=True) == ref).all()
 

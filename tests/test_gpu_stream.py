@@ -135,14 +135,16 @@ def test_stream_forced_masks_every_pattern(rps_mod, oracle, n):
     r.close()
 
 
-def test_stream_shards_reproduce_the_whole_model(rps_mod):
+@pytest.mark.parametrize("average_gradients", [False, True])
+def test_stream_shards_reproduce_the_whole_model(rps_mod, average_gradients):
     for dtype, n, d in (("bf16", 64, 200_017), ("f32", 10, 150_001)):
         w = wl.Workload("stream", n=n, d=d, dtype=dtype, p=0.1, gamma=0.02, sigma=0.1, seed=77, steps=5)
         b = wl.make_targets(w)
         x0 = start(w, 5)
-        ref = run(rps_mod, w, b, x0, w.steps, kernel=4)
+        ref = run(rps_mod, w, b, x0, w.steps, kernel=4, average_gradients=average_gradients)
         pieces = [(0, 64_000), (64_000, 36_032), (100_032, d - 100_032)]
-        parts = [run(rps_mod, w, b, x0, w.steps, shard=piece, kernel=4) for piece in pieces]
+        parts = [run(rps_mod, w, b, x0, w.steps, shard=piece, kernel=4, average_gradients=average_gradients)
+                 for piece in pieces]
         assert (np.concatenate(parts, axis=1) == ref).all()
 
 
