@@ -89,10 +89,23 @@ def fused_kernel_name(args, w) -> str:
     small = w.n * w.d * w.elem_bytes < 148 * 8192
     if args.kernel == 1 or (args.kernel == 0 and small):
         return "rps_fused_direct_kernel"
-    stream_built = w.n >= 2 and not (args.average_gradients and args.track)
+    block_cols = -(-w.d // w.n)
+    stream_built = (w.n >= 2 and not (args.average_gradients and args.track)
+                    and block_cols >= (8 if w.dtype == "bf16" else 4))
     staged_only = args.workers_per_lane or args.copy_mode or args.slice_bytes
-    wide = 32 < w.n <= 52 if args.average_gradients else w.n > 32 or (args.track and w.n >= 32)
-    if stream_built and (args.kernel == 4 or (args.kernel == 0 and w.dtype == "bf16" and wide and not staged_only)):
+    power_of_two = w.n & (w.n - 1) == 0
+    padded = 8
+    while padded < w.n:
+        padded *= 2
+    if w.dtype != "bf16":
+        streamed = not power_of_two
+    elif args.track:
+        streamed = True
+    elif args.average_gradients:
+        streamed = w.n < 5 or (w.n >= 9 and 5 * w.n <= 4 * padded)
+    else:
+        streamed = not power_of_two or w.n > 32 or w.n < 8
+    if stream_built and (args.kernel == 4 or (args.kernel == 0 and streamed and not staged_only)):
         return "rps_fused_stream_kernel"
     ring_built = w.dtype == "bf16" and w.n > 4 and not args.track
     staged_only = args.workers_per_lane or args.consumer_warps or args.copy_mode or args.slice_bytes

@@ -110,11 +110,17 @@ typedef struct rps_options {
                                  the receivers (n >= 2, blocks of at least 16 bytes, tracked
                                  steps in model averaging only; any other step runs as kernel
                                  2 or 3).
-                                 0: kernel 1 for models too short to give every SM a tile, kernel 4
-                                 for bf16 replicas of more than 32 workers (gradient averaging:
-                                 33 to 52), kernel 3 for bf16 replicas of more than 4 workers
-                                 (unless an option that shapes kernel 2 alone is set), else
-                                 kernel 2                                                     */
+                                 0: kernel 1 for models too short to give every SM a tile.  Else
+                                 kernel 4 where n is not a power of two (kernels 2 and 3 pad their
+                                 lane groups to the next one and take as long as that many workers
+                                 would), for bf16 replicas of fewer than 8 or more than 32 workers
+                                 and for tracked bf16 steps; gradient averaging on bf16 replicas
+                                 takes kernel 4 only below 5 workers and, from 9 on, where n is at
+                                 most four fifths of the next power of two.  Else kernel 3 for
+                                 bf16 replicas (5 workers or more, untracked) and kernel 2 for the
+                                 rest (fp32 with 2, 4, 8, 16, 32, 64 workers).  An option that
+                                 shapes kernel 2 alone (workers_per_lane, copy_mode, slice_bytes)
+                                 keeps kernels 3 and 4 out of the choice.                      */
     int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */
     int32_t stages;           /* depth of the shared-memory ring(s) of kernels 2, 3 and 4 (2..8) */
     int32_t consumer_warps;   /* compute warps per CTA of kernel 2 (1..24; shapes that need

@@ -234,19 +234,33 @@ FusedKernel choose_fused_kernel(const FusedParams& prm, const FusedTuning& tune,
         const int64_t bytes_per_column = (int64_t)prm.n * (bf16 ? 2 : 4);
         if (prm.d * bytes_per_column < (int64_t)sm_count * 8192) return FusedKernel::kDirect;
     }
-    // bf16 replicas of more than 32 workers: workers streamed through the teams' rings (what is staged does not
-    // grow with n, every row piece is 2 KB); measured side by side 5 % ahead of the ring kernel at n = 64 and
-    // a third at n = 48, level with it or behind at n <= 32.
-    // Tracked steps take it from 32 workers on (0.55 against 0.73 ms per step at n = 32, 1.16 against 1.62 at n = 64).
-    // Gradient averaging reads x twice in this form, a third of it from DRAM again at n = 64 (1.25 ms per step against
-    // 1.18 for the ring kernel, which holds the tile); the ring kernel's lane groups of 8 workers are full only at
-    // n = 64, though, and take 1.11-1.19 ms from n = 40 on: the streamed form is ahead up to n = 48 (0.83 against 1.11 ms
-    // at n = 40, 0.98 against 1.12 at 48) and level at 56 (1.17 against 1.15), so it takes 33..52 workers.
-    const bool many_workers = prm.average_gradients ? (prm.n > 32 && prm.n <= 52)
-                                                    : (prm.n > 32 || (prm.trace != nullptr && prm.n >= 32));
-    if (tune.kernel == 0 && bf16 && many_workers && stream_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 &&
-        tune.copy_mode == 0 && tune.slice_bytes == 0)
-        return FusedKernel::kStream;
+    // Workers streamed through the teams' rings (what is staged does not grow with n, every row piece is 2 KB).  The
+    // lane groups of the staged and ring kernels hold 4 or 8 workers per lane times a power of two of lanes, so a
+    // worker count between two powers of two runs at the speed of the next one; the streamed kernel's time is
+    // proportional to n.  Measured side by side (ms per step, bf16 d = 16.8 M / fp32 d = 4 M; lane-group form first):
+    //   bf16 plain   n = 8 0.126 / 0.128, 16 0.247 / 0.247, 32 0.489 / 0.499; 2 0.079 / 0.048, 4 0.099 / 0.073,
+    //                6 0.125 / 0.111, 12 0.247 / 0.193, 20 0.489 / 0.322, 28 0.488 / 0.456, 48 1.33x, 64 0.95x
+    //   bf16 tracked streamed ahead at every n from 2 (0.092 / 0.061) to 64 (1.62 / 1.16)
+    //   fp32         n = 8, 16, 32 staged ahead by 2-9 %; 12 0.100 / 0.083, 20 0.187 / 0.146, 24 0.199 / 0.178,
+    //                48 0.418 / 0.364, tracked and gradient averaging likewise
+    // Gradient averaging reads x twice in this form, part of it from DRAM again when n is large (n = 64: 1.25 ms
+    // against 1.18 for the ring kernel, which holds the tile), so there it is taken only where the ring kernel's
+    // lane groups are at most four fifths full: 10 0.269 / 0.225, 12 0.269 / 0.256, 20 0.546 / 0.422,
+    // 24 0.548 / 0.499, 28 0.548 / 0.581, 40 1.115 / 0.826, 48 1.12 / 0.98, 56 1.155 / 1.173; and below 5 workers,
+    // which the ring kernel does not take (4 0.105 / 0.092).
+    if (tune.kernel == 0 && stream_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 && tune.copy_mode == 0 &&
+        tune.slice_bytes == 0) {
+        const int n = prm.n;
+        const bool power_of_two = (n & (n - 1)) == 0;
+        int padded = 8;  // what the ring kernel's lane groups pad n to
+        while (padded < n) padded *= 2;
+        bool streamed;
+        if (!bf16) streamed = !power_of_two;
+        else if (prm.trace != nullptr) streamed = true;
+        else if (prm.average_gradients) streamed = n < 5 || (n >= 9 && 5 * n <= 4 * padded);
+        else streamed = !power_of_two || n > 32 || n < 8;
+        if (streamed) return FusedKernel::kStream;
+    }
     // bf16 replicas of more than 4 workers: the self-refilling ring (16 compute warps, no producer warp), unless an
     // option that shapes the staged kernel only was set.  Measured side by side it is 3-8 % ahead at every n.
     if (tune.kernel == 0 && bf16 && ring_kernel_covers(prm, bf16) && tune.workers_per_lane == 0 &&

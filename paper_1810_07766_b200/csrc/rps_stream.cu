@@ -32,7 +32,8 @@
 //
 //   * Gradient averaging (GRAD) sums the updates v - x instead, and a receiver's new value x + (average update)
 //     needs its own x after the last worker: the tile's rows of x go through the ring a second time, last rows
-//     first (what was read last is still in L2), and each receiver's row is finished then.  Keepers are stored in the first pass as always.
+//     first (what was read last is still in L2), and each receiver's row is finished then.  Keepers are stored
+//     in the first pass as always.
 //
 // A lane whose slice straddles two blocks or the end of the row (at most n such lanes per step) takes a
 // per-column branch with the same arithmetic, so a column's result does not depend on where it lies.
@@ -73,7 +74,6 @@ struct StreamShape {
     int32_t early_targets;    // 1: the first stages' copies of b are issued before the wait for the kernel ahead in the stream
     uint32_t out_offset;      // of the warps' output slots from the start of the rings
     uint64_t wait_limit_ns;
-
 };
 
 // Tracked steps (distance of the averaged model to the optimum, consensus error; see Tracker in rps_device.cuh),

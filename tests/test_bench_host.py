@@ -150,5 +150,12 @@ def test_default_suite_and_kernel_names():
     args.track, args.average_gradients = False, True
     assert bench.fused_kernel_name(args, wl.WORKLOADS["cfg5"]) == "rps_fused_ring_kernel"
     assert bench.fused_kernel_name(args, replace(wl.WORKLOADS["cfg5"], n=48)) == "rps_fused_stream_kernel"
+    assert bench.fused_kernel_name(args, replace(wl.WORKLOADS["cfg5"], n=56)) == "rps_fused_ring_kernel"
+    args.average_gradients = False
+    # between two powers of two the streamed kernel serves both types
+    assert bench.fused_kernel_name(args, replace(wl.WORKLOADS["cfg5"], n=24)) == "rps_fused_stream_kernel"
+    assert bench.fused_kernel_name(args, replace(wl.WORKLOADS["cfg4"], n=24)) == "rps_fused_stream_kernel"
+    assert bench.fused_kernel_name(args, replace(wl.WORKLOADS["cfg5"], n=16)) == "rps_fused_ring_kernel"
+    assert bench.fused_kernel_name(args, replace(wl.WORKLOADS["cfg5"], n=4)) == "rps_fused_stream_kernel"
     w = bench.resolve_workload(argparse.Namespace(d=1000, sigma=0.0, n=6), "cfg2", p=0.3)
     assert (w.n, w.d, w.p, w.sigma, w.gamma, w.seed) == (6, 1000, 0.3, 0.0, 0.05, 1)

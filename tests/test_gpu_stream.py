@@ -329,3 +329,24 @@ def test_fused_launches_are_counted_and_tracked_steps_stay_single(rps_mod):
     r.step_n(5)   # three tracked steps singly, then two in one launch (no new masks: steps 40..44 of the window 32..63)
     assert r.launch_count() - before == 4 and r.read_trace().shape == (3, 2)
     r.close()
+
+
+@pytest.mark.parametrize("dtype,n,d,extra,kernel", [
+    ("f32", 12, 70_001, {}, 4), ("f32", 16, 70_001, {}, 2), ("f32", 6, 100_003, dict(average_gradients=True), 4),
+    ("bf16", 24, 70_001, {}, 4), ("bf16", 16, 100_003, {}, 3), ("bf16", 4, 200_003, {}, 4), ("bf16", 64, 50_001, {}, 4),
+    ("bf16", 12, 100_003, dict(average_gradients=True), 4), ("bf16", 28, 70_001, dict(average_gradients=True), 3),
+    ("bf16", 3, 300_007, dict(average_gradients=True), 4), ("bf16", 64, 50_001, dict(average_gradients=True), 3),
+])
+def test_the_librarys_own_choice_of_kernel(rps_mod, dtype, n, d, extra, kernel):
+    """The lane groups of the staged and ring kernels are padded to a power of two of workers, the streamed kernel's
+    time is proportional to n: left to itself the library takes the streamed kernel between two powers of two (and
+    for bf16 replicas of fewer than 8 or more than 32 workers), the others where their groups are full.  Seen in
+    the bits: the summation order differs between the forms."""
+    w = wl.Workload("choice", n=n, d=d, dtype=dtype, p=0.2, gamma=0.05, sigma=0.1, seed=40 + n, steps=3)
+    b = wl.make_targets(w)
+    x0 = start(w, 8)
+    own = run(rps_mod, w, b, x0, w.steps, strict_padding=kernel == 4, **extra)  # (only the streamed kernel never writes padding)
+    assert (own == run(rps_mod, w, b, x0, w.steps, strict_padding=False, kernel=kernel, **extra)).all()
+    if n > 4:  # with up to 4 workers every form adds them up in the same order
+        others = [k for k in (2, 3, 4) if k != kernel and not (k == 3 and dtype == "f32")]
+        assert any((own != run(rps_mod, w, b, x0, w.steps, strict_padding=False, kernel=k, **extra)).any() for k in others)
