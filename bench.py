@@ -98,7 +98,7 @@ def fused_kernel_name(args, w) -> str:
     while padded < w.n:
         padded *= 2
     if w.dtype != "bf16":
-        streamed = not power_of_two
+        streamed = not power_of_two or (not args.average_gradients and (w.n == 2 or (w.n == 4 and args.track)))
     elif args.track:
         streamed = True
     elif args.average_gradients:

@@ -118,7 +118,8 @@ typedef struct rps_options {
                                  takes kernel 4 only below 5 workers and, from 9 on, where n is at
                                  most four fifths of the next power of two.  Else kernel 3 for
                                  bf16 replicas (5 workers or more, untracked) and kernel 2 for the
-                                 rest (fp32 with 2, 4, 8, 16, 32, 64 workers).  An option that
+                                 rest (fp32 with 4, 8, 16, 32, 64 workers; 2 workers run as kernel 4
+                                 in model averaging, 4 workers when tracked).  An option that
                                  shapes kernel 2 alone (workers_per_lane, copy_mode, slice_bytes)
                                  keeps kernels 3 and 4 out of the choice.                      */
     int32_t workers_per_lane; /* 2, 4 or 8 workers' slices held in registers by one lane      */

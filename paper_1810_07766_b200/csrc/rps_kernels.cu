@@ -242,7 +242,8 @@ FusedKernel choose_fused_kernel(const FusedParams& prm, const FusedTuning& tune,
     //                6 0.125 / 0.111, 12 0.247 / 0.193, 20 0.489 / 0.322, 28 0.488 / 0.456, 48 1.33x, 64 0.95x
     //   bf16 tracked streamed ahead at every n from 2 (0.092 / 0.061) to 64 (1.62 / 1.16)
     //   fp32         n = 8, 16, 32 staged ahead by 2-9 %; 12 0.100 / 0.083, 20 0.187 / 0.146, 24 0.199 / 0.178,
-    //                48 0.418 / 0.364, tracked and gradient averaging likewise
+    //                48 0.418 / 0.364, tracked and gradient averaging likewise; at d = 25.6 M: 2 0.147 / 0.105
+    //                (tracked 0.166 / 0.130), 4 0.181 / 0.190 (tracked 0.213 / 0.193), 12 0.609 / 0.579
     // Gradient averaging reads x twice in this form, part of it from DRAM again when n is large (n = 64: 1.25 ms
     // against 1.18 for the ring kernel, which holds the tile), so there it is taken only where the ring kernel's
     // lane groups are at most four fifths full: 10 0.269 / 0.225, 12 0.269 / 0.256, 20 0.546 / 0.422,
@@ -255,7 +256,7 @@ FusedKernel choose_fused_kernel(const FusedParams& prm, const FusedTuning& tune,
         int padded = 8;  // what the ring kernel's lane groups pad n to
         while (padded < n) padded *= 2;
         bool streamed;
-        if (!bf16) streamed = !power_of_two;
+        if (!bf16) streamed = !power_of_two || (!prm.average_gradients && (n == 2 || (n == 4 && prm.trace != nullptr)));
         else if (prm.trace != nullptr) streamed = true;
         else if (prm.average_gradients) streamed = n < 5 || (n >= 9 && 5 * n <= 4 * padded);
         else streamed = !power_of_two || n > 32 || n < 8;

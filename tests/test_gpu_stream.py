@@ -333,6 +333,7 @@ def test_fused_launches_are_counted_and_tracked_steps_stay_single(rps_mod):
 
 @pytest.mark.parametrize("dtype,n,d,extra,kernel", [
     ("f32", 12, 70_001, {}, 4), ("f32", 16, 70_001, {}, 2), ("f32", 6, 100_003, dict(average_gradients=True), 4),
+    ("f32", 2, 300_007, {}, 4),
     ("bf16", 24, 70_001, {}, 4), ("bf16", 16, 100_003, {}, 3), ("bf16", 4, 200_003, {}, 4), ("bf16", 64, 50_001, {}, 4),
     ("bf16", 12, 100_003, dict(average_gradients=True), 4), ("bf16", 28, 70_001, dict(average_gradients=True), 3),
     ("bf16", 3, 300_007, dict(average_gradients=True), 4), ("bf16", 64, 50_001, dict(average_gradients=True), 3),
