@@ -43,11 +43,11 @@ FALLBACK_HBM_GBS = 6650.0
 # algorithmic bytes.  "cold_bytes_per_launch": one launch alone at full size with the caches flushed first
 # (also a one-pass capture; the writes of the last lines are still in L2 when the launch ends).  Both are bytes PER
 # STEP: cfg5's steps go out several per launch, and its figure is one launch of 32 steps divided by 32 (one step per
-# launch, --fuse-steps 1, moves the same: 6,414,654,848 B).
+# launch, --fuse-steps 1, moves the same: 6,414,896,384 B).
 NCU_TRAFFIC = {
-    "kernel_digest": "8f62f761f26c9d7b",
-    "bytes_per_launch": {"cfg2": 954717466, "cfg3": 4800623795, "cfg4": 1430456755, "cfg5": 6413626536},
-    "cold_bytes_per_launch": {"cfg2": 1020613888, "cfg3": 4859930368, "cfg4": 1487139840, "cfg5": 6387704064},
+    "kernel_digest": "fa57c8c79867b80b",
+    "bytes_per_launch": {"cfg2": 962904755, "cfg3": 4808150886, "cfg4": 1431978445, "cfg5": 6413386088},
+    "cold_bytes_per_launch": {"cfg2": 1020994304, "cfg3": 4860927488, "cfg4": 1486595328, "cfg5": 6387756800},
 }
 
 
