@@ -139,6 +139,7 @@ class ClockSampler:
         self.samples, self.reason_bits, self.power_w = [], 0, []
         self.max_mhz = None
         self._stop = threading.Event()
+        self._ready = threading.Event()
         self._thread = None
         self._nvml = None
 
@@ -152,6 +153,7 @@ class ClockSampler:
             self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._dev, pynvml.NVML_CLOCK_SM))
             self._thread = threading.Thread(target=self._run, daemon=True)
             self._thread.start()
+            self._ready.wait(timeout=2.0)
         except Exception:
             self._nvml = None
         return self
@@ -165,6 +167,13 @@ class ClockSampler:
 
     def _run(self):
         nv = self._nvml
+        try:  # the first queries of a process can take tens of milliseconds: make them before the region starts
+            nv.nvmlDeviceGetClockInfo(self._dev, nv.NVML_CLOCK_SM)
+            self._reasons()
+            nv.nvmlDeviceGetPowerUsage(self._dev)
+        except Exception:
+            pass
+        self._ready.set()
         while not self._stop.is_set():
             try:
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._dev, nv.NVML_CLOCK_SM)))
