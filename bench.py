@@ -297,10 +297,11 @@ def resolve_workload(args, name, p=None):
 def measure(args, ctx, w, b, *, with_e2e, with_upwards, p_sweep=()):
     """Times one workload on this rank's GPU.  Returns its entry of the JSON line.
 
-    Pass 1 brackets every launch with events (per-kernel durations; this serialises what the programmatic launch
-    overlap hides, so the mean launch can be longer than the step it is part of), pass 2 is W warm-up steps and
-    exactly K timed steps, pass 3 (optional) the same steps through the host-buffer call.  `p_sweep`: further drop
-    probabilities timed on the same arrays (pass 2 only).
+    Pass 1 is W warm-up steps and exactly K timed steps (first, so that nothing but the warm-up precedes the timed
+    steps: the largest workload reaches the board's power cap some 50 ms into a run), pass 2 brackets every launch
+    with events (per-kernel durations; this serialises what the programmatic launch overlap hides, so the mean
+    launch can be longer than the step it is part of; it starts after a second of idle, from the power state pass 1
+    started from), pass 3 (optional) the same steps through the host-buffer call.  `p_sweep`: further drop probabilities timed on the same arrays (pass 1 only).
     """
     import numpy as np
 
@@ -336,16 +337,18 @@ def measure(args, ctx, w, b, *, with_e2e, with_upwards, p_sweep=()):
         return ms, r.launch_count() - before
 
     r = make(w.p)
-    # the clocks are sampled from here to the end of the timed steps: an NVML query takes milliseconds, so
-    # the timed region alone (tens of milliseconds) would yield a single sample
+    # the clocks are sampled over the warm-up and the timed steps (an NVML query takes a millisecond or so)
     with ClockSampler(local_rank) as clocks:
-        r.step_n(max(args.warmup, 3))
-        r.profile(True)
-        profile_steps = max(args.steps, mask_window + 1)  # long enough to see the mask kernel, which runs once per window
-        r.step_n(profile_steps)
-        fused_ms, fused_n, mask_ms, mask_n = r.profile_read()
-        r.profile(False)
         total_ms, gpu_launches = timed_run(r)
+    # a second of idle, so that the next pass starts from the power state the first one started from
+    torch.cuda.synchronize(device)
+    time.sleep(1.0)
+    r.step_n(max(args.warmup, 3))
+    r.profile(True)
+    profile_steps = max(args.steps, mask_window + 1)  # long enough to see the mask kernel, which runs once per window
+    r.step_n(profile_steps)
+    fused_ms, fused_n, mask_ms, mask_n = r.profile_read()
+    r.profile(False)
 
     e2e = None
     if with_e2e:
