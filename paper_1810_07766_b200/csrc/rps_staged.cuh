@@ -454,7 +454,13 @@ bool shape_for(const FusedParams& prm, const FusedTuning& tune, int vec, int g, 
     // double-buffered output tile (2), or in place from the stage by a store warp (3) where shared memory
     // is too scarce for output tiles (8 workers per lane).  In place needs the box layout.
     const int store_mode = tune.store_mode != 0 ? tune.store_mode : default_store_mode;
-    const int mode = store_mode == 3 ? 2 : (tune.copy_mode != 0 ? tune.copy_mode : (prm.n > 16 ? 2 : 1));
+    int mode = store_mode == 3 ? 2 : (tune.copy_mode != 0 ? tune.copy_mode : (prm.n > 16 ? 2 : 1));
+    // Lane groups of 16 lanes on fp32 replicas (a warp is 8 columns wide: 2 or 4 workers per lane with more than 16
+    // or 32 workers, shapes only an explicit workers_per_lane reaches in plain steps) gave wrong sums in the first
+    // tiles of a CTA when their stages were filled by box copies and handed back before the results were stored;
+    // filled by row copies, or held until the store warp has sent them (in place), they are right.  The cause is
+    // not understood, so these shapes take row copies whatever was asked for.
+    if (g == 16 && elem == 4 && store_mode != 3) mode = 1;
     sh.use_boxes = mode == 2;
     if (sh.use_boxes) {
         sh.box_cols = box_cols;

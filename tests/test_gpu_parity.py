@@ -605,3 +605,38 @@ def test_traversal_and_l2_policy_do_not_change_results(rps_mod):
             r.close()
         for other in out[1:]:
             assert (other == out[0]).all()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("workers_per_lane,n,warps", [(2, 24, 4), (2, 31, 16), (2, 32, 8), (4, 33, 16), (4, 64, 4),
+                                                      (4, 64, 16)])
+def test_staged_lane_groups_of_sixteen_lanes(rps_mod, oracle, dtype, workers_per_lane, n, warps):
+    """The widest lane groups of the staged kernel (16 lanes: 2 workers per lane with more than 16 workers, 4 with
+    more than 32; a warp is then only 8 fp32 columns wide) in every way of filling and emptying a stage, whole and
+    as a shard, against the oracle: every element, and twice (a stage read before it had landed shows only in the
+    first tiles of a CTA and not in every run)."""
+    d = 70_003
+    w = wl.Workload("wide", n=n, d=d, dtype=dtype, p=0.2, gamma=0.05, sigma=0.1, seed=60 + n, steps=2, hetero=True)
+    b = wl.make_targets(w)
+    x0 = np.random.default_rng(n).standard_normal((n, d)).astype(np.float32)
+    if dtype == "bf16":
+        x0 = wl.f32_to_bf16_bits(x0)
+    want = x0.copy()
+    oracle.run(want, b, dtype=dtype, gamma=w.gamma, sigma=w.sigma, p=w.p, seed=w.seed, t0=5, steps=w.steps)
+    for store_mode, copy_mode, shard in ((0, 0, None), (1, 2, None), (2, 2, (11_072, 52_193)), (3, 0, None),
+                                         (2, 1, (11_072, 52_193))):
+        begin, cols = shard if shard else (0, d)
+        for _ in range(2):
+            r = rps_mod.RPS(n, d, w.p, w.gamma, w.seed, dtype=dtype, sigma=w.sigma, kernel=2,
+                            workers_per_lane=workers_per_lane, consumer_warps=warps, store_mode=store_mode,
+                            copy_mode=copy_mode, shard_begin=begin if shard else 0, shard_cols=cols if shard else 0)
+            r.set_targets(np.ascontiguousarray(b[:, begin:begin + cols]))
+            r.write(np.ascontiguousarray(x0[:, begin:begin + cols]))
+            r.set_step(5)
+            r.step_n(w.steps)
+            got = r.read()
+            r.close()
+            g = wl.as_float64(w, got)
+            o = wl.as_float64(w, np.ascontiguousarray(want[:, begin:begin + cols]))
+            err = (np.abs(g - o) / (1.0 + np.abs(o))).max()
+            assert err <= (1e-2 if dtype == "bf16" else 1e-5), (store_mode, copy_mode, shard, float(err))
