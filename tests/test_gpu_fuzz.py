@@ -21,6 +21,16 @@ def rps_mod():
     return binding
 
 
+def bf16_tolerance(case, steps):
+    """1e-2, the tolerance of a bf16 step.  Where the replicas are not pulled together (gradient averaging; nine
+    messages in ten lost, or all), a stored bf16 value that was rounded the other way than the oracle's is never
+    contracted away, and the differences add up like a random walk over the steps: on one seeded case every fused
+    kernel, the direct one included, gives the same 7.8e-3 after 5 steps and 1.3e-2 after 7 (two ulps of a value
+    just below 2); over 4000 more seeds the largest was 2.1e-2 after 8 steps."""
+    loose = case["average_gradients"] or case["p"] >= 0.9
+    return 1e-2 * max(1.0, steps / 3) if loose else 1e-2
+
+
 def draw_case(rng):
     n = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 9, 15, 16, 17, 31, 32, 33, 48, 63, 64]))
     d = int(rng.choice([1, 2, 5, 63, 64, 65, 257, 1000, 4099, 20_011, 70_003]))
@@ -81,7 +91,7 @@ def test_random_options_against_the_oracle(rps_mod, oracle, index):
     r.close()
     g = wl.as_float64(w, got)
     o = wl.as_float64(w, np.ascontiguousarray(want[:, begin:begin + cols]))
-    tol = 1e-2 if dtype == "bf16" else 1e-5
+    tol = bf16_tolerance(case, w.steps) if dtype == "bf16" else 1e-5
     err = np.abs(g - o) / (1.0 + np.abs(o))
     assert err.max() <= tol, (case, opts, shard, float(err.max()))
 
@@ -147,11 +157,6 @@ def test_random_options_of_the_ring_and_streamed_kernels_against_the_oracle(rps_
     r.close()
     g = wl.as_float64(w, got)
     o = wl.as_float64(w, np.ascontiguousarray(want[:, begin:begin + cols]))
-    tol = 1e-2 if dtype == "bf16" else 1e-5
-    if dtype == "bf16" and case["average_gradients"]:
-        # Gradient averaging does not pull the replicas together, so a rounding of the stored bf16 value that goes
-        # the other way than the oracle's is never contracted away: the differences add up like a random walk over
-        # the steps (all four kernels give the same 1.3e-2 after 7 steps where 5 steps give 7.8e-3).
-        tol *= max(1.0, w.steps / 4)
+    tol = bf16_tolerance(case, w.steps) if dtype == "bf16" else 1e-5
     err = np.abs(g - o) / (1.0 + np.abs(o))
     assert err.max() <= tol, (case, opts, shard, float(err.max()))
