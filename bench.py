@@ -43,11 +43,11 @@ FALLBACK_HBM_GBS = 6650.0
 # algorithmic bytes.  "cold_bytes_per_launch": one launch alone at full size with the caches flushed first
 # (also a one-pass capture; the writes of the last lines are still in L2 when the launch ends).  Both are bytes PER
 # STEP: cfg5's steps go out several per launch, and its figure is one launch of 32 steps divided by 32 (one step per
-# launch, --fuse-steps 1, moves the same: 6,414,896,384 B).
+# launch, --fuse-steps 1, moves the same: 6,415,262,182 B).
 NCU_TRAFFIC = {
-    "kernel_digest": "fa57c8c79867b80b",
-    "bytes_per_launch": {"cfg2": 962904755, "cfg3": 4808150886, "cfg4": 1431978445, "cfg5": 6413386088},
-    "cold_bytes_per_launch": {"cfg2": 1020994304, "cfg3": 4860927488, "cfg4": 1486595328, "cfg5": 6387756800},
+    "kernel_digest": "0aeaffc63f21b5c0",
+    "bytes_per_launch": {"cfg2": 962079770, "cfg3": 4805608013, "cfg4": 1425085158, "cfg5": 6411869744},
+    "cold_bytes_per_launch": {"cfg2": 1020622080, "cfg3": 4859442944, "cfg4": 1488037376, "cfg5": 6387771392},
 }
 
 
