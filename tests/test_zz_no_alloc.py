@@ -9,6 +9,7 @@ tolerance), with the device's free memory unchanged across the calls.  It lives 
 last, so a failure here cannot hide the results of the other tests.
 """
 import gc
+from dataclasses import replace
 
 import numpy as np
 import pytest
@@ -21,14 +22,18 @@ pytestmark = pytest.mark.gpu
 STEP_TOL = 1e-6
 
 
-@pytest.mark.parametrize("name,d", [("cfg2", 100_010), ("cfg4", 50_001), ("cfg5", 32_768)])
-def test_static_step_matches_the_bound_step_twice_in_a_row(name, d, oracle):
+@pytest.mark.parametrize("name,d,n", [("cfg2", 100_010, None), ("cfg4", 50_001, None), ("cfg5", 32_768, None),
+                                      # worker counts between two powers of two: the streamed kernel, both types
+                                      ("cfg5", 40_008, 24), ("cfg4", 60_004, 12), ("cfg5", 30_001, 5)])
+def test_static_step_matches_the_bound_step_twice_in_a_row(name, d, n, oracle):
     if not torch.cuda.is_available():
         pytest.fail("this test needs a CUDA device")
     from paper_1810_07766_b200 import binding, build
 
     build.build()
     w = wl.WORKLOADS[name].scaled(d=d, steps=2)
+    if n is not None:
+        w = replace(w, n=n)
     b = wl.make_targets(w)
 
     # the existing path: a handle with caller-lent scratch
